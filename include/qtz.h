@@ -1,0 +1,243 @@
+/*
+ * qtz.h -- C ABI of libqtz: integer-only inference of quantized convolution layers
+ * under uniform affine quantization, for NVIDIA B200 (sm_100a).
+ *
+ * The operations follow R. Krishnamoorthi, "Quantizing deep convolutional networks
+ * for efficient inference: A whitepaper" (2018); every entry point names the section
+ * or equation that defines what it computes.
+ *
+ * Conventions
+ *  - Every call returns a qtz_status: 0 on success, a negative code otherwise.  Nothing
+ *    throws or aborts.  After QTZ_ERR_CUDA, qtz_last_error() describes the CUDA failure.
+ *  - Pointers named *_dev are device pointers on the handle's device, *_host are host
+ *    pointers.  The caller owns every buffer it passes.  The library owns only what
+ *    qtz_create / qtz_conv_create return, until the matching destroy call.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
+ *    enqueued on it and the call returns without waiting, except where stated.
+ *  - Calls that share one handle or one plan must be issued in stream order on ONE stream
+ *    at a time: the handle and the plans hold small device scratch buffers that
+ *    consecutive calls reuse.
+ *  - Activations are uint8, NHWC, with a channel pitch: pixel p, channel c lives at
+ *    base[p * c_pitch + c].  Pitches are multiples of 16 and base pointers 16-byte
+ *    aligned (else QTZ_ERR_MISALIGNED).  Bytes in [c, c_pitch) are never read as data;
+ *    outputs leave them unspecified.
+ *  - Tensors handed to calibrate / quantize / dequantize are viewed as
+ *    x[outer][axis_len][inner] (row-major); one quantizer per index of the middle axis.
+ *    axis_len == 1 is per-layer quantization (Section 2.6).
+ */
+#ifndef QTZ_H
+#define QTZ_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define QTZ_API __attribute__((visibility("default")))
+#else
+#define QTZ_API
+#endif
+
+typedef int32_t qtz_status;
+#define QTZ_OK 0
+#define QTZ_ERR_INVALID_ARG (-1)    /* null pointer, non-positive size, bad enum            */
+#define QTZ_ERR_MISALIGNED (-2)     /* pointer or pitch not a multiple of 16 bytes          */
+#define QTZ_ERR_UNSUPPORTED (-3)    /* well-formed request outside what is implemented      */
+#define QTZ_ERR_OVERFLOW (-4)       /* reduction length too large for int32 accumulation    */
+#define QTZ_ERR_NONFINITE (-5)      /* NaN or Inf met while calibrating                     */
+#define QTZ_ERR_CUDA (-6)           /* a CUDA runtime/driver call failed                    */
+#define QTZ_ERR_DEVICE_TIMEOUT (-7) /* a bounded device-side wait gave up                   */
+#define QTZ_ERR_NO_DEVICE (-8)      /* no usable CUDA device                                */
+
+typedef struct qtz_ctx* qtz_handle;     /* library-owned, opaque */
+typedef struct qtz_plan* qtz_conv_plan; /* library-owned: prepacked weights and tables */
+
+/* Scale, zero point and the nudged real range of one quantizer (Section 2.1). */
+typedef struct {
+    float scale;        /* Delta */
+    int32_t zero_point; /* z, an integer so that real 0.0 is exactly a code */
+    float min_nudged;   /* real value of the lowest code,  (0 - z) * Delta  */
+    float max_nudged;   /* real value of the highest code, (L - z) * Delta  */
+} qtz_qparams;
+
+typedef enum { QTZ_U8 = 0, QTZ_S8 = 1, QTZ_S4_PACKED = 2, QTZ_S32 = 3 } qtz_dtype;
+
+typedef enum {
+    QTZ_W_S8_PER_CHANNEL_SYM = 0,       /* int8 codes, one scale per output channel, z_w = 0 */
+    QTZ_W_U8_PER_LAYER_ASYM = 1,        /* uint8 codes, one (scale, z_w) for the layer       */
+    QTZ_W_S4_PACKED_PER_CHANNEL_SYM = 2 /* 4-bit codes in [-8,7], two per byte, z_w = 0      */
+} qtz_wkind;
+
+typedef enum { QTZ_OUT_U8 = 0, QTZ_OUT_S32_RAW = 1 } qtz_outkind;
+
+/* Geometry of one convolution.  Input NHWC [batch][h][w][c] with pitch c_pitch_in; output
+ * [batch][oh][ow][n] with pitch c_pitch_out, oh = (h + 2 pad - kh)/stride + 1 (same for ow).
+ * For a depthwise plan n must equal c.  With QTZ_OUT_S32_RAW the output is a dense int32
+ * array [batch*oh*ow][n] and c_pitch_out is ignored.                                       */
+typedef struct {
+    int32_t batch, h, w, c, c_pitch_in;
+    int32_t n, c_pitch_out;
+    int32_t kh, kw, stride, pad;
+    int32_t wkind;   /* qtz_wkind   */
+    int32_t outkind; /* qtz_outkind */
+} qtz_conv_desc;
+
+/* ---- library ------------------------------------------------------------------------- */
+
+/* Creates a handle bound to CUDA device `device` (allocates a few MB of device scratch).
+ * Blocking.  QTZ_ERR_NO_DEVICE when the device cannot be used.                            */
+QTZ_API qtz_status qtz_create(qtz_handle* out, int device);
+QTZ_API qtz_status qtz_destroy(qtz_handle h);
+QTZ_API const char* qtz_status_string(qtz_status s);
+/* Text of the last CUDA error seen through this handle ("" if none).  Host only.          */
+QTZ_API const char* qtz_last_error(qtz_handle h);
+/* Status word written by device code whose bounded waits gave up: 0, or
+ * QTZ_ERR_DEVICE_TIMEOUT with *site_id telling which wait.  Synchronises `stream`.        */
+QTZ_API qtz_status qtz_last_device_status(qtz_handle h, int32_t* site_id, void* stream);
+
+/* ---- quantizer parameters (Sections 2.1, 2.2, 2.5, 2.6) ------------------------------- */
+
+/* Range estimation by min/max (Section 2.5) followed by parameter derivation.
+ * Affine (symmetric == 0, Section 2.1): the range is first relaxed to contain 0, then
+ *   Delta = (max - min)/(2^bits - 1), z = round(-min/Delta) clamped to [0, 2^bits - 1], and
+ *   the representable range is nudged to [(0-z)Delta, (2^bits-1-z)Delta].
+ * Symmetric (Section 2.2): z = 0, Delta = max|x| / (2^(bits-1) - 1).
+ * A tensor (or channel) that is all zero gets Delta = 1, z = 0.
+ * Reads x_dev (fp32, device, outer*axis_len*inner values), writes axis_len entries to
+ * out_host.  BLOCKS until `stream` has finished.  bits in [2,8].
+ * Errors: QTZ_ERR_NONFINITE if any value is NaN/Inf (out_host is then unspecified).       */
+QTZ_API qtz_status qtz_calibrate_minmax(qtz_handle h, const float* x_dev, int64_t outer,
+                                int64_t axis_len, int64_t inner, int32_t bits,
+                                int32_t symmetric, qtz_qparams* out_host, void* stream);
+
+/* The range reduction alone (Section 2.5): min and max of each axis slice, written to
+ * lo_host / hi_host (axis_len floats each).  BLOCKS until `stream` has finished.
+ * QTZ_ERR_NONFINITE as above.  Lets a caller post-process a range (for instance clamp it to
+ * [0,6] for a layer followed by ReLU6) before deriving parameters from it.                */
+QTZ_API qtz_status qtz_minmax(qtz_handle h, const float* x_dev, int64_t outer, int64_t axis_len,
+                              int64_t inner, float* lo_host, float* hi_host, void* stream);
+
+/* Host-only: parameters from a known real range (same rules as above).                    */
+QTZ_API qtz_status qtz_params_from_range(float lo, float hi, int32_t bits, int32_t symmetric,
+                                 qtz_qparams* out_host);
+
+/* ---- quantize / dequantize (Eq. 1-3, 7-11) --------------------------------------------- */
+
+/* x_int = round(x / Delta) + z, clamped to the code range (Eq. 1-2; Eq. 7-11 with z = 0).
+ * The quotient is one IEEE fp32 division and round() is round-half-to-even.  Code ranges:
+ *   QTZ_U8 [0,255] (restrict_range: [0,254]); QTZ_S8 [-128,127] (restrict_range, Eq. 10:
+ *   [-127,127]); QTZ_S4_PACKED [-8,7] (restrict_range: [-7,7]).
+ * NaN maps to the lowest code, +-Inf saturate.
+ * params_host: axis_len entries, read before the call returns.
+ * QTZ_S4_PACKED: two's-complement nibbles packed along the innermost run of the view
+ * (`inner`, or `axis_len` when inner == 1): element 2i in the low nibble and 2i+1 in the
+ * high nibble of byte i; each run occupies (len+1)/2 bytes, an odd tail's high nibble is 0. */
+QTZ_API qtz_status qtz_quantize_tensor(qtz_handle h, const float* x_dev, int64_t outer,
+                               int64_t axis_len, int64_t inner, const qtz_qparams* params_host,
+                               int32_t out_dtype, int32_t restrict_range, void* q_dev,
+                               void* stream);
+
+/* x = (q - z) * Delta with one fp32 multiply (Eq. 3; z = 0 for the symmetric quantizer).
+ * in_dtype QTZ_S32 dequantizes int32 accumulators: zero_point must be 0 and `scale` holds
+ * the product Delta_x * Delta_w[n] of Eq. 4.                                                */
+QTZ_API qtz_status qtz_dequantize(qtz_handle h, const void* q_dev, int32_t in_dtype, int64_t outer,
+                          int64_t axis_len, int64_t inner, const qtz_qparams* params_host,
+                          float* x_dev, void* stream);
+
+/* ---- batch-norm folding (Eq. 20-21) ------------------------------------------------------ */
+
+/* W_inf[n][:] = gamma[n] W[n][:] / sigma[n],  Bias_inf[n] = beta[n] + gamma[n] (b[n] - mu[n]) /
+ * sigma[n], with sigma = sqrt(var + eps) and b = conv_bias (NULL means 0).  W is [n][k]
+ * (OHWI flattened), arithmetic in fp64 rounded once to fp32.  w_inf_dev may alias w_dev.     */
+QTZ_API qtz_status qtz_fold_batchnorm(qtz_handle h, const float* w_dev, const float* conv_bias_dev,
+                              const float* gamma_dev, const float* beta_dev,
+                              const float* mean_dev, const float* var_dev, float eps, int64_t n,
+                              int64_t k, float* w_inf_dev, float* bias_inf_dev, void* stream);
+
+/* bias_q[n] = sat_int32(round(bias[n] / (Delta_x * Delta_w[n]))): the bias in the scale of the
+ * accumulator of Eq. 4, zero point 0.  w_params_host has n entries (or 1 if per_layer != 0).  */
+QTZ_API qtz_status qtz_quantize_bias(qtz_handle h, const float* bias_dev, int64_t n, float x_scale,
+                             const qtz_qparams* w_params_host, int32_t per_layer,
+                             int32_t* bias_q_dev, void* stream);
+
+/* ---- fixed-point rescale helpers (host only; implied by Eq. 4, defined by this library) ---- */
+
+/* Real multiplier M >= 0 as m * 2^-rshift with 2^30 <= m < 2^31 and 1 <= rshift <= 62
+ * (M = 0 gives m = 0, rshift = 1).  QTZ_ERR_UNSUPPORTED when M is too large or too small.      */
+QTZ_API qtz_status qtz_quantize_multiplier(double real_multiplier, int32_t* mult, int32_t* rshift);
+/* Clamp range of a fused activation in the quantized domain (Section 3.2.1: the activation
+ * fuses into the producing op).  kind 0 none [0,255]; 1 ReLU [z_y,255];
+ * 2 ReLU6 [z_y, min(255, z_y + round(6/Delta_y))].                                            */
+QTZ_API qtz_status qtz_activation_range(int32_t kind, float y_scale, int32_t y_zero_point,
+                                int32_t* act_min, int32_t* act_max);
+/* Multipliers of the element-wise add (Section 3.2.1): the larger of Delta_a/Delta_y and
+ * Delta_b/Delta_y fixes rshift through qtz_quantize_multiplier, the other is round(M 2^rshift). */
+QTZ_API qtz_status qtz_add_params(float a_scale, float b_scale, float y_scale, int32_t* a_mult,
+                          int32_t* b_mult, int32_t* rshift);
+
+/* ---- convolution (Eq. 4-6) -------------------------------------------------------------- */
+
+/* One-time preparation of a layer ("the weights are constant at inference", Section 2.1):
+ * copies and re-lays the weights for the kernels, and precomputes per output channel the
+ * weight sums of the zero-point cross term of Eq. 5-6 (for padded 3x3 layers one sum per
+ * border class, so that padding behaves as real zero, i.e. the code z_x).
+ *   w_q_dev     OHWI codes [n][kh][kw][c] (depthwise: [kh][kw][c]); int8, uint8, or 4-bit
+ *               packed along the flattened kh*kw*c run of each output channel (depthwise:
+ *               along c), per desc->wkind.
+ *   bias_q_dev  n int32 (scale Delta_x Delta_w[n]); NULL means no bias.
+ *   w_zero_point_host  NULL, or 1 value (per-layer asymmetric weights).
+ *   mult_host, rshift_host  n entries: fixed-point form of Delta_x Delta_w[n] / Delta_y
+ *               (ignored, may be NULL, with QTZ_OUT_S32_RAW).
+ * The caller may free or overwrite all inputs once `stream` has passed this call.
+ * Errors: QTZ_ERR_OVERFLOW when kh*kw*c > 32768; QTZ_ERR_UNSUPPORTED for depthwise layers
+ * other than 3x3 / pad 1 / stride 1 or 2.                                                      */
+QTZ_API qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, int32_t depthwise,
+                           const void* w_q_dev, const int32_t* bias_q_dev,
+                           const int32_t* w_zero_point_host, const int32_t* mult_host,
+                           const int32_t* rshift_host, qtz_conv_plan* out, void* stream);
+QTZ_API qtz_status qtz_conv_destroy(qtz_conv_plan p);
+/* Name of the kernel family a plan dispatches to ("tcgen05", "direct", "depthwise").           */
+QTZ_API const char* qtz_conv_plan_kernel(qtz_conv_plan p);
+
+/* Quantized convolution, evaluated through the expansion of Eq. 5-6:
+ *   acc = conv(w_Q, x_Q) - z_w sum(x_Q) - z_x sum(w_Q) + K_valid z_x z_w + bias_q
+ * which equals Eq. 4's conv(w_Q - z_w, x_Q - z_x) exactly; sums run over in-image taps and
+ * K_valid counts them.  Then y = clamp(z_y + ((acc * mult[n] + 2^(rshift[n]-1)) >> rshift[n]),
+ * act_min, act_max), 0 <= act_min <= act_max <= 255 (the fused ReLU/ReLU6 clamp).  With
+ * QTZ_OUT_S32_RAW y_dev receives acc as int32 and y_zero_point / act_* are ignored.
+ * x_dev / y_dev follow the plan's geometry; they must not overlap.                             */
+QTZ_API qtz_status qtz_conv2d_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point,
+                         void* y_dev, int32_t y_zero_point, int32_t act_min, int32_t act_max,
+                         void* stream);
+/* Depthwise form of the same (depth multiplier 1; Section 3.1.3 networks): the sum runs over
+ * the kh x kw taps of one channel.  Plan must have been created with depthwise != 0.           */
+QTZ_API qtz_status qtz_depthwise_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point,
+                            void* y_dev, int32_t y_zero_point, int32_t act_min, int32_t act_max,
+                            void* stream);
+
+/* ---- integer glue ops of a quantized network (Section 3.2.1) -------------------------------- */
+
+/* Element-wise add with both inputs rescaled to the output scale, fused clamp:
+ *   y = clamp(z_y + (((a - z_a) a_mult + (b - z_b) b_mult + 2^(rshift-1)) >> rshift)).
+ * a, b, y: `pixels` rows of c channels with the same pitch.                                     */
+QTZ_API qtz_status qtz_add_u8(qtz_handle h, const uint8_t* a_dev, int32_t a_zp, int32_t a_mult,
+                      const uint8_t* b_dev, int32_t b_zp, int32_t b_mult, int32_t rshift,
+                      uint8_t* y_dev, int32_t y_zp, int32_t act_min, int32_t act_max,
+                      int64_t pixels, int32_t c, int32_t c_pitch, void* stream);
+/* k x k max pooling on codes (the quantizer is monotone, so input and output share (Delta, z));
+ * out-of-image taps are skipped.                                                                */
+QTZ_API qtz_status qtz_maxpool_u8(qtz_handle h, const uint8_t* x_dev, uint8_t* y_dev, int32_t batch,
+                          int32_t hh, int32_t ww, int32_t c, int32_t c_pitch, int32_t k,
+                          int32_t stride, int32_t pad, void* stream);
+/* Global average pool: S = sum_{h,w}(x - z_x); y = clamp(z_y + ((S mult + 2^(rshift-1)) >> rshift),
+ * 0, 255) with (mult, rshift) the fixed-point form of Delta_x / (hw Delta_y).  y: [batch][c_pitch]. */
+QTZ_API qtz_status qtz_global_avgpool_u8(qtz_handle h, const uint8_t* x_dev, int32_t x_zp, uint8_t* y_dev,
+                                 int32_t y_zp, int32_t mult, int32_t rshift, int32_t batch,
+                                 int32_t hw, int32_t c, int32_t c_pitch, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QTZ_H */

@@ -1,0 +1,153 @@
+// Integer glue operations of a quantized network (Section 3.2.1): element-wise add with
+// rescale and fused clamp, max pooling, global average pooling.  All HBM-bound; each
+// thread moves 16 bytes per operand.
+#include <algorithm>
+
+#include "qtz_internal.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+struct AddRule {
+    int32_t a_zp, a_mult, b_zp, b_mult, rshift, y_zp, act_min, act_max;
+};
+
+__device__ __forceinline__ uint32_t add1(uint32_t a, uint32_t b, const AddRule& r, int64_t bias)
+{
+    const int64_t v = static_cast<int64_t>(static_cast<int32_t>(a) - r.a_zp) * r.a_mult +
+                      static_cast<int64_t>(static_cast<int32_t>(b) - r.b_zp) * r.b_mult + bias;
+    const int64_t y = v >> r.rshift;
+    return static_cast<uint32_t>(min(max(y, static_cast<int64_t>(r.act_min)), static_cast<int64_t>(r.act_max)));
+}
+
+__device__ __forceinline__ uint32_t add4(uint32_t a, uint32_t b, const AddRule& r, int64_t bias)
+{
+    return add1(a & 0xff, b & 0xff, r, bias) | (add1((a >> 8) & 0xff, (b >> 8) & 0xff, r, bias) << 8) |
+           (add1((a >> 16) & 0xff, (b >> 16) & 0xff, r, bias) << 16) | (add1(a >> 24, b >> 24, r, bias) << 24);
+}
+
+// y = clamp(z_y + ((a' m_a + b' m_b + 2^(r-1)) >> r)); the rounding constant and z_y 2^r are
+// folded into one 64-bit addend (|a' m| < 2^39 and r <= 62 - 9 keep the sum inside int64).
+__global__ void __launch_bounds__(kThreads)
+add_u8_kernel(const uint8_t* __restrict__ a, const uint8_t* __restrict__ b, int64_t bytes, AddRule r,
+              uint8_t* __restrict__ y)
+{
+    const int64_t bias = (static_cast<int64_t>(1) << (r.rshift - 1)) + (static_cast<int64_t>(r.y_zp) << r.rshift);
+    const int64_t groups = bytes >> 4;
+    const int64_t g = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+    if (g >= groups) return;
+    const uint4 va = __ldcs(reinterpret_cast<const uint4*>(a) + g);
+    const uint4 vb = __ldcs(reinterpret_cast<const uint4*>(b) + g);
+    uint4 o;
+    o.x = add4(va.x, vb.x, r, bias); o.y = add4(va.y, vb.y, r, bias);
+    o.z = add4(va.z, vb.z, r, bias); o.w = add4(va.w, vb.w, r, bias);
+    reinterpret_cast<uint4*>(y)[g] = o;
+}
+
+// One thread per (output pixel, 16-channel group).
+__global__ void __launch_bounds__(kThreads)
+maxpool_u8_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ y, int batch, int hh, int ww, int pitch,
+                  int k, int stride, int pad, int oh_n, int ow_n)
+{
+    const int groups = pitch >> 4;
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+    const int64_t total = static_cast<int64_t>(batch) * oh_n * ow_n * groups;
+    if (t >= total) return;
+    const int g = static_cast<int>(t % groups);
+    int64_t p = t / groups;
+    const int ow = static_cast<int>(p % ow_n); p /= ow_n;
+    const int oh = static_cast<int>(p % oh_n);
+    const int b = static_cast<int>(p / oh_n);
+    uint4 m = make_uint4(0, 0, 0, 0);
+    for (int i = 0; i < k; ++i) {
+        const int ih = oh * stride - pad + i;
+        if (ih < 0 || ih >= hh) continue;
+        for (int j = 0; j < k; ++j) {
+            const int iw = ow * stride - pad + j;
+            if (iw < 0 || iw >= ww) continue;
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + ((static_cast<int64_t>(b) * hh + ih) * ww + iw) * pitch) + g);
+            m.x = __vmaxu4(m.x, v.x); m.y = __vmaxu4(m.y, v.y); m.z = __vmaxu4(m.z, v.z); m.w = __vmaxu4(m.w, v.w);
+        }
+    }
+    reinterpret_cast<uint4*>(y + ((static_cast<int64_t>(b) * oh_n + oh) * ow_n + ow) * pitch)[g] = m;
+}
+
+// One thread per (image, 4-channel group); sums hw pixels, then one requantisation.
+__global__ void __launch_bounds__(kThreads)
+global_avgpool_u8_kernel(const uint8_t* __restrict__ x, int32_t x_zp, uint8_t* __restrict__ y, int32_t y_zp,
+                         int32_t mult, int32_t rshift, int batch, int hw, int pitch)
+{
+    const int groups = pitch >> 2;
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+    if (t >= static_cast<int64_t>(batch) * groups) return;
+    const int g = static_cast<int>(t % groups), b = static_cast<int>(t / groups);
+    int32_t s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+    const uint8_t* base = x + static_cast<int64_t>(b) * hw * pitch + 4 * g;
+    for (int p = 0; p < hw; ++p) {
+        const uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(base + static_cast<int64_t>(p) * pitch));
+        s0 += v & 0xff; s1 += (v >> 8) & 0xff; s2 += (v >> 16) & 0xff; s3 += v >> 24;
+    }
+    const int64_t rnd = static_cast<int64_t>(1) << (rshift - 1);
+    const int32_t off = hw * x_zp;
+    auto rq = [&](int32_t s) -> uint32_t {
+        const int64_t v = static_cast<int64_t>(s - off) * mult + rnd;
+        const int64_t r = static_cast<int64_t>(y_zp) + (v >> rshift);
+        return static_cast<uint32_t>(r < 0 ? 0 : (r > 255 ? 255 : r));
+    };
+    reinterpret_cast<uint32_t*>(y + static_cast<int64_t>(b) * pitch)[g] = rq(s0) | (rq(s1) << 8) | (rq(s2) << 16) | (rq(s3) << 24);
+}
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+}  // namespace
+
+extern "C" qtz_status qtz_add_u8(qtz_handle h, const uint8_t* a_dev, int32_t a_zp, int32_t a_mult,
+                                 const uint8_t* b_dev, int32_t b_zp, int32_t b_mult, int32_t rshift, uint8_t* y_dev,
+                                 int32_t y_zp, int32_t act_min, int32_t act_max, int64_t pixels, int32_t c,
+                                 int32_t c_pitch, void* stream)
+{
+    if (!h || !a_dev || !b_dev || !y_dev || pixels <= 0 || c <= 0 || c_pitch < c) return QTZ_ERR_INVALID_ARG;
+    if (a_mult < 0 || b_mult < 0 || act_min < 0 || act_max > 255 || act_min > act_max) return QTZ_ERR_INVALID_ARG;
+    if (y_zp < 0 || y_zp > 255 || a_zp < 0 || a_zp > 255 || b_zp < 0 || b_zp > 255) return QTZ_ERR_INVALID_ARG;
+    if (rshift < 1 || rshift > 53) return QTZ_ERR_UNSUPPORTED;
+    if ((c_pitch & 15) || !qtz_aligned16(a_dev) || !qtz_aligned16(b_dev) || !qtz_aligned16(y_dev)) return QTZ_ERR_MISALIGNED;
+    const int64_t bytes = pixels * c_pitch;
+    const AddRule r{a_zp, a_mult, b_zp, b_mult, rshift, y_zp, act_min, act_max};
+    add_u8_kernel<<<static_cast<unsigned>(ceil_div(bytes >> 4, kThreads)), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        a_dev, b_dev, bytes, r, y_dev);
+    QTZ_LAUNCH_CHECK(h, "add_u8_kernel");
+    return QTZ_OK;
+}
+
+extern "C" qtz_status qtz_maxpool_u8(qtz_handle h, const uint8_t* x_dev, uint8_t* y_dev, int32_t batch, int32_t hh,
+                                     int32_t ww, int32_t c, int32_t c_pitch, int32_t k, int32_t stride, int32_t pad,
+                                     void* stream)
+{
+    if (!h || !x_dev || !y_dev || batch <= 0 || hh <= 0 || ww <= 0 || c <= 0 || c_pitch < c || k <= 0 || stride <= 0 ||
+        pad < 0 || pad >= k)
+        return QTZ_ERR_INVALID_ARG;
+    if ((c_pitch & 15) || !qtz_aligned16(x_dev) || !qtz_aligned16(y_dev)) return QTZ_ERR_MISALIGNED;
+    const int oh_n = (hh + 2 * pad - k) / stride + 1, ow_n = (ww + 2 * pad - k) / stride + 1;
+    if (oh_n <= 0 || ow_n <= 0) return QTZ_ERR_INVALID_ARG;
+    const int64_t total = static_cast<int64_t>(batch) * oh_n * ow_n * (c_pitch >> 4);
+    maxpool_u8_kernel<<<static_cast<unsigned>(ceil_div(total, kThreads)), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        x_dev, y_dev, batch, hh, ww, c_pitch, k, stride, pad, oh_n, ow_n);
+    QTZ_LAUNCH_CHECK(h, "maxpool_u8_kernel");
+    return QTZ_OK;
+}
+
+extern "C" qtz_status qtz_global_avgpool_u8(qtz_handle h, const uint8_t* x_dev, int32_t x_zp, uint8_t* y_dev,
+                                            int32_t y_zp, int32_t mult, int32_t rshift, int32_t batch, int32_t hw,
+                                            int32_t c, int32_t c_pitch, void* stream)
+{
+    if (!h || !x_dev || !y_dev || batch <= 0 || hw <= 0 || c <= 0 || c_pitch < c || mult < 0) return QTZ_ERR_INVALID_ARG;
+    if (rshift < 1 || rshift > 62 || x_zp < 0 || x_zp > 255 || y_zp < 0 || y_zp > 255) return QTZ_ERR_INVALID_ARG;
+    if (hw > (1 << 22)) return QTZ_ERR_OVERFLOW;
+    if ((c_pitch & 15) || !qtz_aligned16(x_dev) || !qtz_aligned16(y_dev)) return QTZ_ERR_MISALIGNED;
+    const int64_t total = static_cast<int64_t>(batch) * (c_pitch >> 2);
+    global_avgpool_u8_kernel<<<static_cast<unsigned>(ceil_div(total, kThreads)), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        x_dev, x_zp, y_dev, y_zp, mult, rshift, batch, hw, c_pitch);
+    QTZ_LAUNCH_CHECK(h, "global_avgpool_u8_kernel");
+    return QTZ_OK;
+}

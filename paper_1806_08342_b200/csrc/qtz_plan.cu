@@ -1,0 +1,237 @@
+// Per-layer preparation (weights are constant at inference, Section 2.1) and dispatch of
+// the convolution entry points.
+#include <new>
+#include <vector>
+
+#include "qtz_plan.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// Reads weight code k of output channel `row` from the API layout and moves it to int8:
+// int8 stays, uint8 is shifted by -128 (its zero point moves with it), 4-bit is sign-extended.
+__device__ __forceinline__ int32_t load_code_s8(const void* w, int wkind, int64_t row, int64_t k, int64_t k_total)
+{
+    if (wkind == QTZ_W_S8_PER_CHANNEL_SYM) return static_cast<const int8_t*>(w)[row * k_total + k];
+    if (wkind == QTZ_W_U8_PER_LAYER_ASYM) return static_cast<int32_t>(static_cast<const uint8_t*>(w)[row * k_total + k]) - 128;
+    const uint32_t byte = static_cast<const uint8_t*>(w)[row * ((k_total + 1) >> 1) + (k >> 1)];
+    const uint32_t nib = (k & 1) ? (byte >> 4) : (byte & 0xfu);
+    return static_cast<int32_t>(nib << 28) >> 28;
+}
+
+__global__ void __launch_bounds__(kThreads)
+prepack_direct_kernel(const void* __restrict__ w, int wkind, int n, int k_total, int n_padded, int k_padded,
+                      int8_t* __restrict__ out)
+{
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+    if (i >= static_cast<int64_t>(n_padded) * k_padded) return;
+    const int64_t row = i / k_padded, k = i - row * k_padded;
+    out[i] = (row < n && k < k_total) ? static_cast<int8_t>(load_code_s8(w, wkind, row, k, k_total)) : 0;
+}
+
+// wsum[row] = sum over the whole receptive field of the int8 codes.
+__global__ void __launch_bounds__(kThreads)
+weight_sum_kernel(const int8_t* __restrict__ w, int k_padded, int32_t* __restrict__ wsum)
+{
+    __shared__ int32_t part[kThreads / 32];
+    const int row = blockIdx.x;
+    int32_t s = 0;
+    for (int k = threadIdx.x; k < k_padded; k += kThreads) s += w[static_cast<int64_t>(row) * k_padded + k];
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int32_t t = 0;
+        for (int i = 0; i < kThreads / 32; ++i) t += part[i];
+        wsum[row] = t;
+    }
+}
+
+// Depthwise weights [taps][c] -> int16 [taps][pitch] holding (code - z_w), zero padded.
+__global__ void __launch_bounds__(kThreads)
+prepack_depthwise_kernel(const void* __restrict__ w, int wkind, int taps, int c, int pitch, int zw_signed,
+                         int16_t* __restrict__ out)
+{
+    const int i = blockIdx.x * kThreads + threadIdx.x;
+    if (i >= taps * pitch) return;
+    const int tap = i / pitch, ch = i - tap * pitch;
+    out[i] = ch < c ? static_cast<int16_t>(load_code_s8(w, wkind, tap, ch, c) - zw_signed) : 0;
+}
+
+__global__ void fill_i32_kernel(int32_t* p, int n, int32_t v)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) p[i] = v;
+}
+
+qtz_status validate_desc(const qtz_conv_desc& d, int depthwise)
+{
+    if (d.batch <= 0 || d.h <= 0 || d.w <= 0 || d.c <= 0 || d.n <= 0 || d.kh <= 0 || d.kw <= 0 || d.stride <= 0 ||
+        d.pad < 0 || d.c_pitch_in < d.c)
+        return QTZ_ERR_INVALID_ARG;
+    if (d.wkind < QTZ_W_S8_PER_CHANNEL_SYM || d.wkind > QTZ_W_S4_PACKED_PER_CHANNEL_SYM) return QTZ_ERR_INVALID_ARG;
+    if (d.outkind != QTZ_OUT_U8 && d.outkind != QTZ_OUT_S32_RAW) return QTZ_ERR_INVALID_ARG;
+    if (d.c_pitch_in & 15) return QTZ_ERR_MISALIGNED;
+    if (d.outkind == QTZ_OUT_U8) {
+        if (d.c_pitch_out < d.n) return QTZ_ERR_INVALID_ARG;
+        if (d.c_pitch_out & 15) return QTZ_ERR_MISALIGNED;
+    }
+    if (d.h + 2 * d.pad < d.kh || d.w + 2 * d.pad < d.kw) return QTZ_ERR_INVALID_ARG;
+    if (d.kh > 64 || d.kw > 64 || d.pad >= d.kh || d.pad >= d.kw) return QTZ_ERR_INVALID_ARG;
+    const int64_t k = depthwise ? static_cast<int64_t>(d.kh) * d.kw : static_cast<int64_t>(d.kh) * d.kw * d.c;
+    if (k > 32768) return QTZ_ERR_OVERFLOW;
+    if (depthwise) {
+        if (d.n != d.c) return QTZ_ERR_INVALID_ARG;
+        if (d.kh != 3 || d.kw != 3 || d.pad != 1 || (d.stride != 1 && d.stride != 2) || d.outkind != QTZ_OUT_U8)
+            return QTZ_ERR_UNSUPPORTED;
+    }
+    return QTZ_OK;
+}
+
+}  // namespace
+
+extern "C" qtz_status qtz_conv_destroy(qtz_conv_plan p)
+{
+    if (!p) return QTZ_ERR_INVALID_ARG;
+    cudaSetDevice(p->device);
+    cudaDeviceSynchronize();
+    qtz_tc_release(p);
+    cudaFree(p->w_direct);
+    cudaFree(p->w_depthwise);
+    cudaFree(p->bias);
+    cudaFree(p->wsum);
+    cudaFree(p->mult);
+    cudaFree(p->rshift);
+    cudaFree(p->x_gather);
+    (void)cudaGetLastError();
+    delete p;
+    return QTZ_OK;
+}
+
+extern "C" const char* qtz_conv_plan_kernel(qtz_conv_plan p)
+{
+    if (!p) return "";
+    return p->family == QTZ_K_TCGEN05 ? "tcgen05" : (p->family == QTZ_K_DEPTHWISE ? "depthwise" : "direct");
+}
+
+extern "C" qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, int32_t depthwise, const void* w_q_dev,
+                                      const int32_t* bias_q_dev, const int32_t* w_zero_point_host,
+                                      const int32_t* mult_host, const int32_t* rshift_host, qtz_conv_plan* out,
+                                      void* stream)
+{
+    if (!h || !desc || !w_q_dev || !out) return QTZ_ERR_INVALID_ARG;
+    *out = nullptr;
+    qtz_status s = validate_desc(*desc, depthwise);
+    if (s != QTZ_OK) return s;
+    const qtz_conv_desc& d = *desc;
+    const bool raw = d.outkind == QTZ_OUT_S32_RAW;
+    if (!raw && (!mult_host || !rshift_host)) return QTZ_ERR_INVALID_ARG;
+    if (d.wkind == QTZ_W_U8_PER_LAYER_ASYM && !w_zero_point_host) return QTZ_ERR_INVALID_ARG;
+    if (d.wkind != QTZ_W_U8_PER_LAYER_ASYM && w_zero_point_host && *w_zero_point_host != 0) return QTZ_ERR_INVALID_ARG;
+    if (w_zero_point_host && (*w_zero_point_host < 0 || *w_zero_point_host > 255)) return QTZ_ERR_INVALID_ARG;
+    if (!raw)
+        for (int i = 0; i < d.n; ++i)
+            if (mult_host[i] < 0 || rshift_host[i] < 1 || rshift_host[i] > 62) return QTZ_ERR_INVALID_ARG;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    QTZ_CUDA(h, cudaSetDevice(h->device));
+    qtz_plan* p = new (std::nothrow) qtz_plan();
+    if (!p) return QTZ_ERR_INVALID_ARG;
+    p->h = h;
+    p->device = h->device;
+    p->d = d;
+    p->depthwise = depthwise ? 1 : 0;
+    p->oh = (d.h + 2 * d.pad - d.kh) / d.stride + 1;
+    p->ow = (d.w + 2 * d.pad - d.kw) / d.stride + 1;
+    p->k_total = depthwise ? d.kh * d.kw : d.kh * d.kw * d.c;
+    p->w_zp_signed = d.wkind == QTZ_W_U8_PER_LAYER_ASYM ? *w_zero_point_host - 128 : 0;
+
+#define PLAN_CUDA(expr)                                        \
+    do {                                                       \
+        cudaError_t _e = (expr);                               \
+        if (_e != cudaSuccess) {                               \
+            qtz_cuda_fail(h, _e, #expr);                       \
+            qtz_conv_destroy(p);                               \
+            return QTZ_ERR_CUDA;                               \
+        }                                                      \
+    } while (0)
+
+    const size_t nb = sizeof(int32_t) * static_cast<size_t>(d.n);
+    PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->bias), nb));
+    if (bias_q_dev)
+        PLAN_CUDA(cudaMemcpyAsync(p->bias, bias_q_dev, nb, cudaMemcpyDeviceToDevice, st));
+    else
+        PLAN_CUDA(cudaMemsetAsync(p->bias, 0, nb, st));
+    if (!raw) {
+        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->mult), nb));
+        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->rshift), nb));
+        PLAN_CUDA(cudaMemcpyAsync(p->mult, mult_host, nb, cudaMemcpyHostToDevice, st));
+        PLAN_CUDA(cudaMemcpyAsync(p->rshift, rshift_host, nb, cudaMemcpyHostToDevice, st));
+    }
+
+    if (depthwise) {
+        p->family = QTZ_K_DEPTHWISE;
+        const int taps = d.kh * d.kw;
+        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->w_depthwise), sizeof(int16_t) * taps * d.c_pitch_in));
+        prepack_depthwise_kernel<<<(taps * d.c_pitch_in + kThreads - 1) / kThreads, kThreads, 0, st>>>(
+            w_q_dev, d.wkind, taps, d.c, d.c_pitch_in, p->w_zp_signed, p->w_depthwise);
+        PLAN_CUDA(cudaGetLastError());
+    } else if (qtz_tc_supported(d)) {
+        p->family = QTZ_K_TCGEN05;
+        s = qtz_tc_prepare(p, w_q_dev, st);
+        if (s != QTZ_OK) {
+            qtz_conv_destroy(p);
+            return s;
+        }
+    } else {
+        p->family = QTZ_K_DIRECT;
+        p->k_padded = (p->k_total + 15) & ~15;
+        p->n_padded = (d.n + 63) & ~63;
+        const int64_t elems = static_cast<int64_t>(p->n_padded) * p->k_padded;
+        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->w_direct), static_cast<size_t>(elems)));
+        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->wsum), sizeof(int32_t) * p->n_padded));
+        prepack_direct_kernel<<<static_cast<unsigned>((elems + kThreads - 1) / kThreads), kThreads, 0, st>>>(
+            w_q_dev, d.wkind, d.n, p->k_total, p->n_padded, p->k_padded, p->w_direct);
+        PLAN_CUDA(cudaGetLastError());
+        weight_sum_kernel<<<p->n_padded, kThreads, 0, st>>>(p->w_direct, p->k_padded, p->wsum);
+        PLAN_CUDA(cudaGetLastError());
+    }
+#undef PLAN_CUDA
+    *out = p;
+    return QTZ_OK;
+}
+
+static qtz_status check_run_args(qtz_conv_plan p, const void* x, const void* y, int32_t x_zp, int32_t y_zp,
+                                 int32_t act_min, int32_t act_max)
+{
+    if (!p || !x || !y) return QTZ_ERR_INVALID_ARG;
+    if (x_zp < 0 || x_zp > 255) return QTZ_ERR_INVALID_ARG;
+    if (p->d.outkind == QTZ_OUT_U8) {
+        if (y_zp < 0 || y_zp > 255 || act_min < 0 || act_max > 255 || act_min > act_max) return QTZ_ERR_INVALID_ARG;
+    }
+    if (!qtz_aligned16(x) || !qtz_aligned16(y)) return QTZ_ERR_MISALIGNED;
+    return QTZ_OK;
+}
+
+extern "C" qtz_status qtz_conv2d_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point, void* y_dev,
+                                    int32_t y_zero_point, int32_t act_min, int32_t act_max, void* stream)
+{
+    qtz_status s = check_run_args(p, x_dev, y_dev, x_zero_point, y_zero_point, act_min, act_max);
+    if (s != QTZ_OK) return s;
+    if (p->depthwise) return QTZ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (p->family == QTZ_K_TCGEN05)
+        return qtz_tc_launch(p, x_dev, x_zero_point, y_dev, y_zero_point, act_min, act_max, st);
+    return qtz_direct_launch(p, x_dev, x_zero_point, y_dev, y_zero_point, act_min, act_max, st);
+}
+
+extern "C" qtz_status qtz_depthwise_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point, void* y_dev,
+                                       int32_t y_zero_point, int32_t act_min, int32_t act_max, void* stream)
+{
+    qtz_status s = check_run_args(p, x_dev, y_dev, x_zero_point, y_zero_point, act_min, act_max);
+    if (s != QTZ_OK) return s;
+    if (!p->depthwise) return QTZ_ERR_INVALID_ARG;
+    return qtz_depthwise_launch(p, x_dev, x_zero_point, static_cast<uint8_t*>(y_dev), y_zero_point, act_min, act_max,
+                                static_cast<cudaStream_t>(stream));
+}

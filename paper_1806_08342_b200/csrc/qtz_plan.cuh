@@ -1,0 +1,44 @@
+// A convolution plan: the layer's geometry plus everything prepared once per layer
+// (re-laid weights, per-channel weight sums of the zero-point cross term, multipliers).
+#pragma once
+
+#include <cuda.h>
+
+#include "qtz_internal.cuh"
+
+struct qtz_tc_state;  // tensor-core path state (tensor maps, tile shape); see qtz_conv_tc.cu
+
+struct qtz_plan {
+    qtz_ctx* h = nullptr;
+    int device = 0;
+    qtz_conv_desc d{};
+    int depthwise = 0;
+    int family = QTZ_K_DIRECT;
+    int oh = 0, ow = 0;
+    int k_total = 0;      // kh*kw*c
+    int k_padded = 0;     // row length of w_direct (multiple of 16)
+    int n_padded = 0;     // rows of w_direct (multiple of 64)
+    int w_zp_signed = 0;  // weight zero point after moving codes to int8 (z_w - 128 for uint8 weights)
+
+    int8_t* w_direct = nullptr;   // [n_padded][k_padded] int8, zero padded       (direct path)
+    int16_t* w_depthwise = nullptr;  // [kh*kw][c_pitch_in] codes minus zero point  (depthwise path)
+    int32_t* bias = nullptr;      // [n] (zeros when the layer has no bias)
+    int32_t* wsum = nullptr;      // [classes][n] sum of int8 weight codes per border class
+    int32_t* mult = nullptr;      // [n]
+    int32_t* rshift = nullptr;    // [n]
+    uint8_t* x_gather = nullptr;  // strided 1x1 layers: the sub-sampled input, pitched NHWC
+    qtz_tc_state* tc = nullptr;
+};
+
+// Direct (CUDA-core) path.
+qtz_status qtz_direct_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, int32_t y_zp,
+                             int32_t act_min, int32_t act_max, cudaStream_t st);
+qtz_status qtz_depthwise_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, uint8_t* y, int32_t y_zp,
+                                int32_t act_min, int32_t act_max, cudaStream_t st);
+
+// Tensor-core (tcgen05) path.
+bool qtz_tc_supported(const qtz_conv_desc& d);
+qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st);
+void qtz_tc_release(qtz_plan* p);
+qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, int32_t y_zp,
+                         int32_t act_min, int32_t act_max, cudaStream_t st);

@@ -1,0 +1,86 @@
+"""CPU-side checks of the C ABI: the library loads without a GPU, exports every symbol the
+header declares, and its host-only scalar rules agree with the oracle's."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_1806_08342_b200 import build as qbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def qtz():
+    qbuild.build()
+    from paper_1806_08342_b200 import qtz as q
+    q.load_library()
+    return q
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "qtz.h")).read()
+    return sorted(set(re.findall(r"QTZ_API\s+[\w\s\*]+?\b(qtz_\w+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported_and_bound(qtz):
+    lib = qtz.load_library()
+    names = declared_symbols()
+    assert len(names) >= 20
+    for name in names:
+        assert hasattr(lib, name), name
+    assert sorted(qtz.SIGNATURES) == names
+
+
+def test_status_strings(qtz):
+    lib = qtz.load_library()
+    assert lib.qtz_status_string(0) == b"ok"
+    for code in range(-8, 0):
+        assert lib.qtz_status_string(code) not in (b"", b"unknown status")
+
+
+def test_create_without_gpu_fails_loudly(qtz):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("GPU present")
+    with pytest.raises(qtz.QtzError) as e:
+        qtz.Handle(0)
+    assert e.value.code == -8
+
+
+def test_multiplier_matches_oracle(qtz):
+    g = np.random.default_rng(0)
+    for M in list(10 ** g.uniform(-9, 3, 5000)) + [0.0, 0.5, 1.0, 2.0 ** -31, 1 - 2.0 ** -33, 0.75]:
+        assert qtz.quantize_multiplier(float(M)) == oracle.quantize_multiplier(float(M))
+    for bad in (-1.0, float("nan"), float("inf"), 2.0 ** 31, 2.0 ** -40):
+        with pytest.raises(qtz.QtzError):
+            qtz.quantize_multiplier(bad)
+        with pytest.raises(oracle.OracleError):
+            oracle.quantize_multiplier(bad)
+
+
+def test_activation_range_and_add_params_match_oracle(qtz):
+    g = np.random.default_rng(1)
+    for _ in range(2000):
+        s = float(np.float32(10 ** g.uniform(-4, 1)))
+        z = int(g.integers(0, 256))
+        for kind in (0, 1, 2):
+            assert qtz.activation_range(kind, s, z) == oracle.activation_range(kind, s, z)
+        sa, sb, sy = (float(np.float32(10 ** g.uniform(-3, 0))) for _ in range(3))
+        assert qtz.add_params(sa, sb, sy) == oracle.add_params(sa, sb, sy)
+
+
+def test_params_from_range_matches_oracle(qtz):
+    g = np.random.default_rng(2)
+    cases = [(2.1, 3.5), (-3.5, -2.1), (0.0, 0.0), (-1.0, 1.0), (0.0, 6.0), (-1e-30, 1e-30)]
+    for _ in range(3000):
+        lo = float(np.float32(g.normal() * 10 ** g.uniform(-4, 4)))
+        cases.append((lo, float(np.float32(lo + abs(g.normal()) * 10 ** g.uniform(-4, 4)))))
+    for lo, hi in cases:
+        for bits in (4, 8):
+            a, b = qtz.params_from_range(lo, hi, bits, False), oracle.affine_params(lo, hi, bits)
+            assert a.tobytes() == b.tobytes(), (lo, hi, bits, a, b)
+            a, b = qtz.params_from_range(lo, hi, bits, True), oracle.symmetric_params(lo, hi, bits)
+            assert a.tobytes() == b.tobytes()

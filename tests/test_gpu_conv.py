@@ -1,0 +1,289 @@
+"""GPU parity of qtz_conv2d_u8 / qtz_depthwise_u8 against the oracle: every uint8 / int32
+output bit-exact.  Shapes span several tiles with ragged tails, the degenerate cases, every
+weight kind, and the first two workloads (single 3x3 conv; quantized GEMM)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1806_08342_b200 import qtz, synth
+from gpu_util import dev, host, hq, pitched, rup16  # noqa: F401
+
+pytestmark = pytest.mark.gpu
+
+
+def make_weights(wkind, shape, seed):
+    """Random weight codes in the API layout plus the oracle's int32 view and zero point."""
+    g = synth.rng(seed, 70)
+    if wkind == qtz.W_S8_PER_CHANNEL_SYM:
+        codes = g.integers(-127, 128, size=shape).astype(np.int32)
+        codes.flat[0] = -128                                       # raw codes may use the full range
+        return codes.astype(np.int8), codes, None
+    if wkind == qtz.W_U8_PER_LAYER_ASYM:
+        codes = g.integers(0, 256, size=shape).astype(np.int32)
+        return codes.astype(np.uint8), codes, int(g.integers(0, 256))
+    codes = g.integers(-8, 8, size=shape).astype(np.int32)
+    codes.flat[0] = -8
+    return None, codes, None                                        # packed by the caller (layout differs)
+
+
+def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=2, expect_kernel=None):
+    x = synth.uniform_u8((b, h, w, c), seed, 1)
+    xp = pitched(x)
+    api_w, codes, zw = make_weights(wkind, (n, k, k, c), seed)
+    if wkind == qtz.W_S4_PACKED_PER_CHANNEL_SYM:
+        api_w = oracle.pack_s4(codes.reshape(n, -1))
+    g = synth.rng(seed, 71)
+    bias = g.integers(-20000, 20000, size=n).astype(np.int32)
+    z_x = int(g.integers(0, 256))
+    z_w = None if zw is None else np.full(n, zw, np.int32)
+    acc = oracle.conv2d_acc(xp, z_x, codes, z_w, bias, stride, pad, c=c)
+    desc = qtz.conv_desc(b, h, w, c, n, k, k, stride, pad, wkind, qtz.OUT_S32_RAW if raw else qtz.OUT_U8)
+    if raw:
+        plan = hq.conv_create(desc, dev(api_w), dev(bias), zw)
+        got = host(plan(dev(xp), z_x))
+        if expect_kernel:
+            assert plan.kernel == expect_kernel
+        assert got.shape == acc.shape
+        assert np.array_equal(got, acc)
+        return
+    # per-channel multipliers spread over two decades so that outputs use the whole code range
+    span = np.abs(acc).reshape(-1, n).max(axis=0).astype(np.float64) + 1.0
+    real_m = 200.0 / span * np.exp(g.uniform(-1.0, 1.0, size=n))
+    mr = [oracle.quantize_multiplier(float(v)) for v in real_m]
+    mult = np.array([m for m, _ in mr], np.int32)
+    rsh = np.array([r for _, r in mr], np.int32)
+    z_y = int(g.integers(0, 200))
+    lo, hi = {0: (0, 255), 1: (z_y, 255), 2: (z_y, min(255, z_y + 120))}[act]
+    want = oracle.requantize(acc, mult, rsh, z_y, lo, hi)
+    plan = hq.conv_create(desc, dev(api_w), dev(bias), zw, mult, rsh)
+    if expect_kernel:
+        assert plan.kernel == expect_kernel
+    got = host(plan(dev(xp), z_x, z_y, lo, hi))
+    assert got.shape[:3] == want.shape[:3]
+    bad = np.argwhere(got[..., :n].astype(np.int32) != want)
+    assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[0]}: got {got[tuple(bad[0])]} want {want[tuple(bad[0])]}"
+    assert len(np.unique(want)) > 20                                 # the case is not degenerate
+
+
+STEM_SHAPES = [
+    # b, h, w, c, n, k, stride, pad
+    (2, 17, 15, 3, 32, 3, 2, 1),      # MobileNet stem shape (3 input channels, stride 2)
+    (1, 23, 21, 3, 64, 7, 2, 3),      # ResNet stem shape
+    (1, 9, 9, 5, 7, 3, 1, 1),         # odd channel counts, n not a multiple of 4
+    (3, 6, 7, 20, 70, 1, 1, 0),       # pointwise, ragged n tile
+    (1, 8, 8, 16, 16, 3, 1, 0),       # no padding
+    (1, 5, 5, 300, 10, 3, 1, 1),      # K = 2700 spans several K chunks
+    (1, 1, 1, 8, 8, 1, 1, 0),         # single output pixel
+]
+
+
+@pytest.mark.parametrize("shape", STEM_SHAPES)
+@pytest.mark.parametrize("wkind", [qtz.W_S8_PER_CHANNEL_SYM, qtz.W_U8_PER_LAYER_ASYM,
+                                   qtz.W_S4_PACKED_PER_CHANNEL_SYM])
+def test_conv_generic_shapes(hq, shape, wkind):
+    conv_case(hq, *shape, wkind, seed=100 + shape[1])
+
+
+@pytest.mark.parametrize("shape", STEM_SHAPES[:4])
+def test_conv_raw_int32_output(hq, shape):
+    conv_case(hq, *shape, qtz.W_U8_PER_LAYER_ASYM, seed=7, raw=True)
+    conv_case(hq, *shape, qtz.W_S8_PER_CHANNEL_SYM, seed=8, raw=True)
+
+
+@pytest.mark.parametrize("act", [0, 1, 2])
+def test_conv_activation_clamps(hq, act):
+    conv_case(hq, 1, 12, 12, 16, 24, 3, 1, 1, qtz.W_S8_PER_CHANNEL_SYM, seed=20 + act, act=act)
+
+
+# ---- layers the tensor-core path is meant for (1x1 / GEMM / 3x3 stride 1 pad 1) ------------
+TC_SHAPES = [
+    (1, 32, 32, 16, 32, 3, 1, 1),     # the single-conv workload's geometry (M=1024, K=144, N=32)
+    (2, 14, 14, 64, 96, 3, 1, 1),     # small image: pixel tiles span images
+    (3, 7, 7, 128, 48, 3, 1, 1),      # 7x7 image, C a full 128-byte K block
+    (1, 20, 18, 24, 40, 3, 1, 1),     # C = 24 (pitch 32), ragged tiles both ways
+    (4, 10, 10, 32, 64, 1, 1, 0),     # pointwise, M = 400: three full tiles and a ragged one
+    (1, 33, 31, 88, 136, 1, 1, 0),    # MobileNet-v2-1.4 widths, nothing a multiple of 16
+    (1, 16, 16, 256, 272, 1, 1, 0),   # two K blocks, N beyond one 256 tile
+    (2, 9, 9, 512, 24, 1, 1, 0),      # long K, narrow N
+    (1, 12, 12, 64, 32, 1, 2, 0),     # strided pointwise (ResNet down-sampling shortcut)
+]
+
+
+@pytest.mark.parametrize("shape", TC_SHAPES)
+@pytest.mark.parametrize("wkind", [qtz.W_S8_PER_CHANNEL_SYM, qtz.W_U8_PER_LAYER_ASYM,
+                                   qtz.W_S4_PACKED_PER_CHANNEL_SYM])
+def test_conv_tensor_core_shapes(hq, shape, wkind):
+    conv_case(hq, *shape, wkind, seed=200 + shape[3])
+
+
+@pytest.mark.parametrize("shape", TC_SHAPES[:5])
+def test_conv_tensor_core_raw(hq, shape):
+    conv_case(hq, *shape, qtz.W_U8_PER_LAYER_ASYM, seed=300 + shape[3], raw=True)
+
+
+def test_extreme_zero_points_and_codes(hq):
+    # all-255 inputs against all -128 / 255 weights with zero points at both ends
+    for wkind, wval, zw in [(qtz.W_S8_PER_CHANNEL_SYM, -128, None), (qtz.W_U8_PER_LAYER_ASYM, 255, 0),
+                            (qtz.W_U8_PER_LAYER_ASYM, 0, 255)]:
+        b, h, w, c, n = 1, 6, 6, 64, 16
+        x = np.full((b, h, w, c), 255, np.uint8)
+        codes = np.full((n, 3, 3, c), wval, np.int32)
+        api_w = codes.astype(np.int8 if wkind == qtz.W_S8_PER_CHANNEL_SYM else np.uint8)
+        for z_x in (0, 255):
+            z_w = None if zw is None else np.full(n, zw, np.int32)
+            acc = oracle.conv2d_acc(x, z_x, codes, z_w, None, 1, 1)
+            desc = qtz.conv_desc(b, h, w, c, n, 3, 3, 1, 1, wkind, qtz.OUT_S32_RAW)
+            plan = hq.conv_create(desc, dev(api_w), None, zw)
+            assert np.array_equal(host(plan(dev(x), z_x)), acc)
+
+
+# ---- workload 1: one quantized 3x3 convolution, every API call once -------------------------
+def test_single_conv_workload_end_to_end(hq):
+    t = synth.single_conv(seed=1)
+    x, w, bias = t["x"], t["w"], t["bias"]
+    n = w.shape[0]
+    # oracle side
+    xq_p = oracle.calibrate_minmax(x)
+    wq_p = oracle.calibrate_minmax(w, 0, 8, True)
+    xq = oracle.quantize(x, xq_p, None, 0, 255).astype(np.uint8)
+    wq = oracle.quantize(w, wq_p, 0, -127, 127)
+    bq = oracle.quantize_bias(bias, xq_p["scale"][0], wq_p["scale"])
+    z_x = int(xq_p["zero_point"][0])
+    acc = oracle.conv2d_acc(xq, z_x, wq, None, bq, 1, 1)
+    acc_p = np.zeros(n, oracle.QPARAMS)
+    acc_p["scale"] = (xq_p["scale"][0].astype(np.float32) * wq_p["scale"]).astype(np.float32)
+    real = np.clip(oracle.dequantize(acc, acc_p, 3), 0.0, 6.0)       # ReLU6 on the real values
+    yq_p = oracle.calibrate_minmax(real)
+    mr = [oracle.quantize_multiplier(float(xq_p["scale"][0]) * float(s) / float(yq_p["scale"][0]))
+          for s in wq_p["scale"]]
+    mult, rsh = [m for m, _ in mr], [r for _, r in mr]
+    z_y = int(yq_p["zero_point"][0])
+    lo, hi = oracle.activation_range(2, yq_p["scale"][0], z_y)
+    want = oracle.requantize(acc, np.array(mult, np.int32), np.array(rsh, np.int32), z_y, lo, hi)
+
+    # GPU side: the same steps through the C ABI
+    xd, wd = dev(x), dev(w)
+    g_xp = hq.calibrate_minmax(xd)
+    g_wp = hq.calibrate_minmax(wd, axis=0, symmetric=True)
+    assert g_xp.tobytes() == xq_p.tobytes() and g_wp.tobytes() == wq_p.tobytes()
+    assert z_x == 0 and np.isclose(float(g_xp["scale"][0]), 6.0 / 255.0, rtol=1e-3)
+    g_xq = hq.quantize_tensor(xd, g_xp)
+    g_wq = hq.quantize_tensor(wd, g_wp, axis=0, out_dtype=qtz.S8, restrict_range=True)
+    g_bq = hq.quantize_bias(dev(bias), g_xp["scale"][0], g_wp)
+    assert np.array_equal(host(g_xq), xq) and np.array_equal(host(g_wq).astype(np.int32), wq)
+    assert np.array_equal(host(g_bq), bq)
+    raw_plan = hq.conv_create(qtz.conv_desc(1, 32, 32, 16, n, 3, 3, 1, 1, outkind=qtz.OUT_S32_RAW), g_wq, g_bq)
+    g_acc = raw_plan(g_xq, z_x)
+    assert np.array_equal(host(g_acc), acc)
+    g_lo, g_hi = hq.minmax(hq.dequantize(g_acc, acc_p, axis=3))       # ReLU6 clamps the range itself
+    g_yp = np.atleast_1d(qtz.params_from_range(min(max(g_lo[0], 0.0), 6.0), min(max(g_hi[0], 0.0), 6.0)))
+    assert g_yp.tobytes() == yq_p.tobytes()
+    g_mr = [qtz.quantize_multiplier(float(g_xp["scale"][0]) * float(s) / float(g_yp["scale"][0]))
+            for s in g_wp["scale"]]
+    assert [m for m, _ in g_mr] == mult and [r for _, r in g_mr] == rsh
+    assert qtz.activation_range(2, g_yp["scale"][0], z_y) == (lo, hi)
+    plan = hq.conv_create(qtz.conv_desc(1, 32, 32, 16, n, 3, 3, 1, 1), g_wq, g_bq, None, mult, rsh)
+    got = host(plan(g_xq, z_x, z_y, lo, hi))
+    assert np.array_equal(got[..., :n].astype(np.int32), want)
+    # dequantized output agrees with the oracle's within 1e-6 relative
+    g_out = host(hq.dequantize(dev(np.ascontiguousarray(got[..., :n])), g_yp))
+    o_out = oracle.dequantize(want, yq_p, None)
+    assert np.allclose(g_out, o_out, rtol=1e-6, atol=0)
+
+
+# ---- workload 2: quantized GEMM, both operands asymmetric uint8 ------------------------------
+def gemm_case(hq, m, n, k, seed=2, rows=None):
+    t = synth.gemm_u8(m, n, k, seed)
+    a, b = t["a"], t["b"]
+    bt = np.ascontiguousarray(b.T).reshape(n, 1, 1, k)                # OHWI view of B
+    rows = np.arange(m) if rows is None else rows
+    acc = oracle.conv2d_acc(a[rows].reshape(len(rows), 1, 1, k), t["z_a"], bt.astype(np.int32),
+                            np.full(n, t["z_b"], np.int32), t["bias"], 1, 0).reshape(len(rows), n)
+    # one per-layer output quantizer from the accumulator range, replicated per channel
+    span = float(np.abs(acc).max()) + 1.0
+    m_q, r_q = oracle.quantize_multiplier(127.0 / span)
+    mult, rsh = np.full(n, m_q, np.int32), np.full(n, r_q, np.int32)
+    z_y = 128
+    want = oracle.requantize(acc, mult, rsh, z_y, 0, 255)
+    desc = qtz.conv_desc(m, 1, 1, k, n, 1, 1, 1, 0, qtz.W_U8_PER_LAYER_ASYM)
+    plan = hq.conv_create(desc, dev(bt), dev(t["bias"]), t["z_b"], mult, rsh)
+    got = host(plan(dev(a.reshape(m, 1, 1, k)), t["z_a"], z_y, 0, 255)).reshape(m, -1)
+    assert np.array_equal(got[rows][:, :n].astype(np.int32), want)
+    assert len(np.unique(want)) > 50
+    return plan.kernel
+
+
+@pytest.mark.parametrize("size", [512, 1024])
+def test_gemm_workload_full_parity(hq, size):
+    gemm_case(hq, size, size, size)
+
+
+@pytest.mark.parametrize("size", [2048, 4096, 8192])
+def test_gemm_workload_sampled_rows(hq, size):
+    rows = np.unique(np.concatenate([np.arange(0, 130), synth.rng(5, size).integers(0, size, 64),
+                                     np.arange(size - 3, size)]))
+    gemm_case(hq, size, size, size, rows=rows)
+
+
+def test_gemm_ragged(hq):
+    gemm_case(hq, 300, 200, 136)
+    gemm_case(hq, 129, 17, 1000)
+
+
+# ---- depthwise ---------------------------------------------------------------------------------
+DW_SHAPES = [(2, 14, 14, 32, 1), (1, 15, 13, 64, 2), (3, 7, 7, 24, 1), (1, 9, 10, 136, 2),
+             (2, 5, 5, 1024, 1), (1, 1, 1, 16, 1), (1, 2, 3, 8, 2), (1, 112, 112, 32, 1)]
+
+
+@pytest.mark.parametrize("shape", DW_SHAPES)
+@pytest.mark.parametrize("wkind", [qtz.W_S8_PER_CHANNEL_SYM, qtz.W_U8_PER_LAYER_ASYM,
+                                   qtz.W_S4_PACKED_PER_CHANNEL_SYM])
+def test_depthwise(hq, shape, wkind):
+    b, h, w, c, stride = shape
+    x = pitched(synth.uniform_u8((b, h, w, c), 31, c))
+    api_w, codes, zw = make_weights(wkind, (3, 3, c), 31 + c)
+    if wkind == qtz.W_S4_PACKED_PER_CHANNEL_SYM:
+        api_w = oracle.pack_s4(codes.reshape(9, c))
+    g = synth.rng(31, 72)
+    bias = g.integers(-3000, 3000, size=c).astype(np.int32)
+    z_x = int(g.integers(0, 256))
+    z_w = None if zw is None else np.full(c, zw, np.int32)
+    acc = oracle.depthwise_acc(x, z_x, codes, z_w, bias, stride, 1, c=c)
+    span = np.abs(acc).reshape(-1, c).max(axis=0).astype(np.float64) + 1.0
+    mr = [oracle.quantize_multiplier(float(v)) for v in 150.0 / span]
+    mult = np.array([m for m, _ in mr], np.int32)
+    rsh = np.array([r for _, r in mr], np.int32)
+    z_y = 30
+    want = oracle.requantize(acc, mult, rsh, z_y, z_y, 255)
+    desc = qtz.conv_desc(b, h, w, c, c, 3, 3, stride, 1, wkind)
+    plan = hq.conv_create(desc, dev(api_w), dev(bias), zw, mult, rsh, depthwise=True)
+    assert plan.kernel == "depthwise"
+    got = host(plan(dev(x), z_x, z_y, z_y, 255))
+    assert np.array_equal(got[..., :c].astype(np.int32), want)
+
+
+def test_conv_argument_errors(hq):
+    w = dev(np.zeros((8, 3, 3, 16), np.int8))
+    ones = np.full(8, 1 << 30, np.int32), np.full(8, 31, np.int32)
+    with pytest.raises(qtz.QtzError) as e:                                       # K too long
+        hq.conv_create(qtz.conv_desc(1, 8, 8, 4096, 8, 3, 3, 1, 1), w, None, None, *ones)
+    assert e.value.code == -4
+    with pytest.raises(qtz.QtzError) as e:                                       # bad pitch
+        hq.conv_create(qtz.conv_desc(1, 8, 8, 16, 8, 3, 3, 1, 1, c_pitch_in=24), w, None, None, *ones)
+    assert e.value.code == -2
+    with pytest.raises(qtz.QtzError) as e:                                       # missing z_w
+        hq.conv_create(qtz.conv_desc(1, 8, 8, 16, 8, 3, 3, 1, 1, qtz.W_U8_PER_LAYER_ASYM), w, None, None, *ones)
+    assert e.value.code == -1
+    with pytest.raises(qtz.QtzError) as e:                                       # 5x5 depthwise
+        hq.conv_create(qtz.conv_desc(1, 8, 8, 16, 16, 5, 5, 1, 2), w, None, None, np.ones(16, np.int32),
+                       np.ones(16, np.int32), depthwise=True)
+    assert e.value.code == -3
+    plan = hq.conv_create(qtz.conv_desc(1, 8, 8, 16, 8, 3, 3, 1, 1), w, None, None, *ones)
+    x = dev(np.zeros((1, 8, 8, 16), np.uint8))
+    y = plan.empty_output(x.device)
+    lib = hq.lib
+    assert lib.qtz_conv2d_u8(plan.plan, x.data_ptr(), 256, y.data_ptr(), 0, 0, 255, None) == -1
+    assert lib.qtz_conv2d_u8(plan.plan, x.data_ptr(), 0, y.data_ptr(), 0, 10, 5, None) == -1
+    assert lib.qtz_conv2d_u8(plan.plan, x.data_ptr() + 4, 0, y.data_ptr(), 0, 0, 255, None) == -2
+    assert lib.qtz_depthwise_u8(plan.plan, x.data_ptr(), 0, y.data_ptr(), 0, 0, 255, None) == -1
