@@ -1,10 +1,773 @@
-// Tensor-core (tcgen05) convolution path -- placeholder until the kernel lands.
-#include "qtz_plan.cuh"
+// Tensor-core convolution path of libqtz: 1x1 (GEMM) and 3x3 / stride 1 / pad 1 layers as an
+// implicit GEMM on the 5th-generation tensor cores.
+//
+//   raw[p][n] = sum_k x_Q[p][k] * w_Q[n][k]          tcgen05.mma kind::i8, u8 x s8 -> s32 in TMEM
+//   acc       = raw - z_x sum(w_Q) - z_w sum(x_Q) + K_valid z_x z_w + bias_q      (Eq. 5-6)
+//   y         = clamp(z_y + ((acc m_n + 2^(r_n - 1)) >> r_n))                     fused epilogue
+//
+// One persistent CTA per SM, warp-specialised:
+//   warp 0      TMA producer: NHWC activation boxes (one shifted box per filter tap; out-of-image
+//               pixels arrive as zeros) and K-major weight tiles into a ring of swizzled stages
+//   warp 1      MMA issuer: one thread issues tcgen05.mma; two accumulators of up to 256 columns
+//               alternate in TMEM so that the epilogue of tile i overlaps the MMAs of tile i+1
+//   warps 2..5  epilogue: tcgen05.ld, cross terms, requantise, clamp, pack to uint8 in swizzled
+//               shared memory, TMA store (which also clips ragged tile edges)
+// Zero filling stands for padding, so the -z_x sum(w) term must skip the padded taps as well:
+// the weight sums are tabulated per border class (which filter rows / columns are cut) and each
+// epilogue thread, owning one output pixel, picks its class.
+//
+// No cluster multicast is used anywhere.  Every device-side wait is bounded: when its cycle
+// budget runs out the kernel records (QTZ_ERR_DEVICE_TIMEOUT, site) in the handle's status word
+// and all roles drain and return.
+#include <algorithm>
+#include <cstring>
+#include <new>
+#include <vector>
 
-bool qtz_tc_supported(const qtz_conv_desc&) { return false; }
-qtz_status qtz_tc_prepare(qtz_plan*, const void*, cudaStream_t) { return QTZ_ERR_UNSUPPORTED; }
-void qtz_tc_release(qtz_plan*) {}
-qtz_status qtz_tc_launch(qtz_plan*, const uint8_t*, int32_t, void*, int32_t, int32_t, int32_t, cudaStream_t)
+#include "qtz_plan.cuh"
+#include "qtz_ptx.cuh"
+
+using namespace qtz_ptx;
+
+namespace {
+
+constexpr int kTileM = 128;          // rows of one accumulator (TMEM lanes)
+constexpr int kAccStride = 256;      // TMEM columns between the two accumulators
+constexpr int kTmemCols = 512;
+constexpr int kThreadsTc = 192;      // producer warp, MMA warp, four epilogue warps
+constexpr int kEpiThreads = 128;
+constexpr int kMaxStages = 8;
+constexpr int kMaxCls = 16;
+constexpr int kSmemBudget = 227 * 1024 - 1024;  // leave room for the 1 KB alignment slack
+
+struct TcArgs {
+    int32_t is4d;
+    int32_t tw, th, tb, rows;               // pixel box of one tile and its row count (<= 128)
+    int32_t tiles_w, tiles_h, n_tiles;
+    int64_t num_tiles;
+    int32_t W, H, B;                        // output extent (2-D case: W = number of pixels)
+    int32_t taps, kw, pad;
+    int32_t kb_per_tap, c_pad;
+    int32_t BK, BN, N, out_box, stages;
+    uint32_t idesc;
+    const int32_t* bias;
+    const int32_t* wsum;                    // [ncls][N]
+    const int32_t* mult;
+    const int32_t* rshift;
+    const int32_t* xsum;                    // per input pixel channel sums (only when zw != 0)
+    int32_t ncls;
+    int32_t kvalid[kMaxCls];
+    int32_t zx, zw, zy, act_min, act_max, raw, fast_requant;
+    int32_t* y_raw;
+    int32_t* status;
+    long long wait_budget;
+};
+
+struct SmemLayout {
+    uint32_t a_off, b_off, out_off, corr_off, mult_off, rsh_off, bar_off, total;
+    uint32_t a_stage, b_stage;
+};
+
+__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls)
 {
-    return QTZ_ERR_UNSUPPORTED;
+    SmemLayout L;
+    L.a_stage = kTileM * BK;
+    L.b_stage = BN * BK;
+    L.a_off = 0;
+    L.b_off = L.a_off + stages * L.a_stage;
+    L.out_off = L.b_off + stages * L.b_stage;
+    L.corr_off = L.out_off + kTileM * BN;
+    L.mult_off = L.corr_off + ncls * BN * 4;
+    L.rsh_off = L.mult_off + BN * 4;
+    L.bar_off = L.rsh_off + BN * 4;
+    L.total = L.bar_off + (2 * kMaxStages + 4) * 8 + 16;
+    return L;
+}
+
+__device__ __forceinline__ void report_timeout(int32_t* status, int site)
+{
+    if (atomicCAS(status, 0, QTZ_ERR_DEVICE_TIMEOUT) == 0) status[1] = site;
+}
+
+// Swizzled byte offset of (row, col) inside a staging box whose rows are `box` bytes long
+// (32, 64 or 128): the 16-byte chunk index is XORed with the low bits of (offset / 128).
+__device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t col, uint32_t box)
+{
+    const uint32_t off = row * box + col;
+    return off ^ (((off >> 7) & ((box >> 4) - 1)) << 4);
+}
+
+__global__ void __launch_bounds__(kThreadsTc, 1)
+conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_y, const TcArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
+    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls);
+
+    const uint32_t bar_full = base + L.bar_off;
+    const uint32_t bar_empty = bar_full + 8 * kMaxStages;
+    const uint32_t bar_tfull = bar_empty + 8 * kMaxStages;
+    const uint32_t bar_tempty = bar_tfull + 16;
+    volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + (2 * kMaxStages + 4) * 8);
+    volatile uint32_t* const abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < a.stages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_tfull + 8 * i, 1);
+            mbar_init(bar_tempty + 8 * i, kEpiThreads / 32);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+        prefetch_tensormap(&map_y);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int kblocks = a.taps * a.kb_per_tap;
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer ------------------------------
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t issued = 0;
+            const uint32_t tx = static_cast<uint32_t>(a.rows * a.BK + a.BN * a.BK);
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
+                const int n_tile = static_cast<int>(tile % a.n_tiles);
+                const int64_t m_tile = tile / a.n_tiles;
+                int w0 = 0, h0 = 0, b0 = 0;
+                if (a.is4d) {
+                    w0 = static_cast<int>(m_tile % a.tiles_w) * a.tw;
+                    h0 = static_cast<int>((m_tile / a.tiles_w) % a.tiles_h) * a.th;
+                    b0 = static_cast<int>(m_tile / (static_cast<int64_t>(a.tiles_w) * a.tiles_h)) * a.tb;
+                } else {
+                    w0 = static_cast<int>(m_tile) * kTileM;
+                }
+                for (int tap = 0; ok && tap < a.taps; ++tap) {
+                    const int dy = tap / a.kw - a.pad, dx = tap % a.kw - a.pad;
+                    for (int kb = 0; kb < a.kb_per_tap; ++kb) {
+                        if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget) || *abort_flag) {
+                            report_timeout(a.status, QTZ_SITE_SMEM_EMPTY);
+                            *abort_flag = 1;
+                            ok = false;
+                            break;
+                        }
+                        mbar_arrive_expect_tx(bar_full + 8 * stage, tx);
+                        const uint32_t dst_a = base + L.a_off + stage * L.a_stage;
+                        const uint32_t dst_b = base + L.b_off + stage * L.b_stage;
+                        if (a.is4d)
+                            tma_load_4d(dst_a, &map_a, bar_full + 8 * stage, kb * a.BK, w0 + dx, h0 + dy, b0);
+                        else
+                            tma_load_2d(dst_a, &map_a, bar_full + 8 * stage, kb * a.BK, w0);
+                        tma_load_2d(dst_b, &map_b, bar_full + 8 * stage, tap * a.c_pad + kb * a.BK, n_tile * a.BN);
+                        ++issued;
+                        if (++stage == static_cast<uint32_t>(a.stages)) {
+                            stage = 0;
+                            phase ^= 1;
+                        }
+                    }
+                }
+            }
+            if (!ok) {
+                // drain: give the copies already in flight a bounded time to land before the CTA exits
+                const uint32_t pending = issued < static_cast<uint32_t>(a.stages) ? issued : static_cast<uint32_t>(a.stages);
+                for (uint32_t i = 0; i < pending; ++i) {
+                    const uint32_t s = (stage + a.stages - 1 - i) % a.stages;
+                    const uint32_t ph = (s < stage) ? phase : (phase ^ 1);
+                    (void)mbar_wait(bar_full + 8 * s, ph, a.wait_budget);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer --------------------------------
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t local = 0;
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x, ++local) {
+                const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget) || *abort_flag) {
+                    report_timeout(a.status, QTZ_SITE_TMEM_EMPTY);
+                    *abort_flag = 1;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kAccStride;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, a.wait_budget) || *abort_flag) {
+                        report_timeout(a.status, QTZ_SITE_TMA_FULL);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint64_t da = make_kmajor_desc(base + L.a_off + stage * L.a_stage, a.BK);
+                    const uint64_t db = make_kmajor_desc(base + L.b_off + stage * L.b_stage, a.BK);
+                    for (int k = 0; k < a.BK / 32; ++k)  // each MMA consumes 32 bytes of K: advance 2 x 16 B
+                        mma_i8(d_tmem, da + 2 * k, db + 2 * k, a.idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    mma_commit(bar_empty + 8 * stage);  // frees the stage once these MMAs have read it
+                    if (++stage == static_cast<uint32_t>(a.stages)) {
+                        stage = 0;
+                        phase ^= 1;
+                    }
+                }
+                if (ok) mma_commit(bar_tfull + 8 * acc);
+            }
+        }
+    } else {
+        // ------------------------------ epilogue ----------------------------------
+        const int et = threadIdx.x - 64;             // 0..127
+        const int quarter = warp & 3;                // TMEM lane quarter this warp may read
+        const int row = quarter * 32 + lane;         // accumulator row owned by this thread
+        int32_t* const corr_s = reinterpret_cast<int32_t*>(smem + L.corr_off);
+        int32_t* const mult_s = reinterpret_cast<int32_t*>(smem + L.mult_off);
+        int32_t* const rsh_s = reinterpret_cast<int32_t*>(smem + L.rsh_off);
+        uint8_t* const out_s = smem + L.out_off;
+        const int boxes = a.BN / a.out_box;
+        const uint32_t box_bytes = kTileM * a.out_box;
+        int staged_n_tile = -1;
+        uint32_t local = 0;
+        for (int64_t tile = blockIdx.x; tile < a.num_tiles; tile += gridDim.x, ++local) {
+            const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
+            const int n_tile = static_cast<int>(tile % a.n_tiles);
+            const int64_t m_tile = tile / a.n_tiles;
+            const int n0 = n_tile * a.BN;
+
+            // the previous tile's TMA stores must have finished reading the staging buffer
+            if (et == 0) tma_store_wait_read();
+            if (n_tile != staged_n_tile) {
+                named_barrier(2, kEpiThreads);       // everyone is done with the old tables
+                for (int j = et; j < a.BN; j += kEpiThreads) {
+                    const int n = n0 + j;
+                    const bool live = n < a.N;
+                    const int32_t bias = live ? __ldg(a.bias + n) : 0;
+                    for (int c = 0; c < a.ncls; ++c) {
+                        const int32_t ws = live ? __ldg(a.wsum + static_cast<int64_t>(c) * a.N + n) : 0;
+                        corr_s[c * a.BN + j] = bias - a.zx * ws + a.kvalid[c] * a.zx * a.zw;
+                    }
+                    mult_s[j] = (live && !a.raw) ? __ldg(a.mult + n) : 0;
+                    rsh_s[j] = (live && !a.raw) ? __ldg(a.rshift + n) : 40;
+                }
+                staged_n_tile = n_tile;
+            }
+            named_barrier(1, kEpiThreads);
+
+            // which pixel this row is, its border class and its activation-sum term
+            int w0 = 0, h0 = 0, b0 = 0, pw, ph = 0, pb = 0;
+            bool row_live;
+            if (a.is4d) {
+                w0 = static_cast<int>(m_tile % a.tiles_w) * a.tw;
+                h0 = static_cast<int>((m_tile / a.tiles_w) % a.tiles_h) * a.th;
+                b0 = static_cast<int>(m_tile / (static_cast<int64_t>(a.tiles_w) * a.tiles_h)) * a.tb;
+                pw = w0 + row % a.tw;
+                ph = h0 + (row / a.tw) % a.th;
+                pb = b0 + row / (a.tw * a.th);
+                row_live = row < a.rows && pw < a.W && ph < a.H && pb < a.B;
+            } else {
+                w0 = static_cast<int>(m_tile) * kTileM;
+                pw = w0 + row;
+                row_live = pw < a.W;
+            }
+            int cls = 0;
+            if (a.ncls > 1) cls = ((ph == 0) | ((ph == a.H - 1) << 1)) * 4 + ((pw == 0) | ((pw == a.W - 1) << 1));
+            int32_t rowterm = 0;
+            if (a.zw != 0 && row_live) {
+                int32_t xs = 0;
+                if (a.taps == 1) {
+                    xs = __ldg(a.xsum + (static_cast<int64_t>(pb) * a.H + ph) * a.W + pw);
+                } else {
+                    for (int dy = -1; dy <= 1; ++dy)
+                        for (int dx = -1; dx <= 1; ++dx) {
+                            const int hh = ph + dy, ww = pw + dx;
+                            if (hh >= 0 && hh < a.H && ww >= 0 && ww < a.W)
+                                xs += __ldg(a.xsum + (static_cast<int64_t>(pb) * a.H + hh) * a.W + ww);
+                        }
+                }
+                rowterm = -a.zw * xs;
+            }
+            const int32_t* const corr_row = corr_s + cls * a.BN;
+
+            // all 128 epilogue threads take the same decision, so nobody is left alone at a barrier
+            if (!named_barrier_and(3, kEpiThreads, mbar_wait(bar_tfull + 8 * acc, acc_phase, a.wait_budget))) {
+                report_timeout(a.status, QTZ_SITE_TMEM_FULL);
+                *abort_flag = 1;
+                break;
+            }
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kAccStride;
+            const int32_t lo = a.act_min - a.zy, hi = a.act_max - a.zy;
+            const uint32_t zy4 = 0x01010101u * static_cast<uint32_t>(a.zy);
+
+            for (int j0 = 0; j0 < a.BN; j0 += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32(taddr + j0, v);
+                tmem_ld_wait();
+                if (n0 + j0 >= a.N) continue;        // a chunk entirely beyond the real channels
+                if (a.raw) {
+                    if (row_live) {
+                        const int64_t pix = a.is4d ? (static_cast<int64_t>(pb) * a.H + ph) * a.W + pw : pw;
+                        int32_t* out = a.y_raw + pix * a.N + n0 + j0;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + j0 + j < a.N) out[j] = static_cast<int32_t>(v[j]) + corr_row[j0 + j] + rowterm;
+                    }
+                    continue;
+                }
+                uint32_t packed[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int4 c4 = *reinterpret_cast<const int4*>(corr_row + j0 + 4 * q);
+                    const int4 m4 = *reinterpret_cast<const int4*>(mult_s + j0 + 4 * q);
+                    const int4 r4 = *reinterpret_cast<const int4*>(rsh_s + j0 + 4 * q);
+                    const int32_t cc[4] = {c4.x, c4.y, c4.z, c4.w}, mm[4] = {m4.x, m4.y, m4.z, m4.w},
+                                  rr[4] = {r4.x, r4.y, r4.z, r4.w};
+                    uint32_t word = 0;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int32_t full = static_cast<int32_t>(v[4 * q + e]) + cc[e] + rowterm;
+                        int32_t t;
+                        if (a.fast_requant) {
+                            // r >= 33: rounding constant 2^(r-1) sits in the high word; shift the high word only
+                            const int64_t prod = static_cast<int64_t>(full) * mm[e] +
+                                                 (static_cast<int64_t>(1u << (rr[e] - 33)) << 32);
+                            t = static_cast<int32_t>(prod >> 32) >> (rr[e] - 32);
+                            t = min(max(t, lo), hi);
+                        } else {
+                            const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(1) << (rr[e] - 1));
+                            const int64_t s = prod >> rr[e];
+                            t = static_cast<int32_t>(min(max(s, static_cast<int64_t>(lo)), static_cast<int64_t>(hi)));
+                        }
+                        word |= (static_cast<uint32_t>(t) & 0xffu) << (8 * e);
+                    }
+                    packed[q] = __vadd4(word, zy4);
+                }
+                const int box = j0 / a.out_box, col = j0 % a.out_box;
+                uint8_t* const dst = out_s + box * box_bytes;
+                *reinterpret_cast<uint4*>(dst + swz(row, col, a.out_box)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                *reinterpret_cast<uint4*>(dst + swz(row, col + 16, a.out_box)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+            }
+            // accumulator drained: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+
+            if (!a.raw) {
+                fence_proxy_async_smem();
+                named_barrier(1, kEpiThreads);
+                if (et == 0) {
+                    for (int bx = 0; bx < boxes; ++bx) {
+                        const int nn = n0 + bx * a.out_box;
+                        if (nn >= a.N) break;
+                        const uint32_t src = base + L.out_off + bx * box_bytes;
+                        if (a.is4d)
+                            tma_store_4d(&map_y, src, nn, w0, h0, b0);
+                        else
+                            tma_store_2d(&map_y, src, nn, w0);
+                    }
+                    tma_store_commit();
+                }
+            }
+        }
+        if (et == 0) tma_store_wait_all();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Preparation kernels (run once per layer) and small pre-passes
+// ------------------------------------------------------------------------------------------
+constexpr int kPrepThreads = 256;
+
+__device__ __forceinline__ int32_t api_code_s8(const void* w, int wkind, int64_t row, int64_t k, int64_t k_total)
+{
+    if (wkind == QTZ_W_S8_PER_CHANNEL_SYM) return static_cast<const int8_t*>(w)[row * k_total + k];
+    if (wkind == QTZ_W_U8_PER_LAYER_ASYM) return static_cast<int32_t>(static_cast<const uint8_t*>(w)[row * k_total + k]) - 128;
+    const uint32_t byte = static_cast<const uint8_t*>(w)[row * ((k_total + 1) >> 1) + (k >> 1)];
+    const uint32_t nib = (k & 1) ? (byte >> 4) : (byte & 0xfu);
+    return static_cast<int32_t>(nib << 28) >> 28;
+}
+
+// OHWI codes -> int8 [n_pad][taps][c_pad], zero padded (K-major rows for the B operand).
+__global__ void __launch_bounds__(kPrepThreads)
+prepack_tc_kernel(const void* __restrict__ w, int wkind, int n, int taps, int c, int n_pad, int c_pad, int8_t* __restrict__ out)
+{
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
+    const int64_t row_len = static_cast<int64_t>(taps) * c_pad;
+    if (i >= n_pad * row_len) return;
+    const int64_t row = i / row_len, rem = i - row * row_len;
+    const int tap = static_cast<int>(rem / c_pad), ch = static_cast<int>(rem - static_cast<int64_t>(tap) * c_pad);
+    out[i] = (row < n && ch < c) ? static_cast<int8_t>(api_code_s8(w, wkind, row, static_cast<int64_t>(tap) * c + ch, static_cast<int64_t>(taps) * c)) : 0;
+}
+
+// Weight sums per border class.  Class = 4 * rowclass + colclass, each a 2-bit mask
+// (bit 0: first filter row/column is outside the image, bit 1: last one is).
+__global__ void __launch_bounds__(kPrepThreads)
+class_sums_kernel(const int8_t* __restrict__ wp, int n, int taps, int kw, int c_pad, int ncls, int32_t* __restrict__ wsum)
+{
+    __shared__ int32_t tapsum[9];
+    const int row = blockIdx.x;
+    if (threadIdx.x < 9) tapsum[threadIdx.x] = 0;
+    __syncthreads();
+    for (int tap = 0; tap < taps; ++tap) {
+        int32_t s = 0;
+        for (int ch = threadIdx.x; ch < c_pad; ch += kPrepThreads) s += wp[(static_cast<int64_t>(row) * taps + tap) * c_pad + ch];
+        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+        if ((threadIdx.x & 31) == 0 && s != 0) atomicAdd(&tapsum[tap], s);
+    }
+    __syncthreads();
+    if (static_cast<int>(threadIdx.x) < ncls) {
+        const int cls = threadIdx.x, rc = cls >> 2, cc = cls & 3;
+        int32_t s = 0;
+        if (taps == 1) {
+            s = tapsum[0];
+        } else {
+            for (int i = 0; i < 3; ++i)
+                for (int j = 0; j < kw; ++j) {
+                    const bool cut = (i == 0 && (rc & 1)) || (i == 2 && (rc & 2)) || (j == 0 && (cc & 1)) || (j == 2 && (cc & 2));
+                    if (!cut) s += tapsum[i * kw + j];
+                }
+        }
+        wsum[static_cast<int64_t>(cls) * n + row] = s;
+    }
+}
+
+// xsum[p] = sum of the c channel codes of input pixel p (for the -z_w sum(x) term).
+__global__ void __launch_bounds__(kPrepThreads)
+pixel_sum_kernel(const uint8_t* __restrict__ x, int64_t pixels, int c, int pitch, int32_t* __restrict__ xsum)
+{
+    const int warps_per_block = kPrepThreads / 32;
+    const int lane = threadIdx.x & 31;
+    for (int64_t p = static_cast<int64_t>(blockIdx.x) * warps_per_block + (threadIdx.x >> 5); p < pixels;
+         p += static_cast<int64_t>(gridDim.x) * warps_per_block) {
+        const uint8_t* row = x + p * pitch;
+        uint32_t s = 0;
+        for (int off = lane * 16; off < c; off += 32 * 16) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(row + off));
+            uint32_t words[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int first = off + 4 * i;
+                uint32_t word = words[i];
+                if (first + 4 > c) word = first >= c ? 0u : (word & (0xffffffffu >> (8 * (first + 4 - c))));
+                s = __dp4a(word, 0x01010101u, s);
+            }
+        }
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) xsum[p] = static_cast<int32_t>(s);
+    }
+}
+
+// Strided 1x1 convolution: copies the pixels the layer actually reads into a compact tensor.
+__global__ void __launch_bounds__(kPrepThreads)
+stride_gather_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, int batch, int h, int w, int pitch,
+                     int stride, int oh, int ow)
+{
+    const int chunks = pitch >> 4;
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
+    if (t >= static_cast<int64_t>(batch) * oh * ow * chunks) return;
+    const int ck = static_cast<int>(t % chunks);
+    int64_t p = t / chunks;
+    const int ox = static_cast<int>(p % ow); p /= ow;
+    const int oy = static_cast<int>(p % oh);
+    const int64_t b = p / oh;
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + ((b * h + oy * stride) * w + ox * stride) * pitch) + ck);
+    reinterpret_cast<uint4*>(out)[t] = v;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------
+struct qtz_tc_state {
+    TcArgs args{};
+    CUtensorMap map_b{};
+    int8_t* w_packed = nullptr;
+    int32_t* xsum = nullptr;
+    int64_t in_pixels = 0;     // pixels of the (possibly gathered) input
+    int in_h = 0, in_w = 0;    // its spatial extent
+    int n_pad = 0;
+    int swizzle_k = 0, swizzle_out = 0;
+    uint32_t smem_bytes = 0;
+    int grid = 0;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        (void)cudaGetLastError();
+    }
+    return fn;
+}
+
+CUtensorMapSwizzle swizzle_for(int bytes)
+{
+    return bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+}
+
+// rank-2 or rank-4 uint8 tensor map; dims[0] is the contiguous dimension.
+bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                const uint32_t* box, int swizzle_bytes)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t gd[4], gs[3];
+    cuuint32_t bx[4], es[4];
+    for (int i = 0; i < rank; ++i) {
+        gd[i] = dims[i];
+        bx[i] = box[i];
+        es[i] = 1;
+        if (i > 0) gs[i - 1] = strides_bytes[i - 1];
+    }
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, static_cast<cuuint32_t>(rank), const_cast<void*>(base), gd, gs, bx, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(swizzle_bytes), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool is_pointwise(const qtz_conv_desc& d) { return d.kh == 1 && d.kw == 1 && d.pad == 0; }
+bool is_3x3(const qtz_conv_desc& d) { return d.kh == 3 && d.kw == 3 && d.pad == 1 && d.stride == 1; }
+
+}  // namespace
+
+bool qtz_tc_supported(const qtz_conv_desc& d)
+{
+    if (!(is_pointwise(d) || is_3x3(d))) return false;
+    if (d.c < 8) return false;  // tiny reductions (3-channel stems) stay on the CUDA-core kernel
+    if (is_pointwise(d) && d.stride > 4) return false;
+    return true;
+}
+
+void qtz_tc_release(qtz_plan* p)
+{
+    if (!p->tc) return;
+    cudaFree(p->tc->w_packed);
+    cudaFree(p->tc->xsum);
+    delete p->tc;
+    p->tc = nullptr;
+}
+
+qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
+{
+    qtz_ctx* h = p->h;
+    const qtz_conv_desc& d = p->d;
+    if (!encode_fn()) {
+        h->last_error = "cuTensorMapEncodeTiled is not available from the driver";
+        return QTZ_ERR_CUDA;
+    }
+    qtz_tc_state* t = new (std::nothrow) qtz_tc_state();
+    if (!t) return QTZ_ERR_INVALID_ARG;
+    p->tc = t;
+    TcArgs& a = t->args;
+    const bool pw = is_pointwise(d);
+    a.taps = pw ? 1 : 9;
+    a.kw = pw ? 1 : 3;
+    a.pad = pw ? 0 : 1;
+    a.N = d.n;
+    a.B = d.batch;
+    a.H = p->oh;
+    a.W = p->ow;
+    t->in_h = p->oh;  // after the optional stride gather the input has the output's extent
+    t->in_w = p->ow;
+    t->in_pixels = static_cast<int64_t>(d.batch) * p->oh * p->ow;
+
+    // K blocking: the widest swizzle the channel count fills reasonably
+    a.BK = d.c > 64 ? 128 : (d.c > 32 ? 64 : 32);
+    a.c_pad = (d.c + a.BK - 1) / a.BK * a.BK;
+    a.kb_per_tap = a.c_pad / a.BK;
+    // N tiling: as few tiles as possible, each a multiple of 32 columns
+    a.n_tiles = (d.n + 255) / 256;
+    a.BN = ((d.n + a.n_tiles - 1) / a.n_tiles + 31) / 32 * 32;
+    a.out_box = (a.BN % 128 == 0) ? 128 : ((a.BN % 64 == 0) ? 64 : 32);
+    t->n_pad = a.n_tiles * a.BN;
+    a.ncls = pw ? 1 : kMaxCls;
+
+    // pixel tiling
+    if (pw) {
+        a.is4d = 0;
+        a.tw = kTileM; a.th = 1; a.tb = 1; a.rows = kTileM;
+        a.tiles_w = static_cast<int32_t>((t->in_pixels + kTileM - 1) / kTileM);
+        a.tiles_h = 1;
+        a.num_tiles = static_cast<int64_t>(a.tiles_w) * a.n_tiles;
+        // the 2-D view treats all pixels as one row of length M
+        a.W = static_cast<int32_t>(t->in_pixels);
+        a.H = 1;
+        a.B = 1;
+        if (t->in_pixels > 0x7fffffff) return QTZ_ERR_UNSUPPORTED;
+    } else {
+        a.is4d = 1;
+        int64_t best_tiles = INT64_MAX;
+        for (int tw = 1; tw <= std::min(a.W, kTileM); ++tw)
+            for (int th = 1; th <= std::min(a.H, kTileM / tw); ++th) {
+                const int tb = std::min(a.B, kTileM / (tw * th));
+                const int64_t tiles = static_cast<int64_t>((a.W + tw - 1) / tw) * ((a.H + th - 1) / th) * ((a.B + tb - 1) / tb);
+                if (tiles < best_tiles || (tiles == best_tiles && tw > a.tw)) {
+                    best_tiles = tiles;
+                    a.tw = tw; a.th = th; a.tb = tb;
+                }
+            }
+        a.rows = a.tw * a.th * a.tb;
+        a.tiles_w = (a.W + a.tw - 1) / a.tw;
+        a.tiles_h = (a.H + a.th - 1) / a.th;
+        a.num_tiles = best_tiles * a.n_tiles;
+    }
+    for (int cls = 0; cls < kMaxCls; ++cls) {
+        const int rc = cls >> 2, cc = cls & 3;
+        const int rows_valid = pw ? 1 : 3 - (rc & 1) - ((rc >> 1) & 1);
+        const int cols_valid = pw ? 1 : 3 - (cc & 1) - ((cc >> 1) & 1);
+        a.kvalid[cls] = rows_valid * cols_valid * d.c;
+    }
+
+    // shared-memory budget -> pipeline depth
+    for (a.stages = kMaxStages; a.stages >= 2; --a.stages)
+        if (make_layout(a.BK, a.BN, a.stages, a.ncls).total <= static_cast<uint32_t>(kSmemBudget)) break;
+    if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
+    t->smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls).total + 1024;
+
+    // instruction descriptor: s32 accumulate, A = u8, B = s8, both K-major, N and M of the tile
+    a.idesc = (2u << 4) | (0u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) |
+              (static_cast<uint32_t>(kTileM >> 4) << 24);
+
+    // weights: re-lay, then the per-class sums
+    const int64_t wbytes = static_cast<int64_t>(t->n_pad) * a.taps * a.c_pad;
+    QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->w_packed), static_cast<size_t>(wbytes)));
+    prepack_tc_kernel<<<static_cast<unsigned>((wbytes + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
+        w_q_dev, d.wkind, d.n, a.taps, d.c, t->n_pad, a.c_pad, t->w_packed);
+    QTZ_LAUNCH_CHECK(h, "prepack_tc_kernel");
+    QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->wsum), sizeof(int32_t) * a.ncls * d.n));
+    class_sums_kernel<<<d.n, kPrepThreads, 0, st>>>(t->w_packed, d.n, a.taps, a.kw, a.c_pad, a.ncls, p->wsum);
+    QTZ_LAUNCH_CHECK(h, "class_sums_kernel");
+
+    if (p->w_zp_signed != 0)
+        QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->xsum), sizeof(int32_t) * static_cast<size_t>(t->in_pixels)));
+    if (pw && d.stride > 1)
+        QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->x_gather), static_cast<size_t>(t->in_pixels) * d.c_pitch_in));
+
+    // the weight map never changes
+    {
+        const uint64_t dims[2] = {static_cast<uint64_t>(a.taps) * a.c_pad, static_cast<uint64_t>(t->n_pad)};
+        const uint64_t strides[1] = {static_cast<uint64_t>(a.taps) * a.c_pad};
+        const uint32_t box[2] = {static_cast<uint32_t>(a.BK), static_cast<uint32_t>(a.BN)};
+        if (!encode_map(&t->map_b, t->w_packed, 2, dims, strides, box, a.BK)) {
+            h->last_error = "cuTensorMapEncodeTiled failed for the weight tensor";
+            return QTZ_ERR_CUDA;
+        }
+    }
+    a.bias = p->bias;
+    a.wsum = p->wsum;
+    a.mult = p->mult;
+    a.rshift = p->rshift;
+    a.xsum = t->xsum;
+    a.zw = p->w_zp_signed;
+    a.raw = d.outkind == QTZ_OUT_S32_RAW;
+    a.fast_requant = (!a.raw && p->rshift_min >= 33) ? 1 : 0;
+    a.status = h->status_dev;
+    a.wait_budget = 2000000000LL;  // about one second of SM clocks
+    t->grid = static_cast<int>(std::min<int64_t>(a.num_tiles, h->num_sms));
+
+    static bool attr_set = false;
+    if (!attr_set) {
+        QTZ_CUDA(h, cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_set = true;
+    }
+    return QTZ_OK;
+}
+
+qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, int32_t y_zp, int32_t act_min,
+                         int32_t act_max, cudaStream_t st)
+{
+    qtz_ctx* h = p->h;
+    qtz_tc_state* t = p->tc;
+    const qtz_conv_desc& d = p->d;
+    TcArgs a = t->args;
+    const bool pw = is_pointwise(d);
+
+    const uint8_t* xin = x;
+    if (pw && d.stride > 1) {
+        const int64_t work = t->in_pixels * (d.c_pitch_in >> 4);
+        stride_gather_kernel<<<static_cast<unsigned>((work + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
+            x, p->x_gather, d.batch, d.h, d.w, d.c_pitch_in, d.stride, p->oh, p->ow);
+        QTZ_LAUNCH_CHECK(h, "stride_gather_kernel");
+        xin = p->x_gather;
+    }
+    if (a.zw != 0) {
+        const int blocks = static_cast<int>(std::min<int64_t>((t->in_pixels + 7) / 8, static_cast<int64_t>(h->num_sms) * 16));
+        pixel_sum_kernel<<<blocks, kPrepThreads, 0, st>>>(xin, t->in_pixels, d.c, d.c_pitch_in, t->xsum);
+        QTZ_LAUNCH_CHECK(h, "pixel_sum_kernel");
+    }
+
+    CUtensorMap map_a, map_y;
+    const uint64_t pitch = static_cast<uint64_t>(d.c_pitch_in);
+    if (pw) {
+        const uint64_t dims[2] = {static_cast<uint64_t>(d.c), static_cast<uint64_t>(t->in_pixels)};
+        const uint64_t strides[1] = {pitch};
+        const uint32_t box[2] = {static_cast<uint32_t>(a.BK), static_cast<uint32_t>(kTileM)};
+        if (!encode_map(&map_a, xin, 2, dims, strides, box, a.BK)) return QTZ_ERR_CUDA;
+    } else {
+        const uint64_t dims[4] = {static_cast<uint64_t>(d.c), static_cast<uint64_t>(d.w), static_cast<uint64_t>(d.h),
+                                  static_cast<uint64_t>(d.batch)};
+        const uint64_t strides[3] = {pitch, pitch * d.w, pitch * d.w * d.h};
+        const uint32_t box[4] = {static_cast<uint32_t>(a.BK), static_cast<uint32_t>(a.tw), static_cast<uint32_t>(a.th),
+                                 static_cast<uint32_t>(a.tb)};
+        if (!encode_map(&map_a, xin, 4, dims, strides, box, a.BK)) return QTZ_ERR_CUDA;
+    }
+    if (a.raw) {
+        map_y = t->map_b;  // unused by the kernel in this mode
+        a.y_raw = static_cast<int32_t*>(y);
+    } else {
+        const uint64_t opitch = static_cast<uint64_t>(d.c_pitch_out);
+        if (pw) {
+            const uint64_t dims[2] = {static_cast<uint64_t>(d.n), static_cast<uint64_t>(t->in_pixels)};
+            const uint64_t strides[1] = {opitch};
+            const uint32_t box[2] = {static_cast<uint32_t>(a.out_box), static_cast<uint32_t>(kTileM)};
+            if (!encode_map(&map_y, y, 2, dims, strides, box, a.out_box)) return QTZ_ERR_CUDA;
+        } else {
+            const uint64_t dims[4] = {static_cast<uint64_t>(d.n), static_cast<uint64_t>(p->ow), static_cast<uint64_t>(p->oh),
+                                      static_cast<uint64_t>(d.batch)};
+            const uint64_t strides[3] = {opitch, opitch * p->ow, opitch * p->ow * p->oh};
+            const uint32_t box[4] = {static_cast<uint32_t>(a.out_box), static_cast<uint32_t>(a.tw), static_cast<uint32_t>(a.th),
+                                     static_cast<uint32_t>(a.tb)};
+            if (!encode_map(&map_y, y, 4, dims, strides, box, a.out_box)) return QTZ_ERR_CUDA;
+        }
+    }
+    a.zx = x_zp;
+    a.zy = y_zp;
+    a.act_min = act_min;
+    a.act_max = act_max;
+    conv_tc_kernel<<<t->grid, kThreadsTc, t->smem_bytes, st>>>(map_a, t->map_b, map_y, a);
+    QTZ_LAUNCH_CHECK(h, "conv_tc_kernel");
+    return QTZ_OK;
 }

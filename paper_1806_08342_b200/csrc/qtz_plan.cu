@@ -1,5 +1,6 @@
 // Per-layer preparation (weights are constant at inference, Section 2.1) and dispatch of
 // the convolution entry points.
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -146,6 +147,8 @@ extern "C" qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, i
     p->ow = (d.w + 2 * d.pad - d.kw) / d.stride + 1;
     p->k_total = depthwise ? d.kh * d.kw : d.kh * d.kw * d.c;
     p->w_zp_signed = d.wkind == QTZ_W_U8_PER_LAYER_ASYM ? *w_zero_point_host - 128 : 0;
+    if (!raw)
+        for (int i = 0; i < d.n; ++i) p->rshift_min = std::min(p->rshift_min, rshift_host[i]);
 
 #define PLAN_CUDA(expr)                                        \
     do {                                                       \

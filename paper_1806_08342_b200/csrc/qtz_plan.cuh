@@ -18,6 +18,7 @@ struct qtz_plan {
     int k_total = 0;      // kh*kw*c
     int k_padded = 0;     // row length of w_direct (multiple of 16)
     int n_padded = 0;     // rows of w_direct (multiple of 64)
+    int rshift_min = 62;  // smallest per-channel right shift (selects the epilogue's requantise form)
     int w_zp_signed = 0;  // weight zero point after moving codes to int8 (z_w - 128 for uint8 weights)
 
     int8_t* w_direct = nullptr;   // [n_padded][k_padded] int8, zero padded       (direct path)

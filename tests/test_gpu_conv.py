@@ -21,13 +21,13 @@ def make_weights(wkind, shape, seed):
         return codes.astype(np.int8), codes, None
     if wkind == qtz.W_U8_PER_LAYER_ASYM:
         codes = g.integers(0, 256, size=shape).astype(np.int32)
-        return codes.astype(np.uint8), codes, int(g.integers(0, 256))
+        return codes.astype(np.uint8), codes, int(g.integers(64, 192))
     codes = g.integers(-8, 8, size=shape).astype(np.int32)
     codes.flat[0] = -8
     return None, codes, None                                        # packed by the caller (layout differs)
 
 
-def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=2, expect_kernel=None):
+def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=0, expect_kernel=None):
     x = synth.uniform_u8((b, h, w, c), seed, 1)
     xp = pitched(x)
     api_w, codes, zw = make_weights(wkind, (n, k, k, c), seed)
@@ -35,7 +35,7 @@ def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=2, 
         api_w = oracle.pack_s4(codes.reshape(n, -1))
     g = synth.rng(seed, 71)
     bias = g.integers(-20000, 20000, size=n).astype(np.int32)
-    z_x = int(g.integers(0, 256))
+    z_x = int(g.integers(64, 192))
     z_w = None if zw is None else np.full(n, zw, np.int32)
     acc = oracle.conv2d_acc(xp, z_x, codes, z_w, bias, stride, pad, c=c)
     desc = qtz.conv_desc(b, h, w, c, n, k, k, stride, pad, wkind, qtz.OUT_S32_RAW if raw else qtz.OUT_U8)
@@ -49,11 +49,11 @@ def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=2, 
         return
     # per-channel multipliers spread over two decades so that outputs use the whole code range
     span = np.abs(acc).reshape(-1, n).max(axis=0).astype(np.float64) + 1.0
-    real_m = 200.0 / span * np.exp(g.uniform(-1.0, 1.0, size=n))
+    real_m = 100.0 / span * np.exp(g.uniform(-1.0, 1.0, size=n))
     mr = [oracle.quantize_multiplier(float(v)) for v in real_m]
     mult = np.array([m for m, _ in mr], np.int32)
     rsh = np.array([r for _, r in mr], np.int32)
-    z_y = int(g.integers(0, 200))
+    z_y = int(g.integers(100, 156))
     lo, hi = {0: (0, 255), 1: (z_y, 255), 2: (z_y, min(255, z_y + 120))}[act]
     want = oracle.requantize(acc, mult, rsh, z_y, lo, hi)
     plan = hq.conv_create(desc, dev(api_w), dev(bias), zw, mult, rsh)
@@ -63,7 +63,7 @@ def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=2, 
     assert got.shape[:3] == want.shape[:3]
     bad = np.argwhere(got[..., :n].astype(np.int32) != want)
     assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[0]}: got {got[tuple(bad[0])]} want {want[tuple(bad[0])]}"
-    assert len(np.unique(want)) > 20                                 # the case is not degenerate
+    assert want.size < 2000 or len(np.unique(want)) > 20             # the case is not degenerate
 
 
 STEM_SHAPES = [
@@ -114,12 +114,12 @@ TC_SHAPES = [
 @pytest.mark.parametrize("wkind", [qtz.W_S8_PER_CHANNEL_SYM, qtz.W_U8_PER_LAYER_ASYM,
                                    qtz.W_S4_PACKED_PER_CHANNEL_SYM])
 def test_conv_tensor_core_shapes(hq, shape, wkind):
-    conv_case(hq, *shape, wkind, seed=200 + shape[3])
+    conv_case(hq, *shape, wkind, seed=200 + shape[3], expect_kernel="tcgen05")
 
 
 @pytest.mark.parametrize("shape", TC_SHAPES[:5])
 def test_conv_tensor_core_raw(hq, shape):
-    conv_case(hq, *shape, qtz.W_U8_PER_LAYER_ASYM, seed=300 + shape[3], raw=True)
+    conv_case(hq, *shape, qtz.W_U8_PER_LAYER_ASYM, seed=300 + shape[3], raw=True, expect_kernel="tcgen05")
 
 
 def test_extreme_zero_points_and_codes(hq):
@@ -198,6 +198,7 @@ def gemm_case(hq, m, n, k, seed=2, rows=None):
     a, b = t["a"], t["b"]
     bt = np.ascontiguousarray(b.T).reshape(n, 1, 1, k)                # OHWI view of B
     rows = np.arange(m) if rows is None else rows
+    ap = pitched(a)
     acc = oracle.conv2d_acc(a[rows].reshape(len(rows), 1, 1, k), t["z_a"], bt.astype(np.int32),
                             np.full(n, t["z_b"], np.int32), t["bias"], 1, 0).reshape(len(rows), n)
     # one per-layer output quantizer from the accumulator range, replicated per channel
@@ -208,9 +209,10 @@ def gemm_case(hq, m, n, k, seed=2, rows=None):
     want = oracle.requantize(acc, mult, rsh, z_y, 0, 255)
     desc = qtz.conv_desc(m, 1, 1, k, n, 1, 1, 1, 0, qtz.W_U8_PER_LAYER_ASYM)
     plan = hq.conv_create(desc, dev(bt), dev(t["bias"]), t["z_b"], mult, rsh)
-    got = host(plan(dev(a.reshape(m, 1, 1, k)), t["z_a"], z_y, 0, 255)).reshape(m, -1)
+    got = host(plan(dev(ap.reshape(m, 1, 1, -1)), t["z_a"], z_y, 0, 255)).reshape(m, -1)
     assert np.array_equal(got[rows][:, :n].astype(np.int32), want)
     assert len(np.unique(want)) > 50
+    assert plan.kernel == "tcgen05"
     return plan.kernel
 
 
