@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized-convolution hot path on B200.
+
+Workload (default): the quantized GEMM sweep -- uint8 A (MxK) times uint8 B (KxN), both
+asymmetric per layer with zero points in [0,255], int32 bias, uint8 output, M=N=K in
+{512, 1024, 2048, 4096, 8192}.  One step = one pass over the five sizes through
+qtz_conv2d_u8 (activation-sum pre-pass + tcgen05 implicit-GEMM kernel with the fused
+zero-point / requantize epilogue).  Metric: int8 TOP/s, 2 ops per multiply-accumulate of the
+method itself (no padding, no cross-term work counted).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line on rank 0.  With --impl reference the CPU oracle is timed instead
+(a deliberately plain program: a reported baseline, not a target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1806_08342_b200 import synth  # noqa: E402
+
+SIZES = synth.GEMM_SIZES
+METRIC, UNIT = "int8_tops", "TOP/s"
+WORKLOAD = "quantized GEMM sweep u8xu8 asymmetric, M=N=K in {512,1024,2048,4096,8192}, int32 bias, u8 out"
+
+
+def step_ops(sizes=None):
+    return float(sum(2.0 * s * s * s for s in (SIZES if sizes is None else sizes)))
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_burst": float(p["bf16_tflops"]),
+                "bf16_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        busy = [v for v in sm if v > 0]
+        return {"sm_mhz": float(np.median(busy)) if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle leg
+# ------------------------------------------------------------------------------------------
+def oracle_sample(rows_per_size, seed=2):
+    """Runs the oracle on the first `rows` rows of A for each GEMM size; returns (ops, seconds)."""
+    import oracle
+    ops, secs = 0.0, 0.0
+    for size, rows in rows_per_size.items():
+        if rows <= 0:
+            continue
+        t = synth.gemm_u8(rows, size, size, seed)
+        bt = np.ascontiguousarray(t["b"].T).reshape(size, 1, 1, size).astype(np.int32)
+        a = t["a"].reshape(rows, 1, 1, size)
+        zw = np.full(size, t["z_b"], np.int32)
+        m, r = oracle.quantize_multiplier(1e-6)
+        mult, rsh = np.full(size, m, np.int32), np.full(size, r, np.int32)
+        t0 = time.perf_counter()
+        acc = oracle.conv2d_acc(a, t["z_a"], bt, zw, t["bias"], 1, 0)
+        oracle.requantize(acc, mult, rsh, 128, 0, 255)
+        secs += time.perf_counter() - t0
+        ops += 2.0 * rows * size * size
+    return ops, secs
+
+
+def cpu_baseline(target_seconds=15.0):
+    import oracle
+    oracle.build()
+    probe = {SIZES[-1]: 32}
+    ops, secs = oracle_sample(probe)
+    rate = ops / max(secs, 1e-9)
+    budget_ops = rate * target_seconds
+    # same row fraction of every size, so the sample has the sweep's mix of shapes
+    frac = min(1.0, budget_ops / step_ops())
+    rows = {s: max(1, int(round(s * frac))) for s in SIZES}
+    ops, secs = oracle_sample(rows)
+    return {"value": ops / secs / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "first rows of A per size " + json.dumps({str(k): v for k, v in rows.items()}) +
+                      f" against full B ({ops / 1e9:.1f} GOP in {secs:.1f} s)"}
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    probe_ops, probe_s = oracle_sample({8192: 4})
+    rate = probe_ops / max(probe_s, 1e-9)
+    per_step_s = min(8.0, 150.0 / max(1, args.steps + args.warmup))
+    frac = min(1.0, rate * per_step_s / step_ops())
+    rows = {s: max(1, int(round(s * frac))) for s in SIZES}
+    for _ in range(args.warmup):
+        oracle_sample(rows)
+    ops = secs = 0.0
+    for _ in range(args.steps):
+        o, s = oracle_sample(rows)
+        ops += o; secs += s
+    val = ops / secs / 1e12
+    sample = "per step: first rows of A per size " + json.dumps({str(k): v for k, v in rows.items()}) + " against full B"
+    out = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+           "config": {"workload": WORKLOAD, "note": "CPU oracle on host cores; bounded row sample of the workload"},
+           "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+           "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+# GPU leg
+# ------------------------------------------------------------------------------------------
+class GemmCase:
+    """One size of the sweep, resident in HBM: plan, input, output, host copies for the e2e leg."""
+
+    def __init__(self, hq, qtz, torch, size, seed=2):
+        t = synth.gemm_u8(size, size, size, seed)
+        self.size = size
+        self.z_a, self.z_b = t["z_a"], t["z_b"]
+        self.a_host = torch.from_numpy(t["a"].reshape(size, 1, 1, size)).pin_memory()
+        self.a = self.a_host.cuda()
+        bt = torch.from_numpy(np.ascontiguousarray(t["b"].T)).cuda()         # OHWI view of B
+        bias = torch.from_numpy(t["bias"]).cuda()
+        # output quantizer: range of the accumulators, measured with the library itself
+        raw = hq.conv_create(qtz.conv_desc(size, 1, 1, size, size, 1, 1, 1, 0, qtz.W_U8_PER_LAYER_ASYM,
+                                           qtz.OUT_S32_RAW), bt, bias, self.z_b)
+        acc = raw(self.a, self.z_a)
+        unit = np.zeros(1, qtz.QPARAMS); unit["scale"] = 1.0
+        lo, hi = hq.minmax(hq.dequantize(acc.view(-1), unit))
+        raw.close(); del acc
+        m, r = qtz.quantize_multiplier(127.0 / (max(abs(float(lo[0])), abs(float(hi[0]))) + 1.0))
+        self.plan = hq.conv_create(qtz.conv_desc(size, 1, 1, size, size, 1, 1, 1, 0, qtz.W_U8_PER_LAYER_ASYM),
+                                   bt, bias, self.z_b, np.full(size, m, np.int32), np.full(size, r, np.int32))
+        self.y = self.plan.empty_output("cuda")
+        self.y_host = torch.empty(self.y.shape, dtype=torch.uint8).pin_memory()
+        self.ops = 2.0 * size ** 3
+
+    def run(self):
+        self.plan(self.a, self.z_a, 128, 0, 255, out=self.y)
+
+
+def time_hbm_kernels(hq, qtz, torch, peaks):
+    """Achieved GB/s of the element-wise and depthwise kernels (algorithmic bytes / event time)."""
+    res = {}
+    n = 1 << 28                                                    # 1 GiB of fp32: far larger than L2
+    x = torch.empty(n, dtype=torch.float32, device="cuda").uniform_(-1.0, 6.0)
+    p = hq.calibrate_minmax(x)
+    q = hq.quantize_tensor(x, p)
+
+    def timed(fn, reps=5):
+        fn(); torch.cuda.synchronize()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        for _ in range(reps):
+            fn()
+        e.record(); torch.cuda.synchronize()
+        return s.elapsed_time(e) / reps * 1e-3
+
+    def entry(name, secs, nbytes):
+        gbs = nbytes / secs / 1e9
+        res[name] = {"GB/s": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 3),
+                     "ms": round(secs * 1e3, 4)}
+
+    entry("minmax_f32 (4 B/elem)", timed(lambda: hq.minmax(x)), 4.0 * n)
+    entry("quantize_f32_to_u8 (5 B/elem)", timed(lambda: hq.quantize_tensor(x, p, out=q)), 5.0 * n)
+    entry("dequantize_u8_to_f32 (5 B/elem)", timed(lambda: hq.dequantize(q, p, out=x)), 5.0 * n)
+    del x, q
+    # MobileNet-v1 depthwise layers at batch 128: (H, C, stride)
+    for hh, c, stride in [(112, 64, 2), (56, 128, 1), (14, 512, 1)]:
+        xin = torch.randint(0, 256, (128, hh, hh, c), dtype=torch.uint8, device="cuda")
+        w = torch.randint(-127, 128, (3, 3, c), dtype=torch.int8, device="cuda")
+        m, r = qtz.quantize_multiplier(1.0 / 600.0)
+        plan = hq.conv_create(qtz.conv_desc(128, hh, hh, c, c, 3, 3, stride, 1), w, None, None,
+                              np.full(c, m, np.int32), np.full(c, r, np.int32), depthwise=True)
+        y = plan.empty_output("cuda")
+        secs = timed(lambda: plan(xin, 3, 10, 10, 255, out=y), reps=10)
+        entry(f"depthwise3x3 128x{hh}x{hh}x{c} s{stride}", secs, float(xin.numel() + y.numel()))
+        plan.close()
+    a = torch.randint(0, 256, (1 << 28,), dtype=torch.uint8, device="cuda").view(-1, 64)
+    b = torch.randint(0, 256, (1 << 28,), dtype=torch.uint8, device="cuda").view(-1, 64)
+    ma, mb, r = qtz.add_params(0.02, 0.03, 0.04)
+    out = torch.empty_like(a)
+    entry("add_u8 (3 B/elem)", timed(lambda: hq.add_u8(a, 3, ma, b, 5, mb, r, 0, 0, 255, 64, out=out)), 3.0 * a.numel())
+    return res
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    from paper_1806_08342_b200 import build as qbuild
+    qbuild.build()
+    from paper_1806_08342_b200 import qtz
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    peaks = load_peaks()
+    hq = qtz.Handle(local_rank)
+    cases = [GemmCase(hq, qtz, torch, s) for s in SIZES]
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        for c in cases:
+            c.run()
+    # per-launch events of the dominant kernel (recorded by the library around its main kernel)
+    kev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in cases]
+           for _ in range(args.steps)]
+    for row in kev:
+        for s, e in row:
+            s.record(); e.record()
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for step in range(args.steps):
+        for c, (s, e) in zip(cases, kev[step]):
+            c.plan.set_profile_events(s, e)
+            c.run()
+    t1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = t0.elapsed_time(t1)
+    for c in cases:
+        c.plan.set_profile_events(None, None)
+    rc, site = hq.device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} at site {site}")
+    per_size_ms = [float(np.mean([kev[st][i][0].elapsed_time(kev[st][i][1]) for st in range(args.steps)]))
+                   for i in range(len(cases))]
+
+    # end to end: host buffers in, host buffers out, copies inside the timed region
+    e2e_steps = max(1, min(args.steps, 5))
+    for c in cases:
+        c.a.copy_(c.a_host, non_blocking=True); c.run(); c.y_host.copy_(c.y, non_blocking=True)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        for c in cases:
+            c.a.copy_(c.a_host, non_blocking=True)
+            c.run()
+            c.y_host.copy_(c.y, non_blocking=True)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = float(t[0]), float(t[1])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    ops = step_ops()
+    value = world * ops * args.steps / (ms * 1e-3) / 1e12
+    int8_peak = 2.0 * peaks["bf16_burst"]          # dense int8 : bf16 is 2 : 1 on this part (4.5 vs 2.25 POP/s nominal)
+    kernel_tops = ops / (sum(per_size_ms) * 1e-3) / 1e12
+    sweep = {str(c.size): {"kernel_ms": round(per_size_ms[i], 4),
+                           "TOP/s": round(c.ops / (per_size_ms[i] * 1e-3) / 1e12, 1),
+                           "frac_of_int8_peak": round(c.ops / (per_size_ms[i] * 1e-3) / 1e12 / int8_peak, 3)}
+             for i, c in enumerate(cases)}
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u8*s8->s32", "data": "synthetic",
+        "config": {"workload": WORKLOAD if len(SIZES) == 5 else WORKLOAD + f" [subset {list(SIZES)}]", "parallelism": f"replicas x{world}",
+                   "l2": "operands larger than L2: 268 MB touched per step, 201 MB by the largest size alone",
+                   "kernels_per_step": "5 x (pixel_sum_kernel + conv_tc_kernel)"},
+        "clocks": clocks,
+        "e2e": {"value": world * ops * e2e_steps / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+                "h2d_bytes_per_step": int(sum(c.a_host.numel() for c in cases)),
+                "d2h_bytes_per_step": int(sum(c.y_host.numel() for c in cases)), "steps": e2e_steps},
+        "gpu_launches": 2 * len(cases) * args.steps,
+        "roofline": {"bound": "tensor", "kernel": "conv_tc_kernel", "achieved": kernel_tops, "peak": int8_peak,
+                     "unit": UNIT, "frac": kernel_tops / int8_peak, "traffic": None,
+                     "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_burst']} TFLOP/s x 2 (int8:bf16 nominal ratio)",
+                     "frac_of_sustained_peak": kernel_tops / (2.0 * peaks["bf16_sustained"]),
+                     "frac_of_nominal_4500": kernel_tops / 4500.0},
+        "sweep": sweep,
+    }
+    if world == 1 and not args.no_extras:
+        out["hbm_kernels"] = time_hbm_kernels(hq, qtz, torch, peaks)
+        out["cpu_baseline"] = cpu_baseline()
+    print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the HBM-kernel table and the CPU baseline")
+    ap.add_argument("--sizes", default="", help="comma-separated subset of the sweep (profiling runs); default: all")
+    args = ap.parse_args()
+    if args.sizes:
+        global SIZES
+        SIZES = tuple(int(v) for v in args.sizes.split(","))
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -265,8 +265,10 @@ qtz_status qtz_direct_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* 
     const int64_t px_tiles = (a.pixels + kTilePx - 1) / kTilePx;
     if (px_tiles > 0x7fffffff) return QTZ_ERR_UNSUPPORTED;
     dim3 grid(static_cast<unsigned>(px_tiles), static_cast<unsigned>(p->n_padded / kTileN));
+    if (p->ev_start) QTZ_CUDA(p->h, cudaEventRecord(p->ev_start, st));
     direct_conv_kernel<<<grid, kDirectThreads, 0, st>>>(a);
     QTZ_LAUNCH_CHECK(p->h, "direct_conv_kernel");
+    if (p->ev_stop) QTZ_CUDA(p->h, cudaEventRecord(p->ev_stop, st));
     return QTZ_OK;
 }
 
@@ -282,10 +284,12 @@ qtz_status qtz_depthwise_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, uin
     const int64_t total = static_cast<int64_t>(d.batch) * p->oh * a.strips * ((d.c + 3) / 4);
     const int64_t blocks = (total + kDwThreads - 1) / kDwThreads;
     if (blocks > 0x7fffffff) return QTZ_ERR_UNSUPPORTED;
+    if (p->ev_start) QTZ_CUDA(p->h, cudaEventRecord(p->ev_start, st));
     if (d.stride == 1)
         depthwise3x3_kernel<1><<<static_cast<unsigned>(blocks), kDwThreads, 0, st>>>(a);
     else
         depthwise3x3_kernel<2><<<static_cast<unsigned>(blocks), kDwThreads, 0, st>>>(a);
     QTZ_LAUNCH_CHECK(p->h, "depthwise3x3_kernel");
+    if (p->ev_stop) QTZ_CUDA(p->h, cudaEventRecord(p->ev_stop, st));
     return QTZ_OK;
 }

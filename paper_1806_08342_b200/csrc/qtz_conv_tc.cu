@@ -767,7 +767,9 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.zy = y_zp;
     a.act_min = act_min;
     a.act_max = act_max;
+    if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
     conv_tc_kernel<<<t->grid, kThreadsTc, t->smem_bytes, st>>>(map_a, t->map_b, map_y, a);
     QTZ_LAUNCH_CHECK(h, "conv_tc_kernel");
+    if (p->ev_stop) QTZ_CUDA(h, cudaEventRecord(p->ev_stop, st));
     return QTZ_OK;
 }

@@ -110,6 +110,14 @@ extern "C" qtz_status qtz_conv_destroy(qtz_conv_plan p)
     return QTZ_OK;
 }
 
+extern "C" qtz_status qtz_conv_set_profile_events(qtz_conv_plan p, void* start_event, void* stop_event)
+{
+    if (!p || ((start_event == nullptr) != (stop_event == nullptr))) return QTZ_ERR_INVALID_ARG;
+    p->ev_start = static_cast<cudaEvent_t>(start_event);
+    p->ev_stop = static_cast<cudaEvent_t>(stop_event);
+    return QTZ_OK;
+}
+
 extern "C" const char* qtz_conv_plan_kernel(qtz_conv_plan p)
 {
     if (!p) return "";

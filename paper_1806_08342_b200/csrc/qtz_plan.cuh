@@ -29,6 +29,7 @@ struct qtz_plan {
     int32_t* rshift = nullptr;    // [n]
     uint8_t* x_gather = nullptr;  // strided 1x1 layers: the sub-sampled input, pitched NHWC
     qtz_tc_state* tc = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_stop = nullptr;  // optional profiling hook
 };
 
 // Direct (CUDA-core) path.

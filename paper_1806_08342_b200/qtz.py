@@ -62,6 +62,7 @@ SIGNATURES = {
                                   c_void_p, POINTER(c_void_p), c_void_p]),
     "qtz_conv_destroy": (c_int32, [c_void_p]),
     "qtz_conv_plan_kernel": (c_char_p, [c_void_p]),
+    "qtz_conv_set_profile_events": (c_int32, [c_void_p, c_void_p, c_void_p]),
     "qtz_conv2d_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p]),
     "qtz_depthwise_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p]),
     "qtz_add_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p,
@@ -310,6 +311,12 @@ class ConvPlan:
         self.handle._chk(fn(self.plan, _ptr(x), int(x_zero_point), _ptr(out), int(y_zero_point), int(act_min),
                             int(act_max), _stream()), "qtz_depthwise_u8" if self.depthwise else "qtz_conv2d_u8")
         return out
+
+    def set_profile_events(self, start=None, stop=None):
+        """start/stop: torch.cuda.Event(enable_timing=True) already created (recorded once), or None."""
+        s = None if start is None else c_void_p(start.cuda_event)
+        e = None if stop is None else c_void_p(stop.cuda_event)
+        self.handle._chk(self.handle.lib.qtz_conv_set_profile_events(self.plan, s, e), "qtz_conv_set_profile_events")
 
     def close(self):
         if self.plan:
