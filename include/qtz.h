@@ -50,6 +50,7 @@ typedef int32_t qtz_status;
 #define QTZ_ERR_CUDA (-6)           /* a CUDA runtime/driver call failed                    */
 #define QTZ_ERR_DEVICE_TIMEOUT (-7) /* a bounded device-side wait gave up                   */
 #define QTZ_ERR_NO_DEVICE (-8)      /* no usable CUDA device                                */
+#define QTZ_ERR_TOO_LARGE (-9)      /* size beyond the fixed capacity of a non-allocating call */
 
 typedef struct qtz_ctx* qtz_handle;     /* library-owned, opaque */
 typedef struct qtz_plan* qtz_conv_plan; /* library-owned: prepacked weights and tables */
@@ -118,6 +119,29 @@ QTZ_API qtz_status qtz_calibrate_minmax(qtz_handle h, const float* x_dev, int64_
  * [0,6] for a layer followed by ReLU6) before deriving parameters from it.                */
 QTZ_API qtz_status qtz_minmax(qtz_handle h, const float* x_dev, int64_t outer, int64_t axis_len,
                               int64_t inner, float* lo_host, float* hi_host, void* stream);
+
+/* The per-layer range reduction for callers that must not allocate device memory -- for
+ * instance a server that handed all of the GPU's memory to its own pool when it started, or a
+ * latency-critical loop that cannot afford the device-wide synchronisation cudaMalloc/cudaFree
+ * may bring.  (The paper has no counterpart to this call: it is a property of this library,
+ * not of the method.  What it computes is the min/max of Section 2.5, exactly as qtz_minmax.)
+ *   x_dev    `count` fp32 values on the CURRENT device (no handle is involved)
+ *   out_dev  3 x 4 bytes on the device, written by the call: float lo, float hi, and a 32-bit
+ *            word that is non-zero when a NaN or Inf was met (lo/hi are then unspecified)
+ * Asynchronous on `stream`; nothing is copied to the host.
+ * The block partials live in a fixed 48 KB array inside the library image, which every GPU that
+ * loads the library keeps until the process exits.  Consequences:
+ *   - count may not exceed qtz_minmax_static_max_count() (2^28 values); larger tensors are
+ *     refused with QTZ_ERR_TOO_LARGE and nothing is launched;
+ *   - all calls on a device share that array (it keeps the previous call's partials; none of
+ *     them is read before the current call has rewritten it, so nothing needs clearing), and
+ *     two calls whose kernels may overlap on the GPU -- different streams -- race on it: issue
+ *     them in order on one stream, or synchronise in between;
+ *   - the first call on each device looks the array's device address up
+ *     (cudaGetSymbolAddress); make that first call before starting any stream capture.
+ * The call performs no cudaMalloc / cudaFree and uses no allocating library routine.         */
+QTZ_API qtz_status qtz_minmax_static(const float* x_dev, int64_t count, float* out_dev, void* stream);
+QTZ_API int64_t qtz_minmax_static_max_count(void);
 
 /* Host-only: parameters from a known real range (same rules as above).                    */
 QTZ_API qtz_status qtz_params_from_range(float lo, float hi, int32_t bits, int32_t symmetric,

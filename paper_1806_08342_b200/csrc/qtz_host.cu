@@ -18,6 +18,7 @@ extern "C" const char* qtz_status_string(qtz_status s)
         case QTZ_ERR_CUDA: return "CUDA error";
         case QTZ_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
         case QTZ_ERR_NO_DEVICE: return "no usable CUDA device";
+        case QTZ_ERR_TOO_LARGE: return "size exceeds the fixed capacity of this non-allocating call";
         default: return "unknown status";
     }
 }

@@ -48,6 +48,8 @@ SIGNATURES = {
     "qtz_calibrate_minmax": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int32, c_void_p,
                                        c_void_p]),
     "qtz_minmax": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p]),
+    "qtz_minmax_static": (c_int32, [c_void_p, c_int64, c_void_p, c_void_p]),
+    "qtz_minmax_static_max_count": (c_int64, []),
     "qtz_params_from_range": (c_int32, [c_float, c_float, c_int32, c_int32, c_void_p]),
     "qtz_quantize_tensor": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int32, c_int32,
                                       c_void_p, c_void_p]),
@@ -144,6 +146,20 @@ def params_from_range(lo, hi, bits=8, symmetric=False):
     if rc:
         raise QtzError(rc, "qtz_params_from_range")
     return q[0]
+
+
+def minmax_static(x, out=None):
+    """qtz_minmax_static on the current device and stream.  `x`: fp32 CUDA tensor; returns a 3-word
+    CUDA tensor (lo, hi, non-finite flag bits viewed as float).  Allocates only if `out` is None --
+    pass a preallocated 3-element fp32 tensor to keep the call allocation-free."""
+    _check_dev(x, out)
+    assert x.dtype == torch.float32
+    if out is None:
+        out = torch.empty(3, dtype=torch.float32, device=x.device)
+    rc = load_library().qtz_minmax_static(_ptr(x), x.numel(), _ptr(out), _stream())
+    if rc:
+        raise QtzError(rc, "qtz_minmax_static", load_library().qtz_status_string(rc).decode())
+    return out
 
 
 class Handle:

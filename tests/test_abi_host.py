@@ -37,7 +37,7 @@ def test_every_declared_symbol_is_exported_and_bound(qtz):
 def test_status_strings(qtz):
     lib = qtz.load_library()
     assert lib.qtz_status_string(0) == b"ok"
-    for code in range(-8, 0):
+    for code in range(-9, 0):
         assert lib.qtz_status_string(code) not in (b"", b"unknown status")
 
 
