@@ -44,11 +44,12 @@ struct TcArgs {
     int32_t is4d;
     int32_t tw, th, tb, rows;               // pixel box of one tile and its row count (<= 128)
     int32_t tiles_w, tiles_h, n_tiles;
+    int32_t m_tiles, group_m;               // rasterisation: groups of group_m pixel tiles x all n tiles
     int64_t num_tiles;
     int32_t W, H, B;                        // output extent (2-D case: W = number of pixels)
     int32_t taps, kw, pad;
     int32_t kb_per_tap, c_pad;
-    int32_t BK, BN, N, out_box, stages;
+    int32_t BK, BN, N, out_box, out_bufs, stages;
     uint32_t idesc;
     const int32_t* bias;
     const int32_t* wsum;                    // [ncls][N]
@@ -68,7 +69,7 @@ struct SmemLayout {
     uint32_t a_stage, b_stage;
 };
 
-__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls)
+__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int out_bufs)
 {
     SmemLayout L;
     L.a_stage = kTileM * BK;
@@ -76,7 +77,7 @@ __host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, in
     L.a_off = 0;
     L.b_off = L.a_off + stages * L.a_stage;
     L.out_off = L.b_off + stages * L.b_stage;
-    L.corr_off = L.out_off + kTileM * BN;
+    L.corr_off = L.out_off + out_bufs * kTileM * out_box;
     L.mult_off = L.corr_off + ncls * BN * 4;
     L.rsh_off = L.mult_off + BN * 4;
     L.bar_off = L.rsh_off + BN * 4;
@@ -97,6 +98,19 @@ __device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t col, uint32_t box
     return off ^ (((off >> 7) & ((box >> 4) - 1)) << 4);
 }
 
+// Tile order: pixel tiles are taken in groups of group_m; inside a group the pixel tile varies
+// fastest, so the CTAs running at the same time share a band of A panels and a band of B panels
+// that together fit in L2.
+__device__ __forceinline__ void decode_tile(const TcArgs& a, int64_t tile, int64_t& m_tile, int& n_tile)
+{
+    const int64_t per_group = static_cast<int64_t>(a.group_m) * a.n_tiles;
+    const int64_t g = tile / per_group, r = tile - g * per_group;
+    const int64_t m_first = g * a.group_m;
+    const int gm = static_cast<int>(a.m_tiles - m_first < a.group_m ? a.m_tiles - m_first : a.group_m);
+    m_tile = m_first + r % gm;
+    n_tile = static_cast<int>(r / gm);
+}
+
 __global__ void __launch_bounds__(kThreadsTc, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_y, const TcArgs a)
@@ -104,7 +118,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
-    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls);
+    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.out_bufs);
 
     const uint32_t bar_full = base + L.bar_off;
     const uint32_t bar_empty = bar_full + 8 * kMaxStages;
@@ -149,8 +163,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t tx = static_cast<uint32_t>(a.rows * a.BK + a.BN * a.BK);
             bool ok = true;
             for (int64_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
-                const int n_tile = static_cast<int>(tile % a.n_tiles);
-                const int64_t m_tile = tile / a.n_tiles;
+                int n_tile;
+                int64_t m_tile;
+                decode_tile(a, tile, m_tile, n_tile);
                 int w0 = 0, h0 = 0, b0 = 0;
                 if (a.is4d) {
                     w0 = static_cast<int>(m_tile % a.tiles_w) * a.tw;
@@ -242,15 +257,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int boxes = a.BN / a.out_box;
         const uint32_t box_bytes = kTileM * a.out_box;
         int staged_n_tile = -1;
-        uint32_t local = 0;
-        for (int64_t tile = blockIdx.x; tile < a.num_tiles; tile += gridDim.x, ++local) {
+        uint32_t local = 0, stores = 0;
+        bool alive = true;
+        for (int64_t tile = blockIdx.x; alive && tile < a.num_tiles; tile += gridDim.x, ++local) {
             const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
-            const int n_tile = static_cast<int>(tile % a.n_tiles);
-            const int64_t m_tile = tile / a.n_tiles;
+            int n_tile;
+            int64_t m_tile;
+            decode_tile(a, tile, m_tile, n_tile);
             const int n0 = n_tile * a.BN;
 
-            // the previous tile's TMA stores must have finished reading the staging buffer
-            if (et == 0) tma_store_wait_read();
             if (n_tile != staged_n_tile) {
                 named_barrier(2, kEpiThreads);       // everyone is done with the old tables
                 for (int j = et; j < a.BN; j += kEpiThreads) {
@@ -265,8 +280,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     rsh_s[j] = (live && !a.raw) ? __ldg(a.rshift + n) : 40;
                 }
                 staged_n_tile = n_tile;
+                named_barrier(2, kEpiThreads);       // tables visible to all epilogue threads
             }
-            named_barrier(1, kEpiThreads);
 
             // which pixel this row is, its border class and its activation-sum term
             int w0 = 0, h0 = 0, b0 = 0, pw, ph = 0, pb = 0;
@@ -314,12 +329,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int32_t lo = a.act_min - a.zy, hi = a.act_max - a.zy;
             const uint32_t zy4 = 0x01010101u * static_cast<uint32_t>(a.zy);
 
-            for (int j0 = 0; j0 < a.BN; j0 += 32) {
-                uint32_t v[32];
-                tmem_ld_32x32(taddr + j0, v);
-                tmem_ld_wait();
-                if (n0 + j0 >= a.N) continue;        // a chunk entirely beyond the real channels
-                if (a.raw) {
+            if (a.raw) {
+                for (int j0 = 0; j0 < a.BN && n0 + j0 < a.N; j0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(taddr + j0, v);
+                    tmem_ld_wait();
                     if (row_live) {
                         const int64_t pix = a.is4d ? (static_cast<int64_t>(pb) * a.H + ph) * a.W + pw : pw;
                         int32_t* out = a.y_raw + pix * a.N + n0 + j0;
@@ -327,61 +341,76 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         for (int j = 0; j < 32; ++j)
                             if (n0 + j0 + j < a.N) out[j] = static_cast<int32_t>(v[j]) + corr_row[j0 + j] + rowterm;
                     }
-                    continue;
                 }
-                uint32_t packed[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const int4 c4 = *reinterpret_cast<const int4*>(corr_row + j0 + 4 * q);
-                    const int4 m4 = *reinterpret_cast<const int4*>(mult_s + j0 + 4 * q);
-                    const int4 r4 = *reinterpret_cast<const int4*>(rsh_s + j0 + 4 * q);
-                    const int32_t cc[4] = {c4.x, c4.y, c4.z, c4.w}, mm[4] = {m4.x, m4.y, m4.z, m4.w},
-                                  rr[4] = {r4.x, r4.y, r4.z, r4.w};
-                    uint32_t word = 0;
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int32_t full = static_cast<int32_t>(v[4 * q + e]) + cc[e] + rowterm;
-                        int32_t t;
-                        if (a.fast_requant) {
-                            // r >= 33: rounding constant 2^(r-1) sits in the high word; shift the high word only
-                            const int64_t prod = static_cast<int64_t>(full) * mm[e] +
-                                                 (static_cast<int64_t>(1u << (rr[e] - 33)) << 32);
-                            t = static_cast<int32_t>(prod >> 32) >> (rr[e] - 32);
-                            t = min(max(t, lo), hi);
-                        } else {
-                            const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(1) << (rr[e] - 1));
-                            const int64_t s = prod >> rr[e];
-                            t = static_cast<int32_t>(min(max(s, static_cast<int64_t>(lo)), static_cast<int64_t>(hi)));
-                        }
-                        word |= (static_cast<uint32_t>(t) & 0xffu) << (8 * e);
-                    }
-                    packed[q] = __vadd4(word, zy4);
-                }
-                const int box = j0 / a.out_box, col = j0 % a.out_box;
-                uint8_t* const dst = out_s + box * box_bytes;
-                *reinterpret_cast<uint4*>(dst + swz(row, col, a.out_box)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                *reinterpret_cast<uint4*>(dst + swz(row, col + 16, a.out_box)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+                continue;
             }
-            // accumulator drained: hand it back to the MMA warp
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
 
-            if (!a.raw) {
+            // uint8 output: one staging box (128 rows x out_box bytes) at a time, two boxes in flight
+            for (int bx = 0; bx < boxes; ++bx) {
+                const int nn = n0 + bx * a.out_box;
+                if (nn >= a.N) break;                // boxes entirely beyond the real channels
+                const uint32_t buf = stores % a.out_bufs;
+                if (et == 0) {                       // the store that last used this buffer has read it
+                    if (a.out_bufs == 2) tma_store_wait_read_1(); else tma_store_wait_read();
+                }
+                named_barrier(1, kEpiThreads);
+                uint8_t* const dst = out_s + buf * box_bytes;
+                for (int col = 0; col < a.out_box && nn + col < a.N; col += 32) {
+                    const int j0 = bx * a.out_box + col;
+                    uint32_t v[32];
+                    tmem_ld_32x32(taddr + j0, v);
+                    tmem_ld_wait();
+                    uint32_t packed[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const int4 c4 = *reinterpret_cast<const int4*>(corr_row + j0 + 4 * q);
+                        const int4 m4 = *reinterpret_cast<const int4*>(mult_s + j0 + 4 * q);
+                        const int4 r4 = *reinterpret_cast<const int4*>(rsh_s + j0 + 4 * q);
+                        const int32_t cc[4] = {c4.x, c4.y, c4.z, c4.w}, mm[4] = {m4.x, m4.y, m4.z, m4.w},
+                                      rr[4] = {r4.x, r4.y, r4.z, r4.w};
+                        uint32_t word = 0;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int32_t full = static_cast<int32_t>(v[4 * q + e]) + cc[e] + rowterm;
+                            int32_t t;
+                            if (a.fast_requant) {
+                                // r >= 33: the rounding constant 2^(r-1) sits in the high word; shift the high word only
+                                const int64_t prod = static_cast<int64_t>(full) * mm[e] +
+                                                     (static_cast<int64_t>(1u << (rr[e] - 33)) << 32);
+                                t = static_cast<int32_t>(prod >> 32) >> (rr[e] - 32);
+                                t = min(max(t, lo), hi);
+                            } else {
+                                const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(1) << (rr[e] - 1));
+                                const int64_t sh = prod >> rr[e];
+                                t = static_cast<int32_t>(min(max(sh, static_cast<int64_t>(lo)), static_cast<int64_t>(hi)));
+                            }
+                            word |= (static_cast<uint32_t>(t) & 0xffu) << (8 * e);
+                        }
+                        packed[q] = __vadd4(word, zy4);
+                    }
+                    *reinterpret_cast<uint4*>(dst + swz(row, col, a.out_box)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    *reinterpret_cast<uint4*>(dst + swz(row, col + 16, a.out_box)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                }
+                if (bx == boxes - 1 || nn + a.out_box >= a.N) {
+                    // accumulator drained: hand it back to the MMA warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+                }
                 fence_proxy_async_smem();
                 named_barrier(1, kEpiThreads);
                 if (et == 0) {
-                    for (int bx = 0; bx < boxes; ++bx) {
-                        const int nn = n0 + bx * a.out_box;
-                        if (nn >= a.N) break;
-                        const uint32_t src = base + L.out_off + bx * box_bytes;
-                        if (a.is4d)
-                            tma_store_4d(&map_y, src, nn, w0, h0, b0);
-                        else
-                            tma_store_2d(&map_y, src, nn, w0);
-                    }
+                    const uint32_t src = base + L.out_off + buf * box_bytes;
+                    if (a.is4d)
+                        tma_store_4d(&map_y, src, nn, w0, h0, b0);
+                    else
+                        tma_store_2d(&map_y, src, nn, w0);
                     tma_store_commit();
                 }
+                ++stores;
             }
         }
         if (et == 0) tma_store_wait_all();
@@ -651,11 +680,21 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
         a.kvalid[cls] = rows_valid * cols_valid * d.c;
     }
 
+    a.m_tiles = static_cast<int32_t>(a.num_tiles / a.n_tiles);
+    a.group_m = std::max(1, std::min(a.m_tiles, 16));
+    a.out_bufs = 2;
     // shared-memory budget -> pipeline depth
-    for (a.stages = kMaxStages; a.stages >= 2; --a.stages)
-        if (make_layout(a.BK, a.BN, a.stages, a.ncls).total <= static_cast<uint32_t>(kSmemBudget)) break;
+    auto max_stages = [&](int bufs) {
+        int st = kMaxStages;
+        for (; st >= 2; --st)
+            if (make_layout(a.BK, a.BN, st, a.ncls, a.out_box, bufs).total <= static_cast<uint32_t>(kSmemBudget)) break;
+        return st;
+    };
+    // a deeper operand ring beats a second output staging box
+    a.out_bufs = max_stages(1) > max_stages(2) ? 1 : 2;
+    a.stages = max_stages(a.out_bufs);
     if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
-    t->smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls).total + 1024;
+    t->smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.out_bufs).total + 1024;
 
     // instruction descriptor: s32 accumulate, A = u8, B = s8, both K-major, N and M of the tile
     a.idesc = (2u << 4) | (0u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) |
