@@ -251,6 +251,9 @@ def run_ours(args, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     peaks = load_peaks()
     hq = qtz.Handle(local_rank)
+    if args.hbm_only:
+        print(json.dumps({"hbm_kernels": time_hbm_kernels(hq, qtz, torch, peaks)}), flush=True)
+        return
     cases = [GemmCase(hq, qtz, torch, s) for s in SIZES]
     torch.cuda.synchronize()
 
@@ -355,6 +358,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the HBM-kernel table and the CPU baseline")
+    ap.add_argument("--hbm-only", action="store_true",
+                    help="run only the element-wise / depthwise kernel table (profiling runs); prints it as JSON")
     ap.add_argument("--sizes", default="", help="comma-separated subset of the sweep (profiling runs); default: all")
     args = ap.parse_args()
     if args.sizes:

@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libqtz.so")
-SOURCES = ["qtz_host.cu", "qtz_elementwise.cu", "qtz_glue.cu", "qtz_conv_direct.cu", "qtz_conv_tc.cu",
+SOURCES = ["qtz_host.cu", "qtz_elementwise.cu", "qtz_glue.cu", "qtz_conv_direct.cu", "qtz_depthwise.cu", "qtz_conv_tc.cu",
            "qtz_plan.cu", "qtz_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--fmad=false",

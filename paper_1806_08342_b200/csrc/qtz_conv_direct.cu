@@ -1,13 +1,10 @@
-// CUDA-core convolution kernels of libqtz.
+// CUDA-core convolution kernel of libqtz for geometries the other paths do not take.
 //
 //  * direct_conv_kernel: any kh x kw / stride / pad / channel count.  It serves the layers
 //    the tensor-core path does not take (3-channel stem convolutions, odd geometries).  The
 //    zero-point terms follow the expansion of Eq. 5-6: the raw u8 x s8 dot products are
 //    corrected by -z_x sum(w) - z_w sum(x) + K z_x z_w per output.  Out-of-image taps are
 //    staged as the code z_x (real zero, Section 2.1), so every output sees all K taps.
-//  * depthwise3x3_kernel: 3x3 depthwise, stride 1 or 2, pad 1 (the separable blocks of
-//    Section 3.1.3's MobileNets).  Not a dense contraction: each thread keeps 4 channels of a
-//    short row of outputs in registers and slides a 3x3 window over coalesced 32-bit loads.
 #include <algorithm>
 
 #include "qtz_plan.cuh"
@@ -148,106 +145,6 @@ direct_conv_kernel(const DirectArgs a)
     }
 }
 
-// ----------------------------------------------------------------------------------------
-struct DwArgs {
-    const uint8_t* x;
-    const int16_t* w;  // [9][pitch] codes minus zero point
-    const int32_t* bias;
-    const int32_t* mult;
-    const int32_t* rshift;
-    uint8_t* y;
-    int batch, h, w_, c, xp, yp, oh, ow, strips;
-    int zx, zy, act_min, act_max;
-};
-
-constexpr int kDwThreads = 256, kStrip = 4;
-
-template <int kStride>
-__global__ void __launch_bounds__(kDwThreads)
-depthwise3x3_kernel(const DwArgs a)
-{
-    const int groups = (a.c + 3) >> 2;
-    const int64_t t = static_cast<int64_t>(blockIdx.x) * kDwThreads + threadIdx.x;
-    const int64_t total = static_cast<int64_t>(a.batch) * a.oh * a.strips * groups;
-    if (t >= total) return;
-    const int g = static_cast<int>(t % groups);
-    int64_t q = t / groups;
-    const int strip = static_cast<int>(q % a.strips); q /= a.strips;
-    const int oh = static_cast<int>(q % a.oh);
-    const int b = static_cast<int>(q / a.oh);
-    const int ow0 = strip * kStrip, c0 = 4 * g;
-
-    int32_t wd[9][4];
-#pragma unroll
-    for (int tap = 0; tap < 9; ++tap) {
-        const uint2 v = __ldg(reinterpret_cast<const uint2*>(a.w + static_cast<int64_t>(tap) * a.xp + c0));
-        wd[tap][0] = static_cast<int16_t>(v.x & 0xffff); wd[tap][1] = static_cast<int32_t>(v.x) >> 16;
-        wd[tap][2] = static_cast<int16_t>(v.y & 0xffff); wd[tap][3] = static_cast<int32_t>(v.y) >> 16;
-    }
-    int32_t base[4];
-#pragma unroll
-    for (int ch = 0; ch < 4; ++ch) {
-        int32_t s = 0;
-#pragma unroll
-        for (int tap = 0; tap < 9; ++tap) s += wd[tap][ch];
-        const int cc = min(c0 + ch, a.c - 1);
-        base[ch] = __ldg(a.bias + cc) - a.zx * s;  // out-of-image taps hold z_x, so all 9 taps count
-    }
-    int32_t acc[kStrip][4];
-#pragma unroll
-    for (int s = 0; s < kStrip; ++s)
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch) acc[s][ch] = base[ch];
-
-    constexpr int kCols = (kStrip - 1) * kStride + 3;
-    const uint32_t fill = 0x01010101u * static_cast<uint32_t>(a.zx);
-    const int iw0 = ow0 * kStride - 1;
-#pragma unroll
-    for (int i = 0; i < 3; ++i) {
-        const int ih = oh * kStride - 1 + i;
-        const bool row_ok = ih >= 0 && ih < a.h;
-        const uint8_t* row = a.x + ((static_cast<int64_t>(b) * a.h + (row_ok ? ih : 0)) * a.w_) * a.xp + c0;
-        uint32_t col[kCols];
-#pragma unroll
-        for (int j = 0; j < kCols; ++j) {
-            const int iw = iw0 + j;
-            col[j] = (row_ok && iw >= 0 && iw < a.w_) ? __ldg(reinterpret_cast<const uint32_t*>(row + static_cast<int64_t>(iw) * a.xp)) : fill;
-        }
-#pragma unroll
-        for (int j = 0; j < kCols; ++j) {
-            const int32_t x0 = col[j] & 0xff, x1 = (col[j] >> 8) & 0xff, x2 = (col[j] >> 16) & 0xff, x3 = col[j] >> 24;
-#pragma unroll
-            for (int s = 0; s < kStrip; ++s) {
-                const int tapj = j - s * kStride;
-                if (tapj >= 0 && tapj < 3) {
-                    acc[s][0] += x0 * wd[3 * i + tapj][0];
-                    acc[s][1] += x1 * wd[3 * i + tapj][1];
-                    acc[s][2] += x2 * wd[3 * i + tapj][2];
-                    acc[s][3] += x3 * wd[3 * i + tapj][3];
-                }
-            }
-        }
-    }
-    int32_t m[4], r[4];
-#pragma unroll
-    for (int ch = 0; ch < 4; ++ch) {
-        const int cc = min(c0 + ch, a.c - 1);
-        m[ch] = __ldg(a.mult + cc);
-        r[ch] = __ldg(a.rshift + cc);
-    }
-    uint8_t* out = a.y + ((static_cast<int64_t>(b) * a.oh + oh) * a.ow) * a.yp + c0;
-#pragma unroll
-    for (int s = 0; s < kStrip; ++s) {
-        const int ow = ow0 + s;
-        if (ow >= a.ow) break;
-        uint32_t word = 0;
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch)
-            word |= requant_u8(acc[s][ch], m[ch], r[ch], a.zy, a.act_min, a.act_max) << (8 * ch);
-        *reinterpret_cast<uint32_t*>(out + static_cast<int64_t>(ow) * a.yp) = word;
-    }
-}
-
 }  // namespace
 
 qtz_status qtz_direct_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, int32_t y_zp, int32_t act_min,
@@ -268,28 +165,6 @@ qtz_status qtz_direct_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* 
     if (p->ev_start) QTZ_CUDA(p->h, cudaEventRecord(p->ev_start, st));
     direct_conv_kernel<<<grid, kDirectThreads, 0, st>>>(a);
     QTZ_LAUNCH_CHECK(p->h, "direct_conv_kernel");
-    if (p->ev_stop) QTZ_CUDA(p->h, cudaEventRecord(p->ev_stop, st));
-    return QTZ_OK;
-}
-
-qtz_status qtz_depthwise_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, uint8_t* y, int32_t y_zp, int32_t act_min,
-                                int32_t act_max, cudaStream_t st)
-{
-    const qtz_conv_desc& d = p->d;
-    DwArgs a{};
-    a.x = x; a.w = p->w_depthwise; a.bias = p->bias; a.mult = p->mult; a.rshift = p->rshift; a.y = y;
-    a.batch = d.batch; a.h = d.h; a.w_ = d.w; a.c = d.c; a.xp = d.c_pitch_in; a.yp = d.c_pitch_out;
-    a.oh = p->oh; a.ow = p->ow; a.strips = (p->ow + kStrip - 1) / kStrip;
-    a.zx = x_zp; a.zy = y_zp; a.act_min = act_min; a.act_max = act_max;
-    const int64_t total = static_cast<int64_t>(d.batch) * p->oh * a.strips * ((d.c + 3) / 4);
-    const int64_t blocks = (total + kDwThreads - 1) / kDwThreads;
-    if (blocks > 0x7fffffff) return QTZ_ERR_UNSUPPORTED;
-    if (p->ev_start) QTZ_CUDA(p->h, cudaEventRecord(p->ev_start, st));
-    if (d.stride == 1)
-        depthwise3x3_kernel<1><<<static_cast<unsigned>(blocks), kDwThreads, 0, st>>>(a);
-    else
-        depthwise3x3_kernel<2><<<static_cast<unsigned>(blocks), kDwThreads, 0, st>>>(a);
-    QTZ_LAUNCH_CHECK(p->h, "depthwise3x3_kernel");
     if (p->ev_stop) QTZ_CUDA(p->h, cudaEventRecord(p->ev_stop, st));
     return QTZ_OK;
 }

@@ -565,12 +565,27 @@ EncodeTiledFn encode_fn()
 
 CUtensorMapSwizzle swizzle_for(int bytes)
 {
-    return bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+    switch (bytes) {
+        case 128: return CU_TENSOR_MAP_SWIZZLE_128B;
+        case 64: return CU_TENSOR_MAP_SWIZZLE_64B;
+        case 32: return CU_TENSOR_MAP_SWIZZLE_32B;
+        default: return CU_TENSOR_MAP_SWIZZLE_NONE;
+    }
 }
 
-// rank-2 or rank-4 uint8 tensor map; dims[0] is the contiguous dimension.
 bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                 const uint32_t* box, int swizzle_bytes)
+{
+    return qtz_encode_u8_map(m, base, rank, dims, strides_bytes, box, swizzle_bytes);
+}
+
+bool is_pointwise(const qtz_conv_desc& d) { return d.kh == 1 && d.kw == 1 && d.pad == 0; }
+bool is_3x3(const qtz_conv_desc& d) { return d.kh == 3 && d.kw == 3 && d.pad == 1 && d.stride == 1; }
+
+}  // namespace
+
+bool qtz_encode_u8_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                       const uint32_t* box, int swizzle_bytes)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
@@ -586,11 +601,6 @@ bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims
               CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(swizzle_bytes), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-
-bool is_pointwise(const qtz_conv_desc& d) { return d.kh == 1 && d.kw == 1 && d.pad == 0; }
-bool is_3x3(const qtz_conv_desc& d) { return d.kh == 3 && d.kw == 3 && d.pad == 1 && d.stride == 1; }
-
-}  // namespace
 
 bool qtz_tc_supported(const qtz_conv_desc& d)
 {

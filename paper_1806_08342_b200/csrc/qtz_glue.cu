@@ -13,35 +13,60 @@ struct AddRule {
     int32_t a_zp, a_mult, b_zp, b_mult, rshift, y_zp, act_min, act_max;
 };
 
-__device__ __forceinline__ uint32_t add1(uint32_t a, uint32_t b, const AddRule& r, int64_t bias)
+// d = (c << 16) | (sat_u8(a) << 8) | sat_u8(b)
+__device__ __forceinline__ uint32_t pack_sat_u8(int32_t a, int32_t b, uint32_t c)
 {
-    const int64_t v = static_cast<int64_t>(static_cast<int32_t>(a) - r.a_zp) * r.a_mult +
-                      static_cast<int64_t>(static_cast<int32_t>(b) - r.b_zp) * r.b_mult + bias;
-    const int64_t y = v >> r.rshift;
-    return static_cast<uint32_t>(min(max(y, static_cast<int64_t>(r.act_min)), static_cast<int64_t>(r.act_max)));
+    uint32_t d;
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
 }
 
-__device__ __forceinline__ uint32_t add4(uint32_t a, uint32_t b, const AddRule& r, int64_t bias)
+// (a m_a + b m_b + addend) >> r for one byte lane, relative to act_min and clamped to
+// [0, act_max - act_min]; the zero points, the rounding constant and (z_y - act_min) 2^r are all
+// inside `addend`.  |a m| < 2^39, so the shifted value fits 32 bits whenever r >= 10; smaller
+// shifts take the 64-bit route.
+template <int kShiftKind>  // 0: r >= 32, 1: 10 <= r < 32, 2: r < 10
+__device__ __forceinline__ int32_t add1(uint32_t a, uint32_t b, const AddRule& r, int64_t addend, int32_t span)
 {
-    return add1(a & 0xff, b & 0xff, r, bias) | (add1((a >> 8) & 0xff, (b >> 8) & 0xff, r, bias) << 8) |
-           (add1((a >> 16) & 0xff, (b >> 16) & 0xff, r, bias) << 16) | (add1(a >> 24, b >> 24, r, bias) << 24);
+    const int64_t v = static_cast<int64_t>(static_cast<uint64_t>(a) * static_cast<uint32_t>(r.a_mult)) +
+                      static_cast<int64_t>(static_cast<uint64_t>(b) * static_cast<uint32_t>(r.b_mult)) + addend;
+    if (kShiftKind == 0) return __vimin_s32_relu(static_cast<int32_t>(v >> 32) >> (r.rshift - 32), span);
+    if (kShiftKind == 1)
+        return __vimin_s32_relu(static_cast<int32_t>(__funnelshift_r(static_cast<uint32_t>(v), static_cast<uint32_t>(v >> 32), r.rshift)), span);
+    const int64_t s = v >> r.rshift;
+    return static_cast<int32_t>(min(max(s, static_cast<int64_t>(0)), static_cast<int64_t>(span)));
 }
 
-// y = clamp(z_y + ((a' m_a + b' m_b + 2^(r-1)) >> r)); the rounding constant and z_y 2^r are
-// folded into one 64-bit addend (|a' m| < 2^39 and r <= 62 - 9 keep the sum inside int64).
+template <int kShiftKind>
+__device__ __forceinline__ uint32_t add4(uint32_t a, uint32_t b, const AddRule& r, int64_t addend, int32_t span, uint32_t lo4)
+{
+    const int32_t y0 = add1<kShiftKind>(a & 0xff, b & 0xff, r, addend, span);
+    const int32_t y1 = add1<kShiftKind>((a >> 8) & 0xff, (b >> 8) & 0xff, r, addend, span);
+    const int32_t y2 = add1<kShiftKind>((a >> 16) & 0xff, (b >> 16) & 0xff, r, addend, span);
+    const int32_t y3 = add1<kShiftKind>(a >> 24, b >> 24, r, addend, span);
+    return pack_sat_u8(y1, y0, pack_sat_u8(y3, y2, 0u)) + lo4;
+}
+
+// y = clamp(z_y + (((a - z_a) m_a + (b - z_b) m_b + 2^(r-1)) >> r)).  All constants fold into one
+// 64-bit addend: 2^(r-1) + (z_y - act_min) 2^r - z_a m_a - z_b m_b (|.| < 2^62 for r <= 53).
+template <int kShiftKind>
 __global__ void __launch_bounds__(kThreads)
 add_u8_kernel(const uint8_t* __restrict__ a, const uint8_t* __restrict__ b, int64_t bytes, AddRule r,
               uint8_t* __restrict__ y)
 {
-    const int64_t bias = (static_cast<int64_t>(1) << (r.rshift - 1)) + (static_cast<int64_t>(r.y_zp) << r.rshift);
+    const int64_t addend = (static_cast<int64_t>(1) << (r.rshift - 1)) +
+                           static_cast<int64_t>(r.y_zp - r.act_min) * (static_cast<int64_t>(1) << r.rshift) -
+                           static_cast<int64_t>(r.a_zp) * r.a_mult - static_cast<int64_t>(r.b_zp) * r.b_mult;
+    const uint32_t lo4 = 0x01010101u * static_cast<uint32_t>(r.act_min);
+    const int32_t span = r.act_max - r.act_min;
     const int64_t groups = bytes >> 4;
     const int64_t g = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
     if (g >= groups) return;
     const uint4 va = __ldcs(reinterpret_cast<const uint4*>(a) + g);
     const uint4 vb = __ldcs(reinterpret_cast<const uint4*>(b) + g);
     uint4 o;
-    o.x = add4(va.x, vb.x, r, bias); o.y = add4(va.y, vb.y, r, bias);
-    o.z = add4(va.z, vb.z, r, bias); o.w = add4(va.w, vb.w, r, bias);
+    o.x = add4<kShiftKind>(va.x, vb.x, r, addend, span, lo4); o.y = add4<kShiftKind>(va.y, vb.y, r, addend, span, lo4);
+    o.z = add4<kShiftKind>(va.z, vb.z, r, addend, span, lo4); o.w = add4<kShiftKind>(va.w, vb.w, r, addend, span, lo4);
     reinterpret_cast<uint4*>(y)[g] = o;
 }
 
@@ -114,8 +139,14 @@ extern "C" qtz_status qtz_add_u8(qtz_handle h, const uint8_t* a_dev, int32_t a_z
     if ((c_pitch & 15) || !qtz_aligned16(a_dev) || !qtz_aligned16(b_dev) || !qtz_aligned16(y_dev)) return QTZ_ERR_MISALIGNED;
     const int64_t bytes = pixels * c_pitch;
     const AddRule r{a_zp, a_mult, b_zp, b_mult, rshift, y_zp, act_min, act_max};
-    add_u8_kernel<<<static_cast<unsigned>(ceil_div(bytes >> 4, kThreads)), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        a_dev, b_dev, bytes, r, y_dev);
+    const unsigned blocks = static_cast<unsigned>(ceil_div(bytes >> 4, kThreads));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (rshift >= 32)
+        add_u8_kernel<0><<<blocks, kThreads, 0, st>>>(a_dev, b_dev, bytes, r, y_dev);
+    else if (rshift >= 10)
+        add_u8_kernel<1><<<blocks, kThreads, 0, st>>>(a_dev, b_dev, bytes, r, y_dev);
+    else
+        add_u8_kernel<2><<<blocks, kThreads, 0, st>>>(a_dev, b_dev, bytes, r, y_dev);
     QTZ_LAUNCH_CHECK(h, "add_u8_kernel");
     return QTZ_OK;
 }

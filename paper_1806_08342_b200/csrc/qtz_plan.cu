@@ -49,15 +49,25 @@ weight_sum_kernel(const int8_t* __restrict__ w, int k_padded, int32_t* __restric
     }
 }
 
-// Depthwise weights [taps][c] -> int16 [taps][pitch] holding (code - z_w), zero padded.
+// Depthwise weights [3][3][c] -> per filter row and channel one word (k0, k1, k2, 0) of int8 codes,
+// plus the sum of the nine codes; channels beyond c are zero.
 __global__ void __launch_bounds__(kThreads)
-prepack_depthwise_kernel(const void* __restrict__ w, int wkind, int taps, int c, int pitch, int zw_signed,
-                         int16_t* __restrict__ out)
+prepack_depthwise_kernel(const void* __restrict__ w, int wkind, int c, int pitch, uint32_t* __restrict__ taps,
+                         int32_t* __restrict__ wsum)
 {
-    const int i = blockIdx.x * kThreads + threadIdx.x;
-    if (i >= taps * pitch) return;
-    const int tap = i / pitch, ch = i - tap * pitch;
-    out[i] = ch < c ? static_cast<int16_t>(load_code_s8(w, wkind, tap, ch, c) - zw_signed) : 0;
+    const int ch = blockIdx.x * kThreads + threadIdx.x;
+    if (ch >= pitch) return;
+    int32_t total = 0;
+    for (int i = 0; i < 3; ++i) {
+        uint32_t word = 0;
+        for (int j = 0; j < 3; ++j) {
+            const int32_t code = ch < c ? load_code_s8(w, wkind, 3 * i + j, ch, c) : 0;
+            word |= (static_cast<uint32_t>(code) & 0xffu) << (8 * j);
+            total += code;
+        }
+        taps[i * pitch + ch] = word;
+    }
+    wsum[ch] = total;
 }
 
 __global__ void fill_i32_kernel(int32_t* p, int n, int32_t v)
@@ -98,8 +108,10 @@ extern "C" qtz_status qtz_conv_destroy(qtz_conv_plan p)
     cudaSetDevice(p->device);
     cudaDeviceSynchronize();
     qtz_tc_release(p);
+    qtz_depthwise_release(p);
     cudaFree(p->w_direct);
-    cudaFree(p->w_depthwise);
+    cudaFree(p->dw_taps);
+    cudaFree(p->dw_wsum);
     cudaFree(p->bias);
     cudaFree(p->wsum);
     cudaFree(p->mult);
@@ -156,7 +168,10 @@ extern "C" qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, i
     p->k_total = depthwise ? d.kh * d.kw : d.kh * d.kw * d.c;
     p->w_zp_signed = d.wkind == QTZ_W_U8_PER_LAYER_ASYM ? *w_zero_point_host - 128 : 0;
     if (!raw)
-        for (int i = 0; i < d.n; ++i) p->rshift_min = std::min(p->rshift_min, rshift_host[i]);
+        for (int i = 0; i < d.n; ++i) {
+            p->rshift_min = std::min(p->rshift_min, rshift_host[i]);
+            p->rshift_max = std::max(p->rshift_max, rshift_host[i]);
+        }
 
 #define PLAN_CUDA(expr)                                        \
     do {                                                       \
@@ -169,25 +184,33 @@ extern "C" qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, i
     } while (0)
 
     const size_t nb = sizeof(int32_t) * static_cast<size_t>(d.n);
-    PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->bias), nb));
-    if (bias_q_dev)
-        PLAN_CUDA(cudaMemcpyAsync(p->bias, bias_q_dev, nb, cudaMemcpyDeviceToDevice, st));
-    else
-        PLAN_CUDA(cudaMemsetAsync(p->bias, 0, nb, st));
+    const int n_alloc = d.n + 16;  // room for whole 16-byte channel groups past the last channel
+    const size_t nb_alloc = sizeof(int32_t) * static_cast<size_t>(n_alloc);
+    PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->bias), nb_alloc));
+    PLAN_CUDA(cudaMemsetAsync(p->bias, 0, nb_alloc, st));
+    if (bias_q_dev) PLAN_CUDA(cudaMemcpyAsync(p->bias, bias_q_dev, nb, cudaMemcpyDeviceToDevice, st));
     if (!raw) {
-        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->mult), nb));
-        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->rshift), nb));
+        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->mult), nb_alloc));
+        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->rshift), nb_alloc));
+        PLAN_CUDA(cudaMemsetAsync(p->mult, 0, nb_alloc, st));
+        fill_i32_kernel<<<(n_alloc + 255) / 256, 256, 0, st>>>(p->rshift, n_alloc, 40);
+        PLAN_CUDA(cudaGetLastError());
         PLAN_CUDA(cudaMemcpyAsync(p->mult, mult_host, nb, cudaMemcpyHostToDevice, st));
         PLAN_CUDA(cudaMemcpyAsync(p->rshift, rshift_host, nb, cudaMemcpyHostToDevice, st));
     }
 
     if (depthwise) {
         p->family = QTZ_K_DEPTHWISE;
-        const int taps = d.kh * d.kw;
-        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->w_depthwise), sizeof(int16_t) * taps * d.c_pitch_in));
-        prepack_depthwise_kernel<<<(taps * d.c_pitch_in + kThreads - 1) / kThreads, kThreads, 0, st>>>(
-            w_q_dev, d.wkind, taps, d.c, d.c_pitch_in, p->w_zp_signed, p->w_depthwise);
+        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->dw_taps), sizeof(uint32_t) * 3 * d.c_pitch_in));
+        PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->dw_wsum), sizeof(int32_t) * d.c_pitch_in));
+        prepack_depthwise_kernel<<<(d.c_pitch_in + kThreads - 1) / kThreads, kThreads, 0, st>>>(
+            w_q_dev, d.wkind, d.c, d.c_pitch_in, p->dw_taps, p->dw_wsum);
         PLAN_CUDA(cudaGetLastError());
+        s = qtz_depthwise_prepare(p);
+        if (s != QTZ_OK) {
+            qtz_conv_destroy(p);
+            return s;
+        }
     } else if (qtz_tc_supported(d)) {
         p->family = QTZ_K_TCGEN05;
         s = qtz_tc_prepare(p, w_q_dev, st);
