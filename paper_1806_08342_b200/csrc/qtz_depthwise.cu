@@ -36,6 +36,7 @@ constexpr int kDwSmemLimit = 200 * 1024;
 
 struct DwArgs {
     uint8_t* y;
+    int32_t* y_raw;         // when set: int32 accumulators [pixel][c] instead of uint8 codes
     const uint32_t* taps;   // [3][tap_pitch]: per filter row and channel, bytes (k0, k1, k2, 0) as int8
     const int32_t* wsum;    // [tap_pitch]: sum of the nine int8 codes
     const int32_t* bias;    // padded beyond c
@@ -245,8 +246,8 @@ depthwise3x3_kernel(const __grid_constant__ CUtensorMap map_x, const DwArgs a)
             }
 #pragma unroll
             for (int ch = 0; ch < 8; ++ch) {
-                const int32_t r = __ldg(a.rshift + c0 + ch);
-                rq.m[ch] = __ldg(a.mult + c0 + ch);
+                const int32_t r = a.y_raw ? 40 : __ldg(a.rshift + c0 + ch);   // raw output has no multipliers
+                rq.m[ch] = a.y_raw ? 0 : __ldg(a.mult + c0 + ch);
                 rq.sh[ch] = kFast ? r - 32 : r;
                 rq.addhi[ch] = kFast ? (2 * (a.zy - a.act_min) + 1) * (1 << (r - 33)) : 0;
                 base[ch] = __ldg(a.bias + c0 + ch) - a.zx * __ldg(a.wsum + c0 + ch) + 9 * a.zx * a.zw;
@@ -293,12 +294,24 @@ depthwise3x3_kernel(const __grid_constant__ CUtensorMap map_x, const DwArgs a)
             const int r_end = min(min(a.th, r_begin + a.rps), a.oh - t.h0);   // tile-local output rows of this thread
             const uint8_t* cell = tile_s + (r_begin * kStride * a.twin + 2 * pr * kStride) * a.cb + 8 * g;
             const int row_bytes = a.twin * a.cb;
-            uint8_t* out = a.y + ((static_cast<int64_t>(t.b) * a.oh + t.h0 + r_begin) * a.ow + ow0) * a.yp + c0;
+            const int64_t first_px = (static_cast<int64_t>(t.b) * a.oh + t.h0 + r_begin) * a.ow + ow0;
+            uint8_t* out = a.y + first_px * a.yp + c0;
+            int32_t* out_raw = a.y_raw + first_px * a.c + c0;
             const int64_t out_row = static_cast<int64_t>(a.ow) * a.yp;
             const bool second = ow0 + 1 < a.ow;
 
             auto finish = [&](int32_t (&acc)[2][8], int32_t (&xs)[2][8]) {
                 int32_t v[8];
+                if (a.y_raw) {   // calibration: the accumulators themselves
+#pragma unroll
+                    for (int j = 0; j < 2; ++j)
+#pragma unroll
+                        for (int ch = 0; ch < 8; ++ch)
+                            if ((j == 0 || second) && c0 + ch < a.c)
+                                out_raw[j * a.c + ch] = acc[j][ch] - (kAsym ? a.zw * xs[j][ch] : 0);
+                    out_raw += static_cast<int64_t>(a.ow) * a.c;
+                    return;
+                }
 #pragma unroll
                 for (int ch = 0; ch < 8; ++ch) v[ch] = acc[0][ch] - (kAsym ? a.zw * xs[0][ch] : 0);
                 *reinterpret_cast<uint2*>(out) = requant_pixel<kFast>(v, rq);
@@ -450,7 +463,9 @@ qtz_status qtz_depthwise_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, uin
 {
     const qtz_conv_desc& d = p->d;
     DwArgs a = p->dw->args;
-    a.y = y;
+    const bool raw = d.outkind == QTZ_OUT_S32_RAW;
+    a.y = raw ? nullptr : y;
+    a.y_raw = raw ? reinterpret_cast<int32_t*>(y) : nullptr;
     a.zx = x_zp; a.zy = y_zp; a.act_min = act_min; a.act_max = act_max;
     CUtensorMap map;
     const uint64_t pitch = static_cast<uint64_t>(d.c_pitch_in);
@@ -462,7 +477,7 @@ qtz_status qtz_depthwise_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, uin
         p->h->last_error = "cuTensorMapEncodeTiled failed for the depthwise input";
         return QTZ_ERR_CUDA;
     }
-    const bool fast = p->rshift_min >= 33 && p->rshift_max <= 53;
+    const bool fast = !raw && p->rshift_min >= 33 && p->rshift_max <= 53;
     const bool asym = p->w_zp_signed != 0;
     if (p->ev_start) QTZ_CUDA(p->h, cudaEventRecord(p->ev_start, st));
     const unsigned blocks = static_cast<unsigned>(p->dw->grid);

@@ -94,7 +94,7 @@ qtz_status validate_desc(const qtz_conv_desc& d, int depthwise)
     if (k > 32768) return QTZ_ERR_OVERFLOW;
     if (depthwise) {
         if (d.n != d.c) return QTZ_ERR_INVALID_ARG;
-        if (d.kh != 3 || d.kw != 3 || d.pad != 1 || (d.stride != 1 && d.stride != 2) || d.outkind != QTZ_OUT_U8)
+        if (d.kh != 3 || d.kw != 3 || d.pad != 1 || (d.stride != 1 && d.stride != 2))
             return QTZ_ERR_UNSUPPORTED;
     }
     return QTZ_OK;

@@ -1,0 +1,177 @@
+"""Whole-network integer inference through libqtz (MobileNet-v1/v2, ResNet-50 shapes).
+
+Every numerical step is a call into the C ABI (`qtz.py`): batch-norm folding, weight and
+activation calibration, quantization, the convolutions, the residual adds and the pooling all run
+in the library's CUDA kernels.  This module only sequences the calls and keeps the tensors.
+
+`QuantizedNetwork.build()` performs post-training quantization on a calibration batch (Section
+3.1.2 of the paper: ranges of activations from calibration data, per-channel weight quantizers);
+`QuantizedNetwork.forward()` is the integer-only inference pass that the benchmark times.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import qtz, synth
+
+
+def _rup16(v):
+    return (v + 15) // 16 * 16
+
+
+class _Layer:
+    __slots__ = ("op", "plan", "args", "out_shape", "out_c", "out_params")
+
+
+class QuantizedNetwork:
+    def __init__(self, handle: qtz.Handle, ops, seed: int, wbits: int = 8):
+        self.h, self.ops, self.seed, self.wbits = handle, ops, seed, wbits
+        self.layers = []
+        self.params = {}            # tensor name -> qparams record (numpy void) after build()
+        self.batch = None
+
+    # ---- weights ---------------------------------------------------------------------------
+    def _prepare_weights(self, op, index, x_scale):
+        """Folds, calibrates and quantizes the weights of one conv / fc op on the device.
+        Returns (w_q tensor in API layout, per-channel params, int32 bias tensor, wkind)."""
+        h = self.h
+        p = synth.layer_params(op, index, self.seed)
+        depthwise = op["op"] == "conv" and op["depthwise"]
+        w = torch.from_numpy(p["w"]).cuda()
+        if "bn" in p:
+            bn = {k: torch.from_numpy(v).cuda() for k, v in p["bn"].items()}
+            rows = w.permute(2, 0, 1).contiguous() if depthwise else w          # one row per output channel
+            rows, bias = h.fold_batchnorm(rows, None, bn["gamma"], bn["beta"], bn["mean"], bn["var"], 1e-3)
+            w = rows.permute(1, 2, 0).contiguous() if depthwise else rows
+        else:
+            bias = torch.from_numpy(p["bias"]).cuda()
+        axis = 2 if depthwise else 0
+        wp = h.calibrate_minmax(w, axis=axis, bits=self.wbits, symmetric=True)
+        if self.wbits == 8:
+            w_q = h.quantize_tensor(w, wp, axis=axis, out_dtype=qtz.S8, restrict_range=True)
+            wkind = qtz.W_S8_PER_CHANNEL_SYM
+        else:
+            # packed 4-bit: along k of each output channel (dense) or along the channels of each tap (depthwise)
+            flat = w.reshape(9, -1) if depthwise else w.reshape(w.shape[0], -1)
+            w_q = h.quantize_tensor(flat, wp, axis=1 if depthwise else 0, out_dtype=qtz.S4_PACKED)
+            wkind = qtz.W_S4_PACKED_PER_CHANNEL_SYM
+        bias_q = h.quantize_bias(bias, x_scale, wp)
+        return w_q, wp, bias_q, wkind
+
+    # ---- calibration + plan creation -------------------------------------------------------
+    def build(self, images_u8: np.ndarray, calib: int):
+        """images_u8: [B,H,W,3].  Calibrates on images[:calib], creates plans for batch B and runs
+        the whole batch once.  Returns {tensor name: device tensor}."""
+        h = self.h
+        batch = images_u8.shape[0]
+        self.batch = batch
+        x0 = np.zeros(images_u8.shape[:3] + (16,), np.uint8)
+        x0[..., :3] = images_u8
+        rec = np.zeros(1, qtz.QPARAMS)
+        rec["scale"], rec["zero_point"], rec["min_nudged"], rec["max_nudged"] = np.float32(1.0 / 255.0), 0, 0.0, 1.0
+        tensors = {"in": torch.from_numpy(x0).cuda()}
+        chans = {"in": 3}
+        self.params = {"in": rec[0]}
+        self.layers = []
+        for index, op in enumerate(self.ops):
+            kind = op["op"]
+            L = _Layer()
+            L.op = op
+            if kind in ("conv", "fc"):
+                x, xp = tensors[op["src"]], self.params[op["src"]]
+                xs, zx = np.float32(xp["scale"]), int(xp["zero_point"])
+                w_q, wp, bias_q, wkind = self._prepare_weights(op, index, xs)
+                _, hh, ww, pitch = x.shape
+                k, st, pad = (1, 1, 0) if kind == "fc" else (op["k"], op["stride"], op["pad"])
+                cin, cout = op["cin"], op["cout"]
+                dw = kind == "conv" and op["depthwise"]
+                raw_desc = qtz.conv_desc(calib if kind == "conv" else batch, hh, ww, cin, cout, k, k, st, pad, wkind,
+                                         qtz.OUT_S32_RAW, c_pitch_in=pitch)
+                raw_plan = h.conv_create(raw_desc, w_q, bias_q, depthwise=dw)
+                if kind == "fc":
+                    L.plan, L.args = raw_plan, (zx,)
+                    tensors[op["dst"]] = raw_plan(x, zx).reshape(batch, cout)
+                    self.params[op["dst"]] = None
+                    self.layers.append(L)
+                    continue
+                acc = raw_plan(x[:calib], zx)
+                ap = np.zeros(cout, qtz.QPARAMS)
+                ap["scale"] = xs * wp["scale"]                                   # fp32 product, formed once
+                lo, hi = h.minmax(h.dequantize(acc, ap, axis=3))
+                raw_plan.close()
+                lo, hi = float(lo[0]), float(hi[0])
+                if op["act"] == 1:
+                    lo, hi = max(lo, 0.0), max(hi, 0.0)
+                elif op["act"] == 2:
+                    lo, hi = min(max(lo, 0.0), 6.0), min(max(hi, 0.0), 6.0)
+                yp = qtz.params_from_range(lo, hi)
+                mr = [qtz.quantize_multiplier(float(xs) * float(s) / float(yp["scale"])) for s in wp["scale"]]
+                amin, amax = qtz.activation_range(op["act"], yp["scale"], int(yp["zero_point"]))
+                desc = qtz.conv_desc(batch, hh, ww, cin, cout, k, k, st, pad, wkind, qtz.OUT_U8, c_pitch_in=pitch)
+                L.plan = h.conv_create(desc, w_q, bias_q, None, [m for m, _ in mr], [r for _, r in mr], depthwise=dw)
+                L.args = (zx, int(yp["zero_point"]), amin, amax)
+                tensors[op["dst"]] = L.plan(x, *L.args)
+                chans[op["dst"]] = cout
+                self.params[op["dst"]] = yp
+            elif kind == "add":
+                a, b = self.params[op["a"]], self.params[op["b"]]
+                lo = float(np.float32(a["min_nudged"]) + np.float32(b["min_nudged"]))
+                hi = float(np.float32(a["max_nudged"]) + np.float32(b["max_nudged"]))
+                if op["act"] == 1:
+                    lo, hi = max(lo, 0.0), max(hi, 0.0)
+                yp = qtz.params_from_range(lo, hi)
+                ma, mb, r = qtz.add_params(a["scale"], b["scale"], yp["scale"])
+                amin, amax = qtz.activation_range(op["act"], yp["scale"], int(yp["zero_point"]))
+                L.args = (int(a["zero_point"]), ma, int(b["zero_point"]), mb, r, int(yp["zero_point"]), amin, amax,
+                          chans[op["a"]])
+                ta, tb = tensors[op["a"]], tensors[op["b"]]
+                tensors[op["dst"]] = h.add_u8(ta, L.args[0], ma, tb, L.args[2], mb, r, *L.args[5:])
+                chans[op["dst"]] = chans[op["a"]]
+                self.params[op["dst"]] = yp
+            elif kind == "maxpool":
+                x = tensors[op["src"]]
+                L.args = (chans[op["src"]], op["k"], op["stride"], op["pad"])
+                tensors[op["dst"]] = h.maxpool_u8(x, *L.args)
+                chans[op["dst"]] = chans[op["src"]]
+                self.params[op["dst"]] = self.params[op["src"]]
+            elif kind == "avgpool":
+                x, xp = tensors[op["src"]], self.params[op["src"]]
+                m, r = qtz.quantize_multiplier(1.0 / (x.shape[1] * x.shape[2]))
+                z = int(xp["zero_point"])
+                L.args = (z, z, m, r, chans[op["src"]])
+                tensors[op["dst"]] = h.global_avgpool_u8(x, *L.args)
+                chans[op["dst"]] = chans[op["src"]]
+                self.params[op["dst"]] = xp
+            else:
+                raise ValueError(kind)
+            self.layers.append(L)
+        self.tensors = tensors
+        self.chans = chans
+        return tensors
+
+    # ---- the timed pass ----------------------------------------------------------------------
+    def forward(self, x=None):
+        """Integer-only inference of the whole batch with the plans made by build(); writes into the
+        tensors build() allocated.  Returns the int32 logits tensor."""
+        h, t = self.h, self.tensors
+        if x is not None:
+            t["in"] = x
+        for L in self.layers:
+            op = L.op
+            kind = op["op"]
+            if kind == "conv":
+                L.plan(t[op["src"]], *L.args, out=t[op["dst"]])
+            elif kind == "fc":
+                L.plan(t[op["src"]], *L.args, out=t[op["dst"]])
+            elif kind == "add":
+                a = L.args
+                h.add_u8(t[op["a"]], a[0], a[1], t[op["b"]], a[2], a[3], a[4], a[5], a[6], a[7], a[8], out=t[op["dst"]])
+            elif kind == "maxpool":
+                h.maxpool_u8(t[op["src"]], *L.args, out=t[op["dst"]])
+            else:
+                h.global_avgpool_u8(t[op["src"]], *L.args, out=t[op["dst"]])
+        return t["logits"]
+
+    def num_launch_calls(self):
+        return len(self.layers)
