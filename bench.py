@@ -236,6 +236,81 @@ def time_hbm_kernels(hq, qtz, torch, peaks):
     return res
 
 
+NETWORK_CONFIGS = [("mobilenet_v1", 128, 8), ("resnet50", 256, 8), ("mobilenet_v2_14", 256, 4)]
+
+
+def time_networks(hq, qtz, torch, reps=10, detail=False):
+    """Images/s of whole-network integer inference at the batch sizes of the network workloads
+    (calibration and plan creation outside the timed region; activations stay in HBM)."""
+    from paper_1806_08342_b200 import network
+    res = {}
+    for name, batch, wbits in NETWORK_CONFIGS:
+        ops = synth.NETWORKS[name]()
+        images = synth.network_input(batch, 224, 12)
+        net = network.QuantizedNetwork(hq, ops, 12, wbits)
+        net.build(images, 2)
+        for _ in range(3):
+            net.forward()
+        torch.cuda.synchronize()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        for _ in range(reps):
+            net.forward()
+        e.record(); torch.cuda.synchronize()
+        eager_ms = s.elapsed_time(e) / reps
+        # the same pass replayed from a CUDA graph (no host launch gaps)
+        graph_ms = None
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                net.forward()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    net.forward()
+            torch.cuda.current_stream().wait_stream(side)
+            g.replay(); torch.cuda.synchronize()
+            s.record()
+            for _ in range(reps):
+                g.replay()
+            e.record(); torch.cuda.synchronize()
+            graph_ms = s.elapsed_time(e) / reps
+        except Exception as exc:  # graph capture is an optimisation of the harness, not of the library
+            graph_ms = None
+            res.setdefault("graph_errors", []).append(f"{name}: {type(exc).__name__}: {exc}"[:200])
+        best = min(eager_ms, graph_ms) if graph_ms else eager_ms
+        entry = {"batch": batch, "weight_bits": wbits, "ms_eager": round(eager_ms, 4),
+                 "ms_graph": None if graph_ms is None else round(graph_ms, 4), "images_per_s": round(batch / best * 1e3, 1)}
+        if detail:
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(net.layers) + 1)]
+            t = net.tensors
+            evs[0].record()
+            for i, L in enumerate(net.layers):
+                op = L.op
+                if op["op"] in ("conv", "fc"):
+                    L.plan(t[op["src"]], *L.args, out=t[op["dst"]])
+                elif op["op"] == "add":
+                    a = L.args
+                    hq.add_u8(t[op["a"]], a[0], a[1], t[op["b"]], a[2], a[3], a[4], a[5], a[6], a[7], a[8], out=t[op["dst"]])
+                elif op["op"] == "maxpool":
+                    hq.maxpool_u8(t[op["src"]], *L.args, out=t[op["dst"]])
+                else:
+                    hq.global_avgpool_u8(t[op["src"]], *L.args, out=t[op["dst"]])
+                evs[i + 1].record()
+            torch.cuda.synchronize()
+            rows = []
+            for i, L in enumerate(net.layers):
+                op = L.op
+                kern = L.plan.kernel if op["op"] in ("conv", "fc") else op["op"]
+                rows.append((round(evs[i].elapsed_time(evs[i + 1]) * 1e3, 1), op.get("dst"), kern,
+                             tuple(t[op["dst"]].shape)))
+            entry["layers_us"] = rows
+        res[name] = entry
+        del net
+        torch.cuda.empty_cache()
+    return res
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     from paper_1806_08342_b200 import build as qbuild
@@ -253,6 +328,9 @@ def run_ours(args, rank, world, local_rank):
     hq = qtz.Handle(local_rank)
     if args.hbm_only:
         print(json.dumps({"hbm_kernels": time_hbm_kernels(hq, qtz, torch, peaks)}), flush=True)
+        return
+    if args.networks_only:
+        print(json.dumps({"networks": time_networks(hq, qtz, torch, detail=True)}), flush=True)
         return
     cases = [GemmCase(hq, qtz, torch, s) for s in SIZES]
     torch.cuda.synchronize()
@@ -345,6 +423,7 @@ def run_ours(args, rank, world, local_rank):
     }
     if world == 1 and not args.no_extras:
         out["hbm_kernels"] = time_hbm_kernels(hq, qtz, torch, peaks)
+        out["networks"] = time_networks(hq, qtz, torch)
         out["cpu_baseline"] = cpu_baseline()
     print(json.dumps(out), flush=True)
     if dist is not None:
@@ -360,6 +439,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the HBM-kernel table and the CPU baseline")
     ap.add_argument("--hbm-only", action="store_true",
                     help="run only the element-wise / depthwise kernel table (profiling runs); prints it as JSON")
+    ap.add_argument("--networks-only", action="store_true",
+                    help="run only the whole-network timings, with per-layer times; prints them as JSON")
     ap.add_argument("--sizes", default="", help="comma-separated subset of the sweep (profiling runs); default: all")
     args = ap.parse_args()
     if args.sizes:
