@@ -10,7 +10,7 @@
 //               pixels arrive as zeros) and K-major weight tiles into a ring of swizzled stages
 //   warp 1      MMA issuer: one thread issues tcgen05.mma; two accumulators of up to 256 columns
 //               alternate in TMEM so that the epilogue of tile i overlaps the MMAs of tile i+1
-//   warps 2..5  epilogue: tcgen05.ld, cross terms, requantise, clamp, pack to uint8 in swizzled
+//   warps 2..9  epilogue: tcgen05.ld, cross terms, requantise, clamp, pack to uint8 in swizzled
 //               shared memory, TMA store (which also clips ragged tile edges)
 // Zero filling stands for padding, so the -z_x sum(w) term must skip the padded taps as well:
 // the weight sums are tabulated per border class (which filter rows / columns are cut) and each
@@ -34,8 +34,8 @@ namespace {
 constexpr int kTileM = 128;          // rows of one accumulator (TMEM lanes)
 constexpr int kAccStride = 256;      // TMEM columns between the two accumulators
 constexpr int kTmemCols = 512;
-constexpr int kThreadsTc = 192;      // producer warp, MMA warp, four epilogue warps
-constexpr int kEpiThreads = 128;
+constexpr int kThreadsTc = 320;      // producer warp, MMA warp, eight epilogue warps
+constexpr int kEpiThreads = 256;
 constexpr int kMaxStages = 8;
 constexpr int kMaxCls = 16;
 constexpr int kSmemBudget = 227 * 1024 - 1024;  // leave room for the 1 KB alignment slack
@@ -58,14 +58,14 @@ struct TcArgs {
     const int32_t* xsum;                    // per input pixel channel sums (only when zw != 0)
     int32_t ncls;
     int32_t kvalid[kMaxCls];
-    int32_t zx, zw, zy, act_min, act_max, raw, fast_requant;
+    int32_t zx, zw, zy, act_min, act_max, raw, fast_requant, fold;
     int32_t* y_raw;
     int32_t* status;
     long long wait_budget;
 };
 
 struct SmemLayout {
-    uint32_t a_off, b_off, out_off, corr_off, mult_off, rsh_off, bar_off, total;
+    uint32_t a_off, b_off, out_off, corr_off, mult_off, rsh_off, addhi_off, bar_off, total;
     uint32_t a_stage, b_stage;
 };
 
@@ -78,11 +78,20 @@ __host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, in
     L.b_off = L.a_off + stages * L.a_stage;
     L.out_off = L.b_off + stages * L.b_stage;
     L.corr_off = L.out_off + out_bufs * kTileM * out_box;
-    L.mult_off = L.corr_off + ncls * BN * 4;
+    L.mult_off = L.corr_off + (ncls > 1 ? ncls * BN * 4 : BN * 8);   // [ncls][BN] int32, or [BN] int64 when folded
     L.rsh_off = L.mult_off + BN * 4;
-    L.bar_off = L.rsh_off + BN * 4;
+    L.addhi_off = L.rsh_off + BN * 4;
+    L.bar_off = L.addhi_off + BN * 4;
     L.total = L.bar_off + (2 * kMaxStages + 4) * 8 + 16;
     return L;
+}
+
+// d = (c << 16) | (sat_u8(a) << 8) | sat_u8(b)
+__device__ __forceinline__ uint32_t pack_sat_u8(int32_t a, int32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
 }
 
 __device__ __forceinline__ void report_timeout(int32_t* status, int site)
@@ -247,19 +256,27 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         // ------------------------------ epilogue ----------------------------------
-        const int et = threadIdx.x - 64;             // 0..127
+        // Eight warps: two per TMEM lane quarter.  A thread owns one accumulator row (one output
+        // pixel); the two warps of a quarter split the columns of every staging box in halves.
+        const int et = threadIdx.x - 64;             // 0..255
         const int quarter = warp & 3;                // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;            // which half of a box's columns
         const int row = quarter * 32 + lane;         // accumulator row owned by this thread
-        int32_t* const corr_s = reinterpret_cast<int32_t*>(smem + L.corr_off);
+        int32_t* const corr_s = reinterpret_cast<int32_t*>(smem + L.corr_off);       // [ncls][BN] (general form)
+        int64_t* const add64_s = reinterpret_cast<int64_t*>(smem + L.corr_off);      // [BN]       (folded form)
         int32_t* const mult_s = reinterpret_cast<int32_t*>(smem + L.mult_off);
-        int32_t* const rsh_s = reinterpret_cast<int32_t*>(smem + L.rsh_off);
+        int32_t* const sh_s = reinterpret_cast<int32_t*>(smem + L.rsh_off);
+        int32_t* const addhi_s = reinterpret_cast<int32_t*>(smem + L.addhi_off);
         uint8_t* const out_s = smem + L.out_off;
         const int boxes = a.BN / a.out_box;
+        const int half_cols = a.out_box >> 1;        // 32 or 64 columns per thread and box
         const uint32_t box_bytes = kTileM * a.out_box;
+        const int32_t span = a.act_max - a.act_min, off = a.zy - a.act_min;
+        const uint32_t lo4 = 0x01010101u * static_cast<uint32_t>(a.act_min);
+        const bool fold = a.fold != 0;
         int staged_n_tile = -1;
         uint32_t local = 0, stores = 0;
-        bool alive = true;
-        for (int64_t tile = blockIdx.x; alive && tile < a.num_tiles; tile += gridDim.x, ++local) {
+        for (int64_t tile = blockIdx.x; tile < a.num_tiles; tile += gridDim.x, ++local) {
             const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
             int n_tile;
             int64_t m_tile;
@@ -267,17 +284,29 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int n0 = n_tile * a.BN;
 
             if (n_tile != staged_n_tile) {
+                // per-channel constants of this column tile: cross-term correction (Eq. 5-6), multiplier,
+                // shift, and the rounding constant with the output offset folded in
                 named_barrier(2, kEpiThreads);       // everyone is done with the old tables
                 for (int j = et; j < a.BN; j += kEpiThreads) {
                     const int n = n0 + j;
                     const bool live = n < a.N;
                     const int32_t bias = live ? __ldg(a.bias + n) : 0;
-                    for (int c = 0; c < a.ncls; ++c) {
-                        const int32_t ws = live ? __ldg(a.wsum + static_cast<int64_t>(c) * a.N + n) : 0;
-                        corr_s[c * a.BN + j] = bias - a.zx * ws + a.kvalid[c] * a.zx * a.zw;
+                    const int32_t m = (live && !a.raw) ? __ldg(a.mult + n) : 0;
+                    const int32_t r = (live && !a.raw) ? __ldg(a.rshift + n) : 40;
+                    const int32_t addhi = a.fast_requant ? (2 * off + 1) * (1 << (r - 33)) : 0;
+                    mult_s[j] = m;
+                    sh_s[j] = a.fast_requant ? r - 32 : r;
+                    if (fold) {
+                        const int32_t ws = live ? __ldg(a.wsum + n) : 0;
+                        const int32_t corr = bias - a.zx * ws;
+                        add64_s[j] = static_cast<int64_t>(corr) * m + (static_cast<int64_t>(addhi) << 32);
+                    } else {
+                        addhi_s[j] = addhi;
+                        for (int c = 0; c < a.ncls; ++c) {
+                            const int32_t ws = live ? __ldg(a.wsum + static_cast<int64_t>(c) * a.N + n) : 0;
+                            corr_s[c * a.BN + j] = bias - a.zx * ws + a.kvalid[c] * a.zx * a.zw;
+                        }
                     }
-                    mult_s[j] = (live && !a.raw) ? __ldg(a.mult + n) : 0;
-                    rsh_s[j] = (live && !a.raw) ? __ldg(a.rshift + n) : 40;
                 }
                 staged_n_tile = n_tile;
                 named_barrier(2, kEpiThreads);       // tables visible to all epilogue threads
@@ -318,7 +347,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             const int32_t* const corr_row = corr_s + cls * a.BN;
 
-            // all 128 epilogue threads take the same decision, so nobody is left alone at a barrier
+            // all epilogue threads take the same decision, so nobody is left alone at a barrier
             if (!named_barrier_and(3, kEpiThreads, mbar_wait(bar_tfull + 8 * acc, acc_phase, a.wait_budget))) {
                 report_timeout(a.status, QTZ_SITE_TMEM_FULL);
                 *abort_flag = 1;
@@ -326,11 +355,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kAccStride;
-            const int32_t lo = a.act_min - a.zy, hi = a.act_max - a.zy;
-            const uint32_t zy4 = 0x01010101u * static_cast<uint32_t>(a.zy);
 
             if (a.raw) {
-                for (int j0 = 0; j0 < a.BN && n0 + j0 < a.N; j0 += 32) {
+                // int32 accumulators with the cross terms applied; the two warps of a quarter alternate 32-column chunks
+                for (int j0 = 32 * half; j0 < a.BN && n0 + j0 < a.N; j0 += 64) {
                     uint32_t v[32];
                     tmem_ld_32x32(taddr + j0, v);
                     tmem_ld_wait();
@@ -348,7 +376,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 continue;
             }
 
-            // uint8 output: one staging box (128 rows x out_box bytes) at a time, two boxes in flight
+            // uint8 output: one staging box (128 rows x out_box bytes) at a time, up to two boxes in flight
             for (int bx = 0; bx < boxes; ++bx) {
                 const int nn = n0 + bx * a.out_box;
                 if (nn >= a.N) break;                // boxes entirely beyond the real channels
@@ -358,7 +386,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 named_barrier(1, kEpiThreads);
                 uint8_t* const dst = out_s + buf * box_bytes;
-                for (int col = 0; col < a.out_box && nn + col < a.N; col += 32) {
+                for (int col = half * half_cols; col < (half + 1) * half_cols && nn + col < a.N; col += 32) {
                     const int j0 = bx * a.out_box + col;
                     uint32_t v[32];
                     tmem_ld_32x32(taddr + j0, v);
@@ -366,30 +394,38 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     uint32_t packed[8];
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
-                        const int4 c4 = *reinterpret_cast<const int4*>(corr_row + j0 + 4 * q);
                         const int4 m4 = *reinterpret_cast<const int4*>(mult_s + j0 + 4 * q);
-                        const int4 r4 = *reinterpret_cast<const int4*>(rsh_s + j0 + 4 * q);
-                        const int32_t cc[4] = {c4.x, c4.y, c4.z, c4.w}, mm[4] = {m4.x, m4.y, m4.z, m4.w},
-                                      rr[4] = {r4.x, r4.y, r4.z, r4.w};
-                        uint32_t word = 0;
+                        const int4 s4 = *reinterpret_cast<const int4*>(sh_s + j0 + 4 * q);
+                        const int32_t mm[4] = {m4.x, m4.y, m4.z, m4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+                        int32_t y[4];
+                        if (fold) {
+                            // y - act_min = hi32(acc m + A) >> (r - 32), A = corr m + 2^(r-1) + (z_y - act_min) 2^r
+                            const longlong2 a01 = *reinterpret_cast<const longlong2*>(add64_s + j0 + 4 * q);
+                            const longlong2 a23 = *reinterpret_cast<const longlong2*>(add64_s + j0 + 4 * q + 2);
+                            const int64_t aa[4] = {a01.x, a01.y, a23.x, a23.y};
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int32_t full = static_cast<int32_t>(v[4 * q + e]) + cc[e] + rowterm;
-                            int32_t t;
-                            if (a.fast_requant) {
-                                // r >= 33: the rounding constant 2^(r-1) sits in the high word; shift the high word only
-                                const int64_t prod = static_cast<int64_t>(full) * mm[e] +
-                                                     (static_cast<int64_t>(1u << (rr[e] - 33)) << 32);
-                                t = static_cast<int32_t>(prod >> 32) >> (rr[e] - 32);
-                                t = min(max(t, lo), hi);
-                            } else {
-                                const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(1) << (rr[e] - 1));
-                                const int64_t sh = prod >> rr[e];
-                                t = static_cast<int32_t>(min(max(sh, static_cast<int64_t>(lo)), static_cast<int64_t>(hi)));
+                            for (int e = 0; e < 4; ++e) {
+                                const int64_t prod = static_cast<int64_t>(static_cast<int32_t>(v[4 * q + e])) * mm[e] + aa[e];
+                                y[e] = __vimin_s32_relu(static_cast<int32_t>(prod >> 32) >> ss[e], span);
                             }
-                            word |= (static_cast<uint32_t>(t) & 0xffu) << (8 * e);
+                        } else {
+                            const int4 c4 = *reinterpret_cast<const int4*>(corr_row + j0 + 4 * q);
+                            const int4 h4 = *reinterpret_cast<const int4*>(addhi_s + j0 + 4 * q);
+                            const int32_t cc[4] = {c4.x, c4.y, c4.z, c4.w}, hh[4] = {h4.x, h4.y, h4.z, h4.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const int32_t full = static_cast<int32_t>(v[4 * q + e]) + cc[e] + rowterm;
+                                if (a.fast_requant) {
+                                    const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(hh[e]) << 32);
+                                    y[e] = __vimin_s32_relu(static_cast<int32_t>(prod >> 32) >> ss[e], span);
+                                } else {
+                                    const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(1) << (ss[e] - 1));
+                                    const int64_t sh = (prod >> ss[e]) + off;
+                                    y[e] = static_cast<int32_t>(min(max(sh, static_cast<int64_t>(0)), static_cast<int64_t>(span)));
+                                }
+                            }
                         }
-                        packed[q] = __vadd4(word, zy4);
+                        packed[q] = pack_sat_u8(y[1], y[0], pack_sat_u8(y[3], y[2], 0u)) + lo4;
                     }
                     *reinterpret_cast<uint4*>(dst + swz(row, col, a.out_box)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     *reinterpret_cast<uint4*>(dst + swz(row, col + 16, a.out_box)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
@@ -649,8 +685,8 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.kb_per_tap = a.c_pad / a.BK;
     // N tiling: as few tiles as possible, each a multiple of 32 columns
     a.n_tiles = (d.n + 255) / 256;
-    a.BN = ((d.n + a.n_tiles - 1) / a.n_tiles + 31) / 32 * 32;
-    a.out_box = (a.BN % 128 == 0) ? 128 : ((a.BN % 64 == 0) ? 64 : 32);
+    a.BN = ((d.n + a.n_tiles - 1) / a.n_tiles + 63) / 64 * 64;
+    a.out_box = (a.BN % 128 == 0) ? 128 : 64;
     t->n_pad = a.n_tiles * a.BN;
     a.ncls = pw ? 1 : kMaxCls;
 
@@ -742,7 +778,8 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.xsum = t->xsum;
     a.zw = p->w_zp_signed;
     a.raw = d.outkind == QTZ_OUT_S32_RAW;
-    a.fast_requant = (!a.raw && p->rshift_min >= 33) ? 1 : 0;
+    a.fast_requant = (!a.raw && p->rshift_min >= 33 && p->rshift_max <= 53) ? 1 : 0;
+    a.fold = (a.fast_requant && a.ncls == 1 && a.zw == 0) ? 1 : 0;
     a.status = h->status_dev;
     a.wait_budget = 2000000000LL;  // about one second of SM clocks
     t->grid = static_cast<int>(std::min<int64_t>(a.num_tiles, h->num_sms));
