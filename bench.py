@@ -236,6 +236,34 @@ def time_hbm_kernels(hq, qtz, torch, peaks):
     return res
 
 
+def time_layer(hq, qtz, torch, spec, reps=20):
+    """One convolution layer alone: spec = "batch,h,w,c,n,k,stride[,dw]" (profiling runs)."""
+    v = spec.split(",")
+    b, hh, ww, c, n, k, st = (int(x) for x in v[:7])
+    dw = len(v) > 7 and v[7] == "dw"
+    pad = k // 2
+    x = torch.randint(0, 256, (b, hh, ww, (c + 15) // 16 * 16), dtype=torch.uint8, device="cuda")
+    w = torch.randint(-127, 128, (k, k, c) if dw else (n, k, k, c), dtype=torch.int8, device="cuda")
+    m, r = qtz.quantize_multiplier(1.0 / (40.0 * (k * k * (1 if dw else c)) ** 0.5 * 73.0))
+    plan = hq.conv_create(qtz.conv_desc(b, hh, ww, c, n, k, k, st, pad), w, None, None, np.full(n, m, np.int32),
+                          np.full(n, r, np.int32), depthwise=dw)
+    y = plan.empty_output("cuda")
+    for _ in range(3):
+        plan(x, 7, 20, 20, 255, out=y)
+    torch.cuda.synchronize()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s.record()
+    for _ in range(reps):
+        plan(x, 7, 20, 20, 255, out=y)
+    e.record(); torch.cuda.synchronize()
+    ms = s.elapsed_time(e) / reps
+    oh, ow = plan.oh, plan.ow
+    macs = b * oh * ow * n * k * k * (1 if dw else c)
+    nbytes = b * hh * ww * c + b * oh * ow * n
+    return {"layer": spec, "kernel": plan.kernel, "ms": round(ms, 4), "TOP/s": round(2 * macs / ms / 1e9, 1),
+            "GB/s": round(nbytes / ms / 1e6, 1), "distinct_outputs": int(torch.unique(y[..., :n]).numel())}
+
+
 NETWORK_CONFIGS = [("mobilenet_v1", 128, 8), ("resnet50", 256, 8), ("mobilenet_v2_14", 256, 4)]
 
 
@@ -328,6 +356,9 @@ def run_ours(args, rank, world, local_rank):
     hq = qtz.Handle(local_rank)
     if args.hbm_only:
         print(json.dumps({"hbm_kernels": time_hbm_kernels(hq, qtz, torch, peaks)}), flush=True)
+        return
+    if args.layer:
+        print(json.dumps({"layers": [time_layer(hq, qtz, torch, sp) for sp in args.layer.split(";")]}), flush=True)
         return
     if args.networks_only:
         print(json.dumps({"networks": time_networks(hq, qtz, torch, detail=True)}), flush=True)
@@ -439,6 +470,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the HBM-kernel table and the CPU baseline")
     ap.add_argument("--hbm-only", action="store_true",
                     help="run only the element-wise / depthwise kernel table (profiling runs); prints it as JSON")
+    ap.add_argument("--layer", default="", help='time single conv layers: "batch,h,w,c,n,k,stride[,dw];..." (profiling runs)')
     ap.add_argument("--networks-only", action="store_true",
                     help="run only the whole-network timings, with per-layer times; prints them as JSON")
     ap.add_argument("--sizes", default="", help="comma-separated subset of the sweep (profiling runs); default: all")

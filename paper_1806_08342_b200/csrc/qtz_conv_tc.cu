@@ -10,7 +10,7 @@
 //               pixels arrive as zeros) and K-major weight tiles into a ring of swizzled stages
 //   warp 1      MMA issuer: one thread issues tcgen05.mma; two accumulators of up to 256 columns
 //               alternate in TMEM so that the epilogue of tile i overlaps the MMAs of tile i+1
-//   warps 2..9  epilogue: tcgen05.ld, cross terms, requantise, clamp, pack to uint8 in swizzled
+//   warps 2..17 epilogue (two groups of eight warps, one per accumulator): tcgen05.ld, cross terms, requantise, clamp, pack to uint8 in swizzled
 //               shared memory, TMA store (which also clips ragged tile edges)
 // Zero filling stands for padding, so the -z_x sum(w) term must skip the padded taps as well:
 // the weight sums are tabulated per border class (which filter rows / columns are cut) and each
@@ -34,8 +34,9 @@ namespace {
 constexpr int kTileM = 128;          // rows of one accumulator (TMEM lanes)
 constexpr int kAccStride = 256;      // TMEM columns between the two accumulators
 constexpr int kTmemCols = 512;
-constexpr int kThreadsTc = 320;      // producer warp, MMA warp, eight epilogue warps
-constexpr int kEpiThreads = 256;
+constexpr int kEpiGroups = 2;        // epilogue groups: group g drains accumulator g, so their tiles overlap
+constexpr int kGroupThreads = 256;   // eight warps per group: two per TMEM lane quarter
+constexpr int kThreadsTc = 64 + kEpiGroups * kGroupThreads;   // + producer warp and MMA warp
 constexpr int kMaxStages = 8;
 constexpr int kMaxCls = 16;
 constexpr int kSmemBudget = 227 * 1024 - 1024;  // leave room for the 1 KB alignment slack
@@ -45,11 +46,11 @@ struct TcArgs {
     int32_t tw, th, tb, rows;               // pixel box of one tile and its row count (<= 128)
     int32_t tiles_w, tiles_h, n_tiles;
     int32_t m_tiles, group_m;               // rasterisation: groups of group_m pixel tiles x all n tiles
-    int64_t num_tiles;
+    uint32_t num_tiles;
     int32_t W, H, B;                        // output extent (2-D case: W = number of pixels)
     int32_t taps, kw, pad;
     int32_t kb_per_tap, c_pad;
-    int32_t BK, BN, N, out_box, out_bufs, stages;
+    int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
     uint32_t idesc;
     const int32_t* bias;
     const int32_t* wsum;                    // [ncls][N]
@@ -65,11 +66,12 @@ struct TcArgs {
 };
 
 struct SmemLayout {
-    uint32_t a_off, b_off, out_off, corr_off, mult_off, rsh_off, addhi_off, bar_off, total;
+    uint32_t a_off, b_off, out_off, tbl_off, tbl_stride, mult_rel, sh_rel, addhi_rel, bar_off, total;
     uint32_t a_stage, b_stage;
 };
 
-__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int out_bufs)
+// Operand ring, one output staging box and one set of per-channel tables per epilogue group, barriers.
+__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int groups)
 {
     SmemLayout L;
     L.a_stage = kTileM * BK;
@@ -77,11 +79,12 @@ __host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, in
     L.a_off = 0;
     L.b_off = L.a_off + stages * L.a_stage;
     L.out_off = L.b_off + stages * L.b_stage;
-    L.corr_off = L.out_off + out_bufs * kTileM * out_box;
-    L.mult_off = L.corr_off + (ncls > 1 ? ncls * BN * 4 : BN * 8);   // [ncls][BN] int32, or [BN] int64 when folded
-    L.rsh_off = L.mult_off + BN * 4;
-    L.addhi_off = L.rsh_off + BN * 4;
-    L.bar_off = L.addhi_off + BN * 4;
+    L.tbl_off = L.out_off + groups * kTileM * out_box;
+    L.mult_rel = ncls > 1 ? ncls * BN * 4 : BN * 8;   // first table: [ncls][BN] int32, or [BN] int64 when folded
+    L.sh_rel = L.mult_rel + BN * 4;
+    L.addhi_rel = L.sh_rel + BN * 4;
+    L.tbl_stride = L.addhi_rel + BN * 4;
+    L.bar_off = L.tbl_off + groups * L.tbl_stride;
     L.total = L.bar_off + (2 * kMaxStages + 4) * 8 + 16;
     return L;
 }
@@ -110,14 +113,18 @@ __device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t col, uint32_t box
 // Tile order: pixel tiles are taken in groups of group_m; inside a group the pixel tile varies
 // fastest, so the CTAs running at the same time share a band of A panels and a band of B panels
 // that together fit in L2.
-__device__ __forceinline__ void decode_tile(const TcArgs& a, int64_t tile, int64_t& m_tile, int& n_tile)
+__device__ __forceinline__ void decode_tile(const TcArgs& a, uint32_t tile, uint32_t& m_tile, int& n_tile)
 {
-    const int64_t per_group = static_cast<int64_t>(a.group_m) * a.n_tiles;
-    const int64_t g = tile / per_group, r = tile - g * per_group;
-    const int64_t m_first = g * a.group_m;
-    const int gm = static_cast<int>(a.m_tiles - m_first < a.group_m ? a.m_tiles - m_first : a.group_m);
-    m_tile = m_first + r % gm;
-    n_tile = static_cast<int>(r / gm);
+    // 32-bit unsigned arithmetic on purpose: the tile count is below 2^31 and 64-bit divisions
+    // would cost more than the rest of a small tile's bookkeeping
+    const uint32_t per_group = static_cast<uint32_t>(a.group_m) * static_cast<uint32_t>(a.n_tiles);
+    const uint32_t g = tile / per_group, r = tile - g * per_group;
+    const uint32_t m_first = g * static_cast<uint32_t>(a.group_m);
+    const uint32_t left = static_cast<uint32_t>(a.m_tiles) - m_first;
+    const uint32_t gm = left < static_cast<uint32_t>(a.group_m) ? left : static_cast<uint32_t>(a.group_m);
+    const uint32_t q = r / gm;
+    m_tile = m_first + (r - q * gm);
+    n_tile = static_cast<int>(q);
 }
 
 __global__ void __launch_bounds__(kThreadsTc, 1)
@@ -127,7 +134,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
-    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.out_bufs);
+    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups);
 
     const uint32_t bar_full = base + L.bar_off;
     const uint32_t bar_empty = bar_full + 8 * kMaxStages;
@@ -145,7 +152,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_tfull + 8 * i, 1);
-            mbar_init(bar_tempty + 8 * i, kEpiThreads / 32);
+            mbar_init(bar_tempty + 8 * i, kGroupThreads / 32);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -171,15 +178,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t issued = 0;
             const uint32_t tx = static_cast<uint32_t>(a.rows * a.BK + a.BN * a.BK);
             bool ok = true;
-            for (int64_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
+            for (uint32_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
                 int n_tile;
-                int64_t m_tile;
+                uint32_t m_tile;
                 decode_tile(a, tile, m_tile, n_tile);
                 int w0 = 0, h0 = 0, b0 = 0;
                 if (a.is4d) {
-                    w0 = static_cast<int>(m_tile % a.tiles_w) * a.tw;
-                    h0 = static_cast<int>((m_tile / a.tiles_w) % a.tiles_h) * a.th;
-                    b0 = static_cast<int>(m_tile / (static_cast<int64_t>(a.tiles_w) * a.tiles_h)) * a.tb;
+                    w0 = static_cast<int>(m_tile % static_cast<uint32_t>(a.tiles_w)) * a.tw;
+                    h0 = static_cast<int>((m_tile / static_cast<uint32_t>(a.tiles_w)) % static_cast<uint32_t>(a.tiles_h)) * a.th;
+                    b0 = static_cast<int>(m_tile / static_cast<uint32_t>(a.tiles_w * a.tiles_h)) * a.tb;
                 } else {
                     w0 = static_cast<int>(m_tile) * kTileM;
                 }
@@ -224,7 +231,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t stage = 0, phase = 0;
             uint32_t local = 0;
             bool ok = true;
-            for (int64_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x, ++local) {
+            for (uint32_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x, ++local) {
                 const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget) || *abort_flag) {
                     report_timeout(a.status, QTZ_SITE_TMEM_EMPTY);
@@ -256,38 +263,47 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         // ------------------------------ epilogue ----------------------------------
-        // Eight warps: two per TMEM lane quarter.  A thread owns one accumulator row (one output
-        // pixel); the two warps of a quarter split the columns of every staging box in halves.
-        const int et = threadIdx.x - 64;             // 0..255
+        // Two groups of eight warps.  Group g drains accumulator g (every other tile of this CTA), so
+        // the waits, barriers and stores of one group overlap with the arithmetic of the other.  Inside
+        // a group a thread owns one accumulator row (one output pixel); the two warps of a TMEM lane
+        // quarter split the columns of every staging box in halves.
+        const int et = threadIdx.x - 64;             // 0..511
+        const int grp = et >> 8;                     // epilogue group = accumulator index
+        const int gt = et & (kGroupThreads - 1);     // thread within the group
         const int quarter = warp & 3;                // TMEM lane quarter this warp may read
-        const int half = (warp - 2) >> 2;            // which half of a box's columns
+        const int half = ((warp - 2) >> 2) & 1;      // which half of a box's columns
         const int row = quarter * 32 + lane;         // accumulator row owned by this thread
-        int32_t* const corr_s = reinterpret_cast<int32_t*>(smem + L.corr_off);       // [ncls][BN] (general form)
-        int64_t* const add64_s = reinterpret_cast<int64_t*>(smem + L.corr_off);      // [BN]       (folded form)
-        int32_t* const mult_s = reinterpret_cast<int32_t*>(smem + L.mult_off);
-        int32_t* const sh_s = reinterpret_cast<int32_t*>(smem + L.rsh_off);
-        int32_t* const addhi_s = reinterpret_cast<int32_t*>(smem + L.addhi_off);
-        uint8_t* const out_s = smem + L.out_off;
+        uint8_t* const tbl = smem + L.tbl_off + grp * L.tbl_stride;
+        int32_t* const corr_s = reinterpret_cast<int32_t*>(tbl);                     // [ncls][BN] (general form)
+        int64_t* const add64_s = reinterpret_cast<int64_t*>(tbl);                    // [BN]       (folded form)
+        int32_t* const mult_s = reinterpret_cast<int32_t*>(tbl + L.mult_rel);
+        int32_t* const sh_s = reinterpret_cast<int32_t*>(tbl + L.sh_rel);
+        int32_t* const addhi_s = reinterpret_cast<int32_t*>(tbl + L.addhi_rel);
+        const uint32_t box_bytes = kTileM * a.out_box;
+        uint8_t* const dst = smem + L.out_off + grp * box_bytes;                     // this group's staging box
+        const uint32_t dst_addr = base + L.out_off + grp * box_bytes;
         const int boxes = a.BN / a.out_box;
         const int half_cols = a.out_box >> 1;        // 32 or 64 columns per thread and box
-        const uint32_t box_bytes = kTileM * a.out_box;
         const int32_t span = a.act_max - a.act_min, off = a.zy - a.act_min;
         const uint32_t lo4 = 0x01010101u * static_cast<uint32_t>(a.act_min);
         const bool fold = a.fold != 0;
+        const uint32_t bar_box = 1 + grp, bar_tbl = 3 + grp, bar_vote = 5 + grp;
         int staged_n_tile = -1;
-        uint32_t local = 0, stores = 0;
-        for (int64_t tile = blockIdx.x; tile < a.num_tiles; tile += gridDim.x, ++local) {
+        // with two groups in use, group g takes every other tile (accumulator g); with one, group 0 takes all
+        uint32_t local = grp;
+        uint32_t tile = grp < a.groups ? blockIdx.x + grp * gridDim.x : a.num_tiles;
+        for (; tile < a.num_tiles; tile += a.groups * gridDim.x, local += a.groups) {
             const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
             int n_tile;
-            int64_t m_tile;
+            uint32_t m_tile;
             decode_tile(a, tile, m_tile, n_tile);
             const int n0 = n_tile * a.BN;
 
             if (n_tile != staged_n_tile) {
                 // per-channel constants of this column tile: cross-term correction (Eq. 5-6), multiplier,
                 // shift, and the rounding constant with the output offset folded in
-                named_barrier(2, kEpiThreads);       // everyone is done with the old tables
-                for (int j = et; j < a.BN; j += kEpiThreads) {
+                named_barrier(bar_tbl, kGroupThreads);       // everyone is done with the old tables
+                for (int j = gt; j < a.BN; j += kGroupThreads) {
                     const int n = n0 + j;
                     const bool live = n < a.N;
                     const int32_t bias = live ? __ldg(a.bias + n) : 0;
@@ -309,16 +325,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                 }
                 staged_n_tile = n_tile;
-                named_barrier(2, kEpiThreads);       // tables visible to all epilogue threads
+                named_barrier(bar_tbl, kGroupThreads);       // tables visible to the whole group
             }
 
             // which pixel this row is, its border class and its activation-sum term
             int w0 = 0, h0 = 0, b0 = 0, pw, ph = 0, pb = 0;
             bool row_live;
             if (a.is4d) {
-                w0 = static_cast<int>(m_tile % a.tiles_w) * a.tw;
-                h0 = static_cast<int>((m_tile / a.tiles_w) % a.tiles_h) * a.th;
-                b0 = static_cast<int>(m_tile / (static_cast<int64_t>(a.tiles_w) * a.tiles_h)) * a.tb;
+                w0 = static_cast<int>(m_tile % static_cast<uint32_t>(a.tiles_w)) * a.tw;
+                h0 = static_cast<int>((m_tile / static_cast<uint32_t>(a.tiles_w)) % static_cast<uint32_t>(a.tiles_h)) * a.th;
+                b0 = static_cast<int>(m_tile / static_cast<uint32_t>(a.tiles_w * a.tiles_h)) * a.tb;
                 pw = w0 + row % a.tw;
                 ph = h0 + (row / a.tw) % a.th;
                 pb = b0 + row / (a.tw * a.th);
@@ -347,8 +363,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             const int32_t* const corr_row = corr_s + cls * a.BN;
 
-            // all epilogue threads take the same decision, so nobody is left alone at a barrier
-            if (!named_barrier_and(3, kEpiThreads, mbar_wait(bar_tfull + 8 * acc, acc_phase, a.wait_budget))) {
+            // one lane per warp polls; the vote makes the whole group take the same decision, so nobody
+            // is left alone at a barrier
+            bool landed = true;
+            if (lane == 0) landed = mbar_wait(bar_tfull + 8 * acc, acc_phase, a.wait_budget);
+            if (!named_barrier_and(bar_vote, kGroupThreads, landed)) {
                 report_timeout(a.status, QTZ_SITE_TMEM_FULL);
                 *abort_flag = 1;
                 break;
@@ -376,16 +395,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 continue;
             }
 
-            // uint8 output: one staging box (128 rows x out_box bytes) at a time, up to two boxes in flight
+            // uint8 output: one staging box (128 rows x out_box bytes) at a time
             for (int bx = 0; bx < boxes; ++bx) {
                 const int nn = n0 + bx * a.out_box;
                 if (nn >= a.N) break;                // boxes entirely beyond the real channels
-                const uint32_t buf = stores % a.out_bufs;
-                if (et == 0) {                       // the store that last used this buffer has read it
-                    if (a.out_bufs == 2) tma_store_wait_read_1(); else tma_store_wait_read();
-                }
-                named_barrier(1, kEpiThreads);
-                uint8_t* const dst = out_s + buf * box_bytes;
+                if (gt == 0) tma_store_wait_read();  // this group's previous store has read the box
+                named_barrier(bar_box, kGroupThreads);
                 for (int col = half * half_cols; col < (half + 1) * half_cols && nn + col < a.N; col += 32) {
                     const int j0 = bx * a.out_box + col;
                     uint32_t v[32];
@@ -437,19 +452,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
                 }
                 fence_proxy_async_smem();
-                named_barrier(1, kEpiThreads);
-                if (et == 0) {
-                    const uint32_t src = base + L.out_off + buf * box_bytes;
+                named_barrier(bar_box, kGroupThreads);
+                if (gt == 0) {
                     if (a.is4d)
-                        tma_store_4d(&map_y, src, nn, w0, h0, b0);
+                        tma_store_4d(&map_y, dst_addr, nn, w0, h0, b0);
                     else
-                        tma_store_2d(&map_y, src, nn, w0);
+                        tma_store_2d(&map_y, dst_addr, nn, w0);
                     tma_store_commit();
                 }
-                ++stores;
             }
         }
-        if (et == 0) tma_store_wait_all();
+        if (gt == 0) tma_store_wait_all();
     }
 
     tc_fence_before();
@@ -696,7 +709,8 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
         a.tw = kTileM; a.th = 1; a.tb = 1; a.rows = kTileM;
         a.tiles_w = static_cast<int32_t>((t->in_pixels + kTileM - 1) / kTileM);
         a.tiles_h = 1;
-        a.num_tiles = static_cast<int64_t>(a.tiles_w) * a.n_tiles;
+        if (static_cast<int64_t>(a.tiles_w) * a.n_tiles > 0x7fffffff) return QTZ_ERR_UNSUPPORTED;
+        a.num_tiles = static_cast<uint32_t>(a.tiles_w) * a.n_tiles;
         // the 2-D view treats all pixels as one row of length M
         a.W = static_cast<int32_t>(t->in_pixels);
         a.H = 1;
@@ -717,7 +731,8 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
         a.rows = a.tw * a.th * a.tb;
         a.tiles_w = (a.W + a.tw - 1) / a.tw;
         a.tiles_h = (a.H + a.th - 1) / a.th;
-        a.num_tiles = best_tiles * a.n_tiles;
+        if (best_tiles * a.n_tiles > 0x7fffffff) return QTZ_ERR_UNSUPPORTED;
+        a.num_tiles = static_cast<uint32_t>(best_tiles * a.n_tiles);
     }
     for (int cls = 0; cls < kMaxCls; ++cls) {
         const int rc = cls >> 2, cc = cls & 3;
@@ -728,19 +743,11 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
 
     a.m_tiles = static_cast<int32_t>(a.num_tiles / a.n_tiles);
     a.group_m = std::max(1, std::min(a.m_tiles, 16));
-    a.out_bufs = 2;
     // shared-memory budget -> pipeline depth
-    auto max_stages = [&](int bufs) {
-        int st = kMaxStages;
-        for (; st >= 2; --st)
-            if (make_layout(a.BK, a.BN, st, a.ncls, a.out_box, bufs).total <= static_cast<uint32_t>(kSmemBudget)) break;
-        return st;
-    };
-    // a deeper operand ring beats a second output staging box
-    a.out_bufs = max_stages(1) > max_stages(2) ? 1 : 2;
-    a.stages = max_stages(a.out_bufs);
-    if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
-    t->smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.out_bufs).total + 1024;
+    // worst case (all border classes) for the smem opt-in; every launch picks its own depth
+    a.groups = kEpiGroups;
+    a.stages = 2;
+    if (make_layout(a.BK, a.BN, 2, a.ncls, a.out_box, 1).total > static_cast<uint32_t>(kSmemBudget)) return QTZ_ERR_UNSUPPORTED;
 
     // instruction descriptor: s32 accumulate, A = u8, B = s8, both K-major, N and M of the tile
     a.idesc = (2u << 4) | (0u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) |
@@ -853,8 +860,24 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.zy = y_zp;
     a.act_min = act_min;
     a.act_max = act_max;
+    // with z_x = 0 the cross-term correction no longer depends on the border class: one class, small tables
+    if (x_zp == 0) a.ncls = 1;
+    // operand ring depth: two epilogue groups (overlapped tile drains) unless that would leave fewer than
+    // four stages for a reduction that is longer than the ring
+    auto depth = [&](int groups) {
+        int st_ = kMaxStages;
+        for (; st_ >= 2; --st_)
+            if (make_layout(a.BK, a.BN, st_, a.ncls, a.out_box, groups).total <= static_cast<uint32_t>(kSmemBudget)) break;
+        return st_;
+    };
+    const int kblocks = a.taps * a.kb_per_tap;
+    a.groups = (depth(2) >= 4 || depth(2) >= kblocks + 1) ? 2 : 1;
+    a.stages = depth(a.groups);
+    if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
+    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups).total + 1024;
+    a.fold = (a.fast_requant && a.ncls == 1 && a.zw == 0) ? 1 : 0;
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
-    conv_tc_kernel<<<t->grid, kThreadsTc, t->smem_bytes, st>>>(map_a, t->map_b, map_y, a);
+    conv_tc_kernel<<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, a);
     QTZ_LAUNCH_CHECK(h, "conv_tc_kernel");
     if (p->ev_stop) QTZ_CUDA(h, cudaEventRecord(p->ev_stop, st));
     return QTZ_OK;
