@@ -38,6 +38,7 @@ constexpr int kEpiGroups = 2;        // epilogue groups: group g drains accumula
 constexpr int kGroupThreads = 256;   // eight warps per group: two per TMEM lane quarter
 constexpr int kThreadsTc = 64 + kEpiGroups * kGroupThreads;   // + producer warp and MMA warp
 constexpr int kMaxStages = 8;
+constexpr int kProducerLanes = 4;    // lanes of the producer warp that issue TMA copies side by side
 constexpr int kMaxCls = 16;
 constexpr int kSmemBudget = 227 * 1024 - 1024;  // leave room for the 1 KB alignment slack
 
@@ -173,67 +174,84 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
-        if (lane == 0) {
-            uint32_t stage = 0, phase = 0;
-            uint32_t issued = 0;
-            const uint32_t tx = static_cast<uint32_t>(a.rows * a.BK + a.BN * a.BK);
-            bool ok = true;
-            for (uint32_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
-                int n_tile;
-                uint32_t m_tile;
-                decode_tile(a, tile, m_tile, n_tile);
-                int w0 = 0, h0 = 0, b0 = 0;
-                if (a.is4d) {
-                    w0 = static_cast<int>(m_tile % static_cast<uint32_t>(a.tiles_w)) * a.tw;
-                    h0 = static_cast<int>((m_tile / static_cast<uint32_t>(a.tiles_w)) % static_cast<uint32_t>(a.tiles_h)) * a.th;
-                    b0 = static_cast<int>(m_tile / static_cast<uint32_t>(a.tiles_w * a.tiles_h)) * a.tb;
-                } else {
-                    w0 = static_cast<int>(m_tile) * kTileM;
-                }
-                for (int tap = 0; ok && tap < a.taps; ++tap) {
-                    const int dy = tap / a.kw - a.pad, dx = tap % a.kw - a.pad;
-                    for (int kb = 0; kb < a.kb_per_tap; ++kb) {
-                        if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget) || *abort_flag) {
-                            report_timeout(a.status, QTZ_SITE_SMEM_EMPTY);
-                            *abort_flag = 1;
-                            ok = false;
-                            break;
-                        }
+        // A single thread issuing one K block at a time spends several hundred cycles per block on
+        // its own dependent instructions (barrier poll, address arithmetic, two TMA issues).  Up to
+        // kProducerLanes lanes therefore run the loop in lockstep, lane l taking K blocks l, l+P, ...
+        // of the tile; every lane waits on and arms the barrier of its own stage.
+        const int P = min(min(kblocks, kProducerLanes), a.stages);   // never two lanes on one stage at a time
+        const uint32_t tx = static_cast<uint32_t>(a.rows * a.BK + a.BN * a.BK);
+        const uint32_t nstages = static_cast<uint32_t>(a.stages);
+        uint32_t issued_before = 0;          // K blocks of earlier tiles
+        uint32_t last_stage = 0, last_phase = 0;
+        bool issued_any = false, failed = false;
+        for (uint32_t tile = blockIdx.x; tile < a.num_tiles; tile += gridDim.x) {
+            int n_tile;
+            uint32_t m_tile;
+            decode_tile(a, tile, m_tile, n_tile);
+            int w0 = 0, h0 = 0, b0 = 0;
+            if (a.is4d) {
+                w0 = static_cast<int>(m_tile % static_cast<uint32_t>(a.tiles_w)) * a.tw;
+                h0 = static_cast<int>((m_tile / static_cast<uint32_t>(a.tiles_w)) % static_cast<uint32_t>(a.tiles_h)) * a.th;
+                b0 = static_cast<int>(m_tile / static_cast<uint32_t>(a.tiles_w * a.tiles_h)) * a.tb;
+            } else {
+                w0 = static_cast<int>(m_tile) * kTileM;
+            }
+            for (int kb0 = 0; kb0 < kblocks; kb0 += P) {
+                const int kbl = kb0 + lane;
+                const bool active = lane < P && kbl < kblocks;
+                if (active) {
+                    const uint32_t g = issued_before + static_cast<uint32_t>(kbl);
+                    const uint32_t round = g / nstages, stage = g - round * nstages, phase = round & 1;
+                    const int tap = kbl / a.kb_per_tap, kb = kbl - tap * a.kb_per_tap;
+                    if (mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget)) {
                         mbar_arrive_expect_tx(bar_full + 8 * stage, tx);
                         const uint32_t dst_a = base + L.a_off + stage * L.a_stage;
                         const uint32_t dst_b = base + L.b_off + stage * L.b_stage;
-                        if (a.is4d)
-                            tma_load_4d(dst_a, &map_a, bar_full + 8 * stage, kb * a.BK, w0 + dx, h0 + dy, b0);
-                        else
+                        if (a.is4d) {
+                            const int ty = tap / a.kw;
+                            tma_load_4d(dst_a, &map_a, bar_full + 8 * stage, kb * a.BK, w0 + (tap - ty * a.kw) - a.pad,
+                                        h0 + ty - a.pad, b0);
+                        } else {
                             tma_load_2d(dst_a, &map_a, bar_full + 8 * stage, kb * a.BK, w0);
-                        tma_load_2d(dst_b, &map_b, bar_full + 8 * stage, tap * a.c_pad + kb * a.BK, n_tile * a.BN);
-                        ++issued;
-                        if (++stage == static_cast<uint32_t>(a.stages)) {
-                            stage = 0;
-                            phase ^= 1;
                         }
+                        tma_load_2d(dst_b, &map_b, bar_full + 8 * stage, tap * a.c_pad + kb * a.BK, n_tile * a.BN);
+                        last_stage = stage;
+                        last_phase = phase;
+                        issued_any = true;
+                    } else {
+                        failed = true;
                     }
                 }
-            }
-            if (!ok) {
-                // drain: give the copies already in flight a bounded time to land before the CTA exits
-                const uint32_t pending = issued < static_cast<uint32_t>(a.stages) ? issued : static_cast<uint32_t>(a.stages);
-                for (uint32_t i = 0; i < pending; ++i) {
-                    const uint32_t s = (stage + a.stages - 1 - i) % a.stages;
-                    const uint32_t ph = (s < stage) ? phase : (phase ^ 1);
-                    (void)mbar_wait(bar_full + 8 * s, ph, a.wait_budget);
+                if (__any_sync(0xffffffffu, failed || *abort_flag != 0)) {
+                    failed = true;
+                    break;
                 }
             }
+            if (failed) break;
+            issued_before += static_cast<uint32_t>(kblocks);
+        }
+        if (failed) {
+            if (lane == 0) {
+                report_timeout(a.status, QTZ_SITE_SMEM_EMPTY);
+                *abort_flag = 1;
+            }
+            // drain: give this lane's last copy a bounded time to land before the CTA exits
+            if (issued_any) (void)mbar_wait(bar_full + 8 * last_stage, last_phase, a.wait_budget);
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer --------------------------------
         if (lane == 0) {
+            const uint64_t desc_a0 = make_kmajor_desc(base + L.a_off, a.BK);
+            const uint64_t desc_b0 = make_kmajor_desc(base + L.b_off, a.BK);
+            const uint32_t a_step = L.a_stage >> 4, b_step = L.b_stage >> 4;   // descriptor address units
+            const int mmas = a.BK / 32;          // each MMA consumes 32 bytes of K: advance 2 x 16 B
             uint32_t stage = 0, phase = 0;
             uint32_t local = 0;
             bool ok = true;
+            bool ready = mbar_try_wait(bar_full, 0);
             for (uint32_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x, ++local) {
                 const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
-                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget) || *abort_flag) {
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget)) {
                     report_timeout(a.status, QTZ_SITE_TMEM_EMPTY);
                     *abort_flag = 1;
                     break;
@@ -241,22 +259,23 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kAccStride;
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!mbar_wait(bar_full + 8 * stage, phase, a.wait_budget) || *abort_flag) {
+                    if (!ready && !mbar_wait(bar_full + 8 * stage, phase, a.wait_budget)) {
                         report_timeout(a.status, QTZ_SITE_TMA_FULL);
                         *abort_flag = 1;
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint64_t da = make_kmajor_desc(base + L.a_off + stage * L.a_stage, a.BK);
-                    const uint64_t db = make_kmajor_desc(base + L.b_off + stage * L.b_stage, a.BK);
-                    for (int k = 0; k < a.BK / 32; ++k)  // each MMA consumes 32 bytes of K: advance 2 x 16 B
-                        mma_i8(d_tmem, da + 2 * k, db + 2 * k, a.idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                    mma_commit(bar_empty + 8 * stage);  // frees the stage once these MMAs have read it
+                    const uint64_t da = desc_a0 + stage * a_step, db = desc_b0 + stage * b_step;
+                    const uint32_t freed = bar_empty + 8 * stage;
                     if (++stage == static_cast<uint32_t>(a.stages)) {
                         stage = 0;
                         phase ^= 1;
                     }
+                    // poll the next stage now: the answer arrives while the MMAs below are being issued
+                    ready = mbar_try_wait(bar_full + 8 * stage, phase);
+                    for (int k = 0; k < mmas; ++k) mma_i8(d_tmem, da + 2 * k, db + 2 * k, a.idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    mma_commit(freed);           // frees the stage once these MMAs have read it
                 }
                 if (ok) mma_commit(bar_tfull + 8 * acc);
             }
