@@ -593,6 +593,45 @@ stride_gather_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, i
     reinterpret_cast<uint4*>(out)[t] = v;
 }
 
+// Explicit im2col for layers with a short reduction (3-channel stem convolutions, strided 3x3):
+// row p of `out` holds the kh*kw*c window bytes of output pixel p in OHWI order, out-of-image taps
+// as the code z_x (real zero, Section 2.1) and the tail up to the pitch as 0.  The layer then runs
+// as a pointwise layer over this matrix on the tensor cores.  One thread per 16 output bytes;
+// `lut[k]` gives (dy << 24 | dx << 16 | channel) for window byte k.
+__global__ void __launch_bounds__(kPrepThreads)
+im2col_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, const uint32_t* __restrict__ lut, int h, int w,
+              int pitch, int stride, int pad, int oh, int ow, int64_t pixels, int k_total, int k_pitch, int zx)
+{
+    extern __shared__ uint32_t lut_s[];
+    for (int i = threadIdx.x; i < k_pitch; i += kPrepThreads) lut_s[i] = i < k_total ? lut[i] : 0u;
+    __syncthreads();
+    const int chunks = k_pitch >> 4;
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
+    if (t >= pixels * chunks) return;
+    const int ck = static_cast<int>(t % chunks);
+    int64_t p = t / chunks;
+    const int ox = static_cast<int>(p % ow); p /= ow;
+    const int oy = static_cast<int>(p % oh);
+    const int64_t b = p / oh;
+    const int iy0 = oy * stride - pad, ix0 = ox * stride - pad;
+    const uint8_t* img = x + b * h * w * pitch;
+    uint32_t words[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const int k = 16 * ck + j;
+        uint32_t v = 0;
+        if (k < k_total) {
+            const uint32_t e = lut_s[k];
+            const int iy = iy0 + static_cast<int>(e >> 24), ix = ix0 + static_cast<int>((e >> 16) & 0xff);
+            v = (iy >= 0 && iy < h && ix >= 0 && ix < w)
+                    ? img[(static_cast<int64_t>(iy) * w + ix) * pitch + (e & 0xffff)]
+                    : static_cast<uint32_t>(zx);
+        }
+        words[j >> 2] |= v << (8 * (j & 3));
+    }
+    reinterpret_cast<uint4*>(out)[t] = make_uint4(words[0], words[1], words[2], words[3]);
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------------------
@@ -600,6 +639,9 @@ stride_gather_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, i
 // ------------------------------------------------------------------------------------------
 struct qtz_tc_state {
     TcArgs args{};
+    qtz_conv_desc eff{};       // the layer as the kernel sees it (im2col layers become pointwise over the window matrix)
+    bool im2col = false;
+    uint32_t* lut = nullptr;   // im2col: window byte -> (dy, dx, channel)
     CUtensorMap map_b{};
     int8_t* w_packed = nullptr;
     int32_t* xsum = nullptr;
@@ -670,10 +712,18 @@ bool qtz_encode_u8_map(CUtensorMap* m, const void* base, int rank, const uint64_
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Layers with a short reduction that are neither pointwise nor 3x3/stride 1 go through an explicit
+// im2col and then run as pointwise layers.
+static bool wants_im2col(const qtz_conv_desc& d)
+{
+    if (is_pointwise(d) || (is_3x3(d) && d.c >= 8)) return false;
+    return static_cast<int64_t>(d.kh) * d.kw * d.c <= 1024 && d.kh <= 16 && d.kw <= 16;
+}
+
 bool qtz_tc_supported(const qtz_conv_desc& d)
 {
+    if (wants_im2col(d)) return true;
     if (!(is_pointwise(d) || is_3x3(d))) return false;
-    if (d.c < 8) return false;  // tiny reductions (3-channel stems) stay on the CUDA-core kernel
     if (is_pointwise(d) && d.stride > 4) return false;
     return true;
 }
@@ -682,6 +732,7 @@ void qtz_tc_release(qtz_plan* p)
 {
     if (!p->tc) return;
     cudaFree(p->tc->w_packed);
+    cudaFree(p->tc->lut);
     cudaFree(p->tc->xsum);
     delete p->tc;
     p->tc = nullptr;
@@ -690,7 +741,6 @@ void qtz_tc_release(qtz_plan* p)
 qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
 {
     qtz_ctx* h = p->h;
-    const qtz_conv_desc& d = p->d;
     if (!encode_fn()) {
         h->last_error = "cuTensorMapEncodeTiled is not available from the driver";
         return QTZ_ERR_CUDA;
@@ -698,6 +748,24 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     qtz_tc_state* t = new (std::nothrow) qtz_tc_state();
     if (!t) return QTZ_ERR_INVALID_ARG;
     p->tc = t;
+    t->eff = p->d;
+    t->im2col = wants_im2col(p->d);
+    if (t->im2col) {
+        const qtz_conv_desc& o = p->d;
+        const int k_total = o.kh * o.kw * o.c;
+        t->eff.h = p->oh; t->eff.w = p->ow;
+        t->eff.c = k_total; t->eff.c_pitch_in = (k_total + 15) / 16 * 16;
+        t->eff.kh = t->eff.kw = 1; t->eff.stride = 1; t->eff.pad = 0;
+        std::vector<uint32_t> lut(static_cast<size_t>(k_total));
+        for (int k = 0; k < k_total; ++k) {
+            const int tap = k / o.c, ch = k - tap * o.c;
+            lut[k] = (static_cast<uint32_t>(tap / o.kw) << 24) | (static_cast<uint32_t>(tap % o.kw) << 16) | static_cast<uint32_t>(ch);
+        }
+        QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->lut), sizeof(uint32_t) * lut.size()));
+        QTZ_CUDA(h, cudaMemcpyAsync(t->lut, lut.data(), sizeof(uint32_t) * lut.size(), cudaMemcpyHostToDevice, st));
+        QTZ_CUDA(h, cudaStreamSynchronize(st));   // the staging vector goes out of scope
+    }
+    const qtz_conv_desc& d = t->eff;
     TcArgs& a = t->args;
     const bool pw = is_pointwise(d);
     a.taps = pw ? 1 : 9;
@@ -784,7 +852,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
 
     if (p->w_zp_signed != 0)
         QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->xsum), sizeof(int32_t) * static_cast<size_t>(t->in_pixels)));
-    if (pw && d.stride > 1)
+    if ((pw && d.stride > 1) || t->im2col)
         QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->x_gather), static_cast<size_t>(t->in_pixels) * d.c_pitch_in));
 
     // the weight map never changes
@@ -823,12 +891,20 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
 {
     qtz_ctx* h = p->h;
     qtz_tc_state* t = p->tc;
-    const qtz_conv_desc& d = p->d;
+    const qtz_conv_desc& d = t->eff;
     TcArgs a = t->args;
     const bool pw = is_pointwise(d);
 
     const uint8_t* xin = x;
-    if (pw && d.stride > 1) {
+    if (t->im2col) {
+        const qtz_conv_desc& o = p->d;
+        const int64_t work = t->in_pixels * (d.c_pitch_in >> 4);
+        im2col_kernel<<<static_cast<unsigned>((work + kPrepThreads - 1) / kPrepThreads), kPrepThreads,
+                        sizeof(uint32_t) * d.c_pitch_in, st>>>(x, p->x_gather, t->lut, o.h, o.w, o.c_pitch_in, o.stride, o.pad,
+                                                               p->oh, p->ow, t->in_pixels, d.c, d.c_pitch_in, x_zp);
+        QTZ_LAUNCH_CHECK(h, "im2col_kernel");
+        xin = p->x_gather;
+    } else if (pw && d.stride > 1) {
         const int64_t work = t->in_pixels * (d.c_pitch_in >> 4);
         stride_gather_kernel<<<static_cast<unsigned>((work + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
             x, p->x_gather, d.batch, d.h, d.w, d.c_pitch_in, d.stride, p->oh, p->ow);

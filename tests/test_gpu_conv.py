@@ -75,6 +75,8 @@ STEM_SHAPES = [
     (1, 8, 8, 16, 16, 3, 1, 0),       # no padding
     (1, 5, 5, 300, 10, 3, 1, 1),      # K = 2700 spans several K chunks
     (1, 1, 1, 8, 8, 1, 1, 0),         # single output pixel
+    (1, 9, 9, 160, 24, 3, 2, 1),      # strided 3x3 with a long reduction (K = 1440): the CUDA-core fallback
+    (2, 11, 9, 130, 20, 5, 1, 2),     # 5x5 with K = 3250: fallback as well
 ]
 
 
@@ -82,7 +84,8 @@ STEM_SHAPES = [
 @pytest.mark.parametrize("wkind", [qtz.W_S8_PER_CHANNEL_SYM, qtz.W_U8_PER_LAYER_ASYM,
                                    qtz.W_S4_PACKED_PER_CHANNEL_SYM])
 def test_conv_generic_shapes(hq, shape, wkind):
-    conv_case(hq, *shape, wkind, seed=100 + shape[1])
+    long_k = shape[5] * shape[5] * shape[3] > 1024 and shape[5] > 1 and not (shape[5] == 3 and shape[6] == 1 and shape[7] == 1)
+    conv_case(hq, *shape, wkind, seed=100 + shape[1], expect_kernel="direct" if long_k else "tcgen05")
 
 
 @pytest.mark.parametrize("shape", STEM_SHAPES[:4])
