@@ -42,7 +42,32 @@ constexpr int kProducerLanes = 4;    // lanes of the producer warp that issue TM
 constexpr int kMaxCls = 16;
 constexpr int kSmemBudget = 227 * 1024 - 1024;  // leave room for the 1 KB alignment slack
 
+// Division of a 31-bit unsigned number by a constant known on the host, as one high multiply and one
+// shift (round-up reciprocal: q = (n * ceil(2^p / d)) >> p with p = 31 + ceil(log2 d), exact for n < 2^31).
+struct FastDiv {
+    uint32_t mul, shr, d;
+};
+
+__host__ inline FastDiv make_fastdiv(uint32_t d)
+{
+    FastDiv f{0u, 0u, d};
+    if (d > 1) {
+        uint32_t lg = 0;
+        while ((1ull << lg) < d) ++lg;
+        const uint32_t p = 31 + lg;
+        f.mul = static_cast<uint32_t>(((1ull << p) + d - 1) / d);
+        f.shr = p - 32;
+    }
+    return f;
+}
+
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f)
+{
+    return f.d > 1 ? (__umulhi(n, f.mul) >> f.shr) : n;
+}
+
 struct TcArgs {
+    FastDiv dv_per_group, dv_group_m, dv_group_last, dv_tiles_w, dv_tiles_h;
     int32_t is4d;
     int32_t tw, th, tb, rows;               // pixel box of one tile and its row count (<= 128)
     int32_t tiles_w, tiles_h, n_tiles;
@@ -111,21 +136,79 @@ __device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t col, uint32_t box
     return off ^ (((off >> 7) & ((box >> 4) - 1)) << 4);
 }
 
+// Requantises 32 accumulator columns of one row and returns them as 8 packed words.
+//   kMode 0 (folded):  y - act_min = hi32(acc m + A) >> (r - 32), A = corr m + 2^(r-1) + (z_y - act_min) 2^r
+//   kMode 1 (general): the correction (border class, activation sums) is added to acc first
+//   kMode 2 (any shift): 64-bit shift and clamp
+template <int kMode>
+__device__ __forceinline__ void requant32(const uint32_t (&v)[32], const int32_t* __restrict__ mult_s,
+                                          const int32_t* __restrict__ sh_s, const int64_t* __restrict__ add64_s,
+                                          const int32_t* __restrict__ corr_row, const int32_t* __restrict__ addhi_s,
+                                          int32_t rowterm, int32_t span, int32_t off, uint32_t lo4, uint32_t (&packed)[8])
+{
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const int4 m4 = *reinterpret_cast<const int4*>(mult_s + 4 * q);
+        const int4 s4 = *reinterpret_cast<const int4*>(sh_s + 4 * q);
+        const int32_t mm[4] = {m4.x, m4.y, m4.z, m4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+        int32_t y[4];
+        if (kMode == 0) {
+            const longlong2 a01 = *reinterpret_cast<const longlong2*>(add64_s + 4 * q);
+            const longlong2 a23 = *reinterpret_cast<const longlong2*>(add64_s + 4 * q + 2);
+            const int64_t aa[4] = {a01.x, a01.y, a23.x, a23.y};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int64_t prod = static_cast<int64_t>(static_cast<int32_t>(v[4 * q + e])) * mm[e] + aa[e];
+                y[e] = __vimin_s32_relu(static_cast<int32_t>(prod >> 32) >> ss[e], span);
+            }
+        } else {
+            const int4 c4 = *reinterpret_cast<const int4*>(corr_row + 4 * q);
+            const int4 h4 = *reinterpret_cast<const int4*>(addhi_s + 4 * q);
+            const int32_t cc[4] = {c4.x, c4.y, c4.z, c4.w}, hh[4] = {h4.x, h4.y, h4.z, h4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int32_t full = static_cast<int32_t>(v[4 * q + e]) + cc[e] + rowterm;
+                if (kMode == 1) {
+                    const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(hh[e]) << 32);
+                    y[e] = __vimin_s32_relu(static_cast<int32_t>(prod >> 32) >> ss[e], span);
+                } else {
+                    const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(1) << (ss[e] - 1));
+                    const int64_t sh = (prod >> ss[e]) + off;
+                    y[e] = static_cast<int32_t>(min(max(sh, static_cast<int64_t>(0)), static_cast<int64_t>(span)));
+                }
+            }
+        }
+        packed[q] = pack_sat_u8(y[1], y[0], pack_sat_u8(y[3], y[2], 0u)) + lo4;
+    }
+}
+
 // Tile order: pixel tiles are taken in groups of group_m; inside a group the pixel tile varies
 // fastest, so the CTAs running at the same time share a band of A panels and a band of B panels
 // that together fit in L2.
 __device__ __forceinline__ void decode_tile(const TcArgs& a, uint32_t tile, uint32_t& m_tile, int& n_tile)
 {
-    // 32-bit unsigned arithmetic on purpose: the tile count is below 2^31 and 64-bit divisions
-    // would cost more than the rest of a small tile's bookkeeping
-    const uint32_t per_group = static_cast<uint32_t>(a.group_m) * static_cast<uint32_t>(a.n_tiles);
-    const uint32_t g = tile / per_group, r = tile - g * per_group;
+    const uint32_t g = fdiv(tile, a.dv_per_group), r = tile - g * a.dv_per_group.d;
     const uint32_t m_first = g * static_cast<uint32_t>(a.group_m);
-    const uint32_t left = static_cast<uint32_t>(a.m_tiles) - m_first;
-    const uint32_t gm = left < static_cast<uint32_t>(a.group_m) ? left : static_cast<uint32_t>(a.group_m);
-    const uint32_t q = r / gm;
-    m_tile = m_first + (r - q * gm);
+    const bool last = static_cast<uint32_t>(a.m_tiles) - m_first < static_cast<uint32_t>(a.group_m);   // a shorter final group
+    const uint32_t q = last ? fdiv(r, a.dv_group_last) : fdiv(r, a.dv_group_m);
+    m_tile = m_first + (r - q * (last ? a.dv_group_last.d : a.dv_group_m.d));
     n_tile = static_cast<int>(q);
+}
+
+// First pixel (w0, h0, b0) of pixel tile m_tile.
+__device__ __forceinline__ void tile_origin(const TcArgs& a, uint32_t m_tile, int& w0, int& h0, int& b0)
+{
+    if (a.is4d) {
+        const uint32_t q1 = fdiv(m_tile, a.dv_tiles_w);              // m_tile / tiles_w
+        const uint32_t q2 = fdiv(q1, a.dv_tiles_h);                   // ... / tiles_h
+        w0 = static_cast<int>(m_tile - q1 * a.dv_tiles_w.d) * a.tw;
+        h0 = static_cast<int>(q1 - q2 * a.dv_tiles_h.d) * a.th;
+        b0 = static_cast<int>(q2) * a.tb;
+    } else {
+        w0 = static_cast<int>(m_tile) * kTileM;
+        h0 = 0;
+        b0 = 0;
+    }
 }
 
 __global__ void __launch_bounds__(kThreadsTc, 1)
@@ -188,14 +271,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int n_tile;
             uint32_t m_tile;
             decode_tile(a, tile, m_tile, n_tile);
-            int w0 = 0, h0 = 0, b0 = 0;
-            if (a.is4d) {
-                w0 = static_cast<int>(m_tile % static_cast<uint32_t>(a.tiles_w)) * a.tw;
-                h0 = static_cast<int>((m_tile / static_cast<uint32_t>(a.tiles_w)) % static_cast<uint32_t>(a.tiles_h)) * a.th;
-                b0 = static_cast<int>(m_tile / static_cast<uint32_t>(a.tiles_w * a.tiles_h)) * a.tb;
-            } else {
-                w0 = static_cast<int>(m_tile) * kTileM;
-            }
+            int w0, h0, b0;
+            tile_origin(a, m_tile, w0, h0, b0);
             for (int kb0 = 0; kb0 < kblocks; kb0 += P) {
                 const int kbl = kb0 + lane;
                 const bool active = lane < P && kbl < kblocks;
@@ -306,7 +383,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int32_t span = a.act_max - a.act_min, off = a.zy - a.act_min;
         const uint32_t lo4 = 0x01010101u * static_cast<uint32_t>(a.act_min);
         const bool fold = a.fold != 0;
+        const int mode = fold ? 0 : (a.fast_requant ? 1 : 2);
         const uint32_t bar_box = 1 + grp, bar_tbl = 3 + grp, bar_vote = 5 + grp;
+        // this thread's pixel inside a tile never changes
+        const int dr_w = a.is4d ? row % a.tw : row;
+        const int dr_h = a.is4d ? (row / a.tw) % a.th : 0;
+        const int dr_b = a.is4d ? row / (a.tw * a.th) : 0;
         int staged_n_tile = -1;
         // with two groups in use, group g takes every other tile (accumulator g); with one, group 0 takes all
         uint32_t local = grp;
@@ -348,21 +430,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
 
             // which pixel this row is, its border class and its activation-sum term
-            int w0 = 0, h0 = 0, b0 = 0, pw, ph = 0, pb = 0;
-            bool row_live;
-            if (a.is4d) {
-                w0 = static_cast<int>(m_tile % static_cast<uint32_t>(a.tiles_w)) * a.tw;
-                h0 = static_cast<int>((m_tile / static_cast<uint32_t>(a.tiles_w)) % static_cast<uint32_t>(a.tiles_h)) * a.th;
-                b0 = static_cast<int>(m_tile / static_cast<uint32_t>(a.tiles_w * a.tiles_h)) * a.tb;
-                pw = w0 + row % a.tw;
-                ph = h0 + (row / a.tw) % a.th;
-                pb = b0 + row / (a.tw * a.th);
-                row_live = row < a.rows && pw < a.W && ph < a.H && pb < a.B;
-            } else {
-                w0 = static_cast<int>(m_tile) * kTileM;
-                pw = w0 + row;
-                row_live = pw < a.W;
-            }
+            int w0, h0, b0;
+            tile_origin(a, m_tile, w0, h0, b0);
+            const int pw = w0 + dr_w, ph = h0 + dr_h, pb = b0 + dr_b;
+            const bool row_live = row < a.rows && pw < a.W && ph < a.H && pb < a.B;
             int cls = 0;
             if (a.ncls > 1) cls = ((ph == 0) | ((ph == a.H - 1) << 1)) * 4 + ((pw == 0) | ((pw == a.W - 1) << 1));
             int32_t rowterm = 0;
@@ -426,41 +497,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     tmem_ld_32x32(taddr + j0, v);
                     tmem_ld_wait();
                     uint32_t packed[8];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const int4 m4 = *reinterpret_cast<const int4*>(mult_s + j0 + 4 * q);
-                        const int4 s4 = *reinterpret_cast<const int4*>(sh_s + j0 + 4 * q);
-                        const int32_t mm[4] = {m4.x, m4.y, m4.z, m4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
-                        int32_t y[4];
-                        if (fold) {
-                            // y - act_min = hi32(acc m + A) >> (r - 32), A = corr m + 2^(r-1) + (z_y - act_min) 2^r
-                            const longlong2 a01 = *reinterpret_cast<const longlong2*>(add64_s + j0 + 4 * q);
-                            const longlong2 a23 = *reinterpret_cast<const longlong2*>(add64_s + j0 + 4 * q + 2);
-                            const int64_t aa[4] = {a01.x, a01.y, a23.x, a23.y};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const int64_t prod = static_cast<int64_t>(static_cast<int32_t>(v[4 * q + e])) * mm[e] + aa[e];
-                                y[e] = __vimin_s32_relu(static_cast<int32_t>(prod >> 32) >> ss[e], span);
-                            }
-                        } else {
-                            const int4 c4 = *reinterpret_cast<const int4*>(corr_row + j0 + 4 * q);
-                            const int4 h4 = *reinterpret_cast<const int4*>(addhi_s + j0 + 4 * q);
-                            const int32_t cc[4] = {c4.x, c4.y, c4.z, c4.w}, hh[4] = {h4.x, h4.y, h4.z, h4.w};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const int32_t full = static_cast<int32_t>(v[4 * q + e]) + cc[e] + rowterm;
-                                if (a.fast_requant) {
-                                    const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(hh[e]) << 32);
-                                    y[e] = __vimin_s32_relu(static_cast<int32_t>(prod >> 32) >> ss[e], span);
-                                } else {
-                                    const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(1) << (ss[e] - 1));
-                                    const int64_t sh = (prod >> ss[e]) + off;
-                                    y[e] = static_cast<int32_t>(min(max(sh, static_cast<int64_t>(0)), static_cast<int64_t>(span)));
-                                }
-                            }
-                        }
-                        packed[q] = pack_sat_u8(y[1], y[0], pack_sat_u8(y[3], y[2], 0u)) + lo4;
-                    }
+                    if (mode == 0)
+                        requant32<0>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
+                    else if (mode == 1)
+                        requant32<1>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
+                    else
+                        requant32<2>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
                     *reinterpret_cast<uint4*>(dst + swz(row, col, a.out_box)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     *reinterpret_cast<uint4*>(dst + swz(row, col + 16, a.out_box)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
                 }
@@ -830,6 +872,11 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
 
     a.m_tiles = static_cast<int32_t>(a.num_tiles / a.n_tiles);
     a.group_m = std::max(1, std::min(a.m_tiles, 16));
+    a.dv_per_group = make_fastdiv(static_cast<uint32_t>(a.group_m) * a.n_tiles);
+    a.dv_group_m = make_fastdiv(static_cast<uint32_t>(a.group_m));
+    a.dv_group_last = make_fastdiv(static_cast<uint32_t>(std::max(1, a.m_tiles % a.group_m)));
+    a.dv_tiles_w = make_fastdiv(static_cast<uint32_t>(a.tiles_w));
+    a.dv_tiles_h = make_fastdiv(static_cast<uint32_t>(std::max(1, a.tiles_h)));
     // shared-memory budget -> pipeline depth
     // worst case (all border classes) for the smem opt-in; every launch picks its own depth
     a.groups = kEpiGroups;
