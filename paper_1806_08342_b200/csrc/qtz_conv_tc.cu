@@ -77,6 +77,7 @@ struct TcArgs {
     int32_t taps, kw, pad;
     int32_t kb_per_tap, c_pad;
     int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
+    int32_t obuf;                           // staging boxes per epilogue group (1..4)
     uint32_t idesc;
     const int32_t* bias;
     const int32_t* wsum;                    // [ncls][N]
@@ -97,7 +98,7 @@ struct SmemLayout {
 };
 
 // Operand ring, one output staging box and one set of per-channel tables per epilogue group, barriers.
-__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int groups)
+__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int groups, int obuf)
 {
     SmemLayout L;
     L.a_stage = kTileM * BK;
@@ -105,7 +106,7 @@ __host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, in
     L.a_off = 0;
     L.b_off = L.a_off + stages * L.a_stage;
     L.out_off = L.b_off + stages * L.b_stage;
-    L.tbl_off = L.out_off + groups * kTileM * out_box;
+    L.tbl_off = L.out_off + groups * obuf * kTileM * out_box;
     L.mult_rel = ncls > 1 ? ncls * BN * 4 : BN * 8;   // first table: [ncls][BN] int32, or [BN] int64 when folded
     L.sh_rel = L.mult_rel + BN * 4;
     L.addhi_rel = L.sh_rel + BN * 4;
@@ -218,7 +219,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
-    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups);
+    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf);
 
     const uint32_t bar_full = base + L.bar_off;
     const uint32_t bar_empty = bar_full + 8 * kMaxStages;
@@ -376,8 +377,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int32_t* const sh_s = reinterpret_cast<int32_t*>(tbl + L.sh_rel);
         int32_t* const addhi_s = reinterpret_cast<int32_t*>(tbl + L.addhi_rel);
         const uint32_t box_bytes = kTileM * a.out_box;
-        uint8_t* const dst = smem + L.out_off + grp * box_bytes;                     // this group's staging box
-        const uint32_t dst_addr = base + L.out_off + grp * box_bytes;
+        const uint32_t out_rel = L.out_off + grp * a.obuf * box_bytes;               // this group's staging boxes
+        uint32_t slot = 0;                                                           // box written next
         const int boxes = a.BN / a.out_box;
         const int half_cols = a.out_box >> 1;        // 32 or 64 columns per thread and box
         const int32_t span = a.act_max - a.act_min, off = a.zy - a.act_min;
@@ -489,8 +490,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int bx = 0; bx < boxes; ++bx) {
                 const int nn = n0 + bx * a.out_box;
                 if (nn >= a.N) break;                // boxes entirely beyond the real channels
-                if (gt == 0) tma_store_wait_read();  // this group's previous store has read the box
-                named_barrier(bar_box, kGroupThreads);
+                uint8_t* const dst = smem + out_rel + slot * box_bytes;
+                if (a.obuf == 1) {
+                    if (gt == 0) tma_store_wait_read();  // this group's previous store has read the box
+                    named_barrier(bar_box, kGroupThreads);
+                }
                 for (int col = half * half_cols; col < (half + 1) * half_cols && nn + col < a.N; col += 32) {
                     const int j0 = bx * a.out_box + col;
                     uint32_t v[32];
@@ -513,14 +517,23 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
                 }
                 fence_proxy_async_smem();
+                // With several boxes the barrier below also tells the group that the box written next is
+                // free: the store that last used it is the oldest of the obuf - 1 still allowed to be reading.
+                if (gt == 0) {
+                    if (a.obuf == 2) tma_store_wait_read_n<0>();
+                    else if (a.obuf == 3) tma_store_wait_read_n<1>();
+                    else if (a.obuf >= 4) tma_store_wait_read_n<2>();
+                }
                 named_barrier(bar_box, kGroupThreads);
                 if (gt == 0) {
+                    const uint32_t src = base + out_rel + slot * box_bytes;
                     if (a.is4d)
-                        tma_store_4d(&map_y, dst_addr, nn, w0, h0, b0);
+                        tma_store_4d(&map_y, src, nn, w0, h0, b0);
                     else
-                        tma_store_2d(&map_y, dst_addr, nn, w0);
+                        tma_store_2d(&map_y, src, nn, w0);
                     tma_store_commit();
                 }
+                slot = (slot + 1 == static_cast<uint32_t>(a.obuf)) ? 0 : slot + 1;
             }
         }
         if (gt == 0) tma_store_wait_all();
@@ -881,7 +894,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     // worst case (all border classes) for the smem opt-in; every launch picks its own depth
     a.groups = kEpiGroups;
     a.stages = 2;
-    if (make_layout(a.BK, a.BN, 2, a.ncls, a.out_box, 1).total > static_cast<uint32_t>(kSmemBudget)) return QTZ_ERR_UNSUPPORTED;
+    if (make_layout(a.BK, a.BN, 2, a.ncls, a.out_box, 1, 1).total > static_cast<uint32_t>(kSmemBudget)) return QTZ_ERR_UNSUPPORTED;
 
     // instruction descriptor: s32 accumulate, A = u8, B = s8, both K-major, N and M of the tile
     a.idesc = (2u << 4) | (0u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) |
@@ -1004,19 +1017,32 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.act_max = act_max;
     // with z_x = 0 the cross-term correction no longer depends on the border class: one class, small tables
     if (x_zp == 0) a.ncls = 1;
-    // operand ring depth: two epilogue groups (overlapped tile drains) unless that would leave fewer than
-    // four stages for a reduction that is longer than the ring
-    auto depth = [&](int groups) {
+    // Shared memory is split between the operand ring, the epilogue groups and their staging boxes.
+    // Preference: two groups (overlapped tile drains) with two or three boxes each (the store of one box
+    // overlaps the arithmetic of the next), as long as the ring keeps four stages, or the whole
+    // reduction plus one block when that is shorter.
+    auto depth = [&](int groups, int obuf) {
         int st_ = kMaxStages;
         for (; st_ >= 2; --st_)
-            if (make_layout(a.BK, a.BN, st_, a.ncls, a.out_box, groups).total <= static_cast<uint32_t>(kSmemBudget)) break;
+            if (make_layout(a.BK, a.BN, st_, a.ncls, a.out_box, groups, obuf).total <= static_cast<uint32_t>(kSmemBudget)) break;
         return st_;
     };
     const int kblocks = a.taps * a.kb_per_tap;
-    a.groups = (depth(2) >= 4 || depth(2) >= kblocks + 1) ? 2 : 1;
-    a.stages = depth(a.groups);
+    const int need = std::min(4, kblocks + 1);
+    static const int choice[5][2] = {{2, 3}, {2, 2}, {1, 2}, {2, 1}, {1, 1}};
+    a.groups = 1;
+    a.obuf = 1;
+    for (const auto& c : choice) {
+        const int ob = a.raw ? 1 : c[1];             // the boxes rotate across tiles as well
+        if (depth(c[0], ob) >= need) {
+            a.groups = c[0];
+            a.obuf = ob;
+            break;
+        }
+    }
+    a.stages = depth(a.groups, a.obuf);
     if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
-    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups).total + 1024;
+    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf).total + 1024;
     a.fold = (a.fast_requant && a.ncls == 1 && a.zw == 0) ? 1 : 0;
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
     conv_tc_kernel<<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, a);

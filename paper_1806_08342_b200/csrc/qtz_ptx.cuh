@@ -47,14 +47,29 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return done != 0;
 }
 
-// Waits for the phase with the given parity to complete; gives up after `budget` cycles.
+// Same test, but the hardware may park the thread for up to `hint_ns` nanoseconds while the phase is
+// still open; it resumes as soon as the phase completes.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t hint_ns)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return done != 0;
+}
+
+// Waits for the phase with the given parity to complete; gives up after `budget` cycles.  The
+// waiting thread is parked by the barrier unit between polls, so a long wait costs few issue slots.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long budget)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
-    while (!mbar_try_wait(bar, parity)) {
+    while (!mbar_try_wait_parked(bar, parity, 4000u)) {
         if (clock64() - start > budget) return false;
-        __nanosleep(32);   // leave the issue slots to the warps that have work
     }
     return true;
 }
@@ -98,8 +113,12 @@ __device__ __forceinline__ void tma_store_4d(const void* tmap, uint32_t src, int
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Waits until the committed bulk stores have finished READING shared memory.
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-// Same, but the most recently committed group may still be reading.
-__device__ __forceinline__ void tma_store_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+// Same, but the kPending most recently committed groups may still be reading.
+template <int kPending>
+__device__ __forceinline__ void tma_store_wait_read_n()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kPending) : "memory");
+}
 // Waits until the committed bulk stores are complete.
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // Makes generic-proxy writes to shared memory visible to the async proxy (TMA, tcgen05).
