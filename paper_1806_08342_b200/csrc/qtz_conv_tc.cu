@@ -10,8 +10,11 @@
 //               pixels arrive as zeros) and K-major weight tiles into a ring of swizzled stages
 //   warp 1      MMA issuer: one thread issues tcgen05.mma; two accumulators of up to 256 columns
 //               alternate in TMEM so that the epilogue of tile i overlaps the MMAs of tile i+1
-//   warps 2..17 epilogue (two groups of eight warps, one per accumulator): tcgen05.ld, cross terms, requantise, clamp, pack to uint8 in swizzled
-//               shared memory, TMA store (which also clips ragged tile edges)
+//   warps 2..17 epilogue, two groups of eight warps (one group per accumulator): tcgen05.ld, cross
+//               terms, requantise, clamp, pack to uint8 into a rotating set of swizzled staging boxes;
+//               the warps signal each filled box on an mbarrier and never wait for one another
+//   warps 18,19 one store thread per group: TMA store of every filled box (which also clips ragged
+//               tile edges), box handed back once the store has read it
 // Zero filling stands for padding, so the -z_x sum(w) term must skip the padded taps as well:
 // the weight sums are tabulated per border class (which filter rows / columns are cut) and each
 // epilogue thread, owning one output pixel, picks its class.
@@ -36,7 +39,9 @@ constexpr int kAccStride = 256;      // TMEM columns between the two accumulator
 constexpr int kTmemCols = 512;
 constexpr int kEpiGroups = 2;        // epilogue groups: group g drains accumulator g, so their tiles overlap
 constexpr int kGroupThreads = 256;   // eight warps per group: two per TMEM lane quarter
-constexpr int kThreadsTc = 64 + kEpiGroups * kGroupThreads;   // + producer warp and MMA warp
+constexpr int kStoreWarp0 = 2 + kEpiGroups * kGroupThreads / 32;   // first of the store warps (one per group)
+constexpr int kThreadsTc = 64 + kEpiGroups * (kGroupThreads + 32);   // + producer warp, MMA warp, store warps
+constexpr int kMaxObuf = 4;
 constexpr int kMaxStages = 8;
 constexpr int kProducerLanes = 4;    // lanes of the producer warp that issue TMA copies side by side
 constexpr int kMaxCls = 16;
@@ -112,7 +117,7 @@ __host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, in
     L.addhi_rel = L.sh_rel + BN * 4;
     L.tbl_stride = L.addhi_rel + BN * 4;
     L.bar_off = L.tbl_off + groups * L.tbl_stride;
-    L.total = L.bar_off + (2 * kMaxStages + 4) * 8 + 16;
+    L.total = L.bar_off + (2 * kMaxStages + 4 + 2 * kEpiGroups * kMaxObuf) * 8 + 16;
     return L;
 }
 
@@ -225,7 +230,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t bar_empty = bar_full + 8 * kMaxStages;
     const uint32_t bar_tfull = bar_empty + 8 * kMaxStages;
     const uint32_t bar_tempty = bar_tfull + 16;
-    volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + (2 * kMaxStages + 4) * 8);
+    const uint32_t bar_ofull = bar_tempty + 16;                               // [group][box]: box written
+    const uint32_t bar_oempty = bar_ofull + 8 * kEpiGroups * kMaxObuf;        // [group][box]: box read by its store
+    volatile uint32_t* const tmem_slot =
+        reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + (2 * kMaxStages + 4 + 2 * kEpiGroups * kMaxObuf) * 8);
     volatile uint32_t* const abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -238,6 +246,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_tfull + 8 * i, 1);
             mbar_init(bar_tempty + 8 * i, kGroupThreads / 32);
+        }
+        for (int i = 0; i < kEpiGroups * kMaxObuf; ++i) {
+            mbar_init(bar_ofull + 8 * i, kGroupThreads / 32);
+            mbar_init(bar_oempty + 8 * i, 1);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -358,12 +370,63 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (ok) mma_commit(bar_tfull + 8 * acc);
             }
         }
+    } else if (warp >= kStoreWarp0) {
+        // ------------------------------ output stores ------------------------------
+        // One thread per epilogue group turns filled staging boxes into TMA stores and hands each box
+        // back once its store has read it, so the warps doing arithmetic never wait on a store.
+        const int grp = warp - kStoreWarp0;
+        if (lane == 0 && grp < a.groups && !a.raw) {
+            const uint32_t box_bytes = kTileM * a.out_box;
+            const uint32_t out_addr = base + L.out_off + grp * a.obuf * box_bytes;
+            const uint32_t ofull = bar_ofull + 8 * kMaxObuf * grp, oempty = bar_oempty + 8 * kMaxObuf * grp;
+            const bool lag = a.obuf >= 3;            // release a box one store late: its read is long over by then
+            uint32_t slot = 0, phase = 0, prev_slot = 0;
+            bool have_prev = false, ok = true;
+            for (uint32_t tile = blockIdx.x + grp * gridDim.x; ok && tile < a.num_tiles; tile += a.groups * gridDim.x) {
+                int n_tile;
+                uint32_t m_tile;
+                decode_tile(a, tile, m_tile, n_tile);
+                int w0, h0, b0;
+                tile_origin(a, m_tile, w0, h0, b0);
+                for (int nn = n_tile * a.BN, left = a.BN; left > 0 && nn < a.N; nn += a.out_box, left -= a.out_box) {
+                    if (!mbar_wait(ofull + 8 * slot, phase, a.wait_budget)) {
+                        report_timeout(a.status, QTZ_SITE_OUT_FULL);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    if (a.is4d)
+                        tma_store_4d(&map_y, out_addr + slot * box_bytes, nn, w0, h0, b0);
+                    else
+                        tma_store_2d(&map_y, out_addr + slot * box_bytes, nn, w0);
+                    tma_store_commit();
+                    if (lag) {
+                        if (have_prev) {
+                            tma_store_wait_read_n<1>();
+                            mbar_arrive(oempty + 8 * prev_slot);
+                        }
+                        prev_slot = slot;
+                        have_prev = true;
+                    } else {
+                        tma_store_wait_read();
+                        mbar_arrive(oempty + 8 * slot);
+                    }
+                    if (++slot == static_cast<uint32_t>(a.obuf)) {
+                        slot = 0;
+                        phase ^= 1;
+                    }
+                }
+            }
+            tma_store_wait_all();
+        }
     } else {
         // ------------------------------ epilogue ----------------------------------
         // Two groups of eight warps.  Group g drains accumulator g (every other tile of this CTA), so
-        // the waits, barriers and stores of one group overlap with the arithmetic of the other.  Inside
-        // a group a thread owns one accumulator row (one output pixel); the two warps of a TMEM lane
-        // quarter split the columns of every staging box in halves.
+        // the waits of one group overlap with the arithmetic of the other.  Inside a group a thread owns
+        // one accumulator row (one output pixel); the two warps of a TMEM lane quarter split the columns
+        // of every staging box in halves.  The warps of a group run free of one another: a warp waits
+        // for a staging box to be empty, fills its part and signals the box's barrier; the group's store
+        // thread issues the store once all eight warps have signalled.
         const int et = threadIdx.x - 64;             // 0..511
         const int grp = et >> 8;                     // epilogue group = accumulator index
         const int gt = et & (kGroupThreads - 1);     // thread within the group
@@ -377,20 +440,24 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int32_t* const sh_s = reinterpret_cast<int32_t*>(tbl + L.sh_rel);
         int32_t* const addhi_s = reinterpret_cast<int32_t*>(tbl + L.addhi_rel);
         const uint32_t box_bytes = kTileM * a.out_box;
-        const uint32_t out_rel = L.out_off + grp * a.obuf * box_bytes;               // this group's staging boxes
-        uint32_t slot = 0;                                                           // box written next
+        uint8_t* const out_s = smem + L.out_off + grp * a.obuf * box_bytes;          // this group's staging boxes
+        const uint32_t ofull = bar_ofull + 8 * kMaxObuf * grp, oempty = bar_oempty + 8 * kMaxObuf * grp;
+        uint32_t slot = 0, slot_phase = 0;                                           // box written next
         const int boxes = a.BN / a.out_box;
         const int half_cols = a.out_box >> 1;        // 32 or 64 columns per thread and box
         const int32_t span = a.act_max - a.act_min, off = a.zy - a.act_min;
         const uint32_t lo4 = 0x01010101u * static_cast<uint32_t>(a.act_min);
         const bool fold = a.fold != 0;
         const int mode = fold ? 0 : (a.fast_requant ? 1 : 2);
-        const uint32_t bar_box = 1 + grp, bar_tbl = 3 + grp, bar_vote = 5 + grp;
+        const uint32_t bar_tbl = 1 + grp;
         // this thread's pixel inside a tile never changes
         const int dr_w = a.is4d ? row % a.tw : row;
         const int dr_h = a.is4d ? (row / a.tw) % a.th : 0;
         const int dr_b = a.is4d ? row / (a.tw * a.th) : 0;
         int staged_n_tile = -1;
+        // A warp whose wait ran out stops working but keeps meeting the group at the table barriers,
+        // so that nobody is left alone at one; everything else it would have signalled times out too.
+        bool dead = false;
         // with two groups in use, group g takes every other tile (accumulator g); with one, group 0 takes all
         uint32_t local = grp;
         uint32_t tile = grp < a.groups ? blockIdx.x + grp * gridDim.x : a.num_tiles;
@@ -429,6 +496,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 staged_n_tile = n_tile;
                 named_barrier(bar_tbl, kGroupThreads);       // tables visible to the whole group
             }
+            if (dead) continue;
 
             // which pixel this row is, its border class and its activation-sum term
             int w0, h0, b0;
@@ -454,14 +522,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             const int32_t* const corr_row = corr_s + cls * a.BN;
 
-            // one lane per warp polls; the vote makes the whole group take the same decision, so nobody
-            // is left alone at a barrier
-            bool landed = true;
-            if (lane == 0) landed = mbar_wait(bar_tfull + 8 * acc, acc_phase, a.wait_budget);
-            if (!named_barrier_and(bar_vote, kGroupThreads, landed)) {
-                report_timeout(a.status, QTZ_SITE_TMEM_FULL);
-                *abort_flag = 1;
-                break;
+            // every lane polls the accumulator's barrier; the vote keeps the warp's decision uniform
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, a.wait_budget))) {
+                if (lane == 0) {
+                    report_timeout(a.status, QTZ_SITE_TMEM_FULL);
+                    *abort_flag = 1;
+                }
+                dead = true;
+                continue;
             }
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kAccStride;
@@ -490,10 +558,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int bx = 0; bx < boxes; ++bx) {
                 const int nn = n0 + bx * a.out_box;
                 if (nn >= a.N) break;                // boxes entirely beyond the real channels
-                uint8_t* const dst = smem + out_rel + slot * box_bytes;
-                if (a.obuf == 1) {
-                    if (gt == 0) tma_store_wait_read();  // this group's previous store has read the box
-                    named_barrier(bar_box, kGroupThreads);
+                uint8_t* const dst = out_s + slot * box_bytes;
+                // the store that last used this box has read it
+                if (!__all_sync(0xffffffffu, mbar_wait(oempty + 8 * slot, slot_phase ^ 1, a.wait_budget))) {
+                    if (lane == 0) {
+                        report_timeout(a.status, QTZ_SITE_OUT_EMPTY);
+                        *abort_flag = 1;
+                    }
+                    dead = true;
+                    break;
                 }
                 for (int col = half * half_cols; col < (half + 1) * half_cols && nn + col < a.N; col += 32) {
                     const int j0 = bx * a.out_box + col;
@@ -510,33 +583,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     *reinterpret_cast<uint4*>(dst + swz(row, col, a.out_box)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     *reinterpret_cast<uint4*>(dst + swz(row, col + 16, a.out_box)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
                 }
-                if (bx == boxes - 1 || nn + a.out_box >= a.N) {
-                    // accumulator drained: hand it back to the MMA warp
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+                const bool drained = bx == boxes - 1 || nn + a.out_box >= a.N;
+                if (drained) tc_fence_before();
+                fence_proxy_async_smem();            // this thread's box writes, for the TMA store
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(ofull + 8 * slot);
+                    if (drained) mbar_arrive(bar_tempty + 8 * acc);   // accumulator back to the MMA warp
                 }
-                fence_proxy_async_smem();
-                // With several boxes the barrier below also tells the group that the box written next is
-                // free: the store that last used it is the oldest of the obuf - 1 still allowed to be reading.
-                if (gt == 0) {
-                    if (a.obuf == 2) tma_store_wait_read_n<0>();
-                    else if (a.obuf == 3) tma_store_wait_read_n<1>();
-                    else if (a.obuf >= 4) tma_store_wait_read_n<2>();
+                if (++slot == static_cast<uint32_t>(a.obuf)) {
+                    slot = 0;
+                    slot_phase ^= 1;
                 }
-                named_barrier(bar_box, kGroupThreads);
-                if (gt == 0) {
-                    const uint32_t src = base + out_rel + slot * box_bytes;
-                    if (a.is4d)
-                        tma_store_4d(&map_y, src, nn, w0, h0, b0);
-                    else
-                        tma_store_2d(&map_y, src, nn, w0);
-                    tma_store_commit();
-                }
-                slot = (slot + 1 == static_cast<uint32_t>(a.obuf)) ? 0 : slot + 1;
             }
         }
-        if (gt == 0) tma_store_wait_all();
     }
 
     tc_fence_before();

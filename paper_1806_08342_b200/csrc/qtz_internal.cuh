@@ -31,7 +31,7 @@ enum qtz_kernel_family { QTZ_K_DIRECT = 0, QTZ_K_TCGEN05 = 1, QTZ_K_DEPTHWISE = 
 
 // Device status sites (which bounded wait gave up).
 enum { QTZ_SITE_TMA_FULL = 1, QTZ_SITE_SMEM_EMPTY = 2, QTZ_SITE_TMEM_FULL = 3,
-       QTZ_SITE_TMEM_EMPTY = 4, QTZ_SITE_STORE = 5 };
+       QTZ_SITE_TMEM_EMPTY = 4, QTZ_SITE_STORE = 5, QTZ_SITE_OUT_FULL = 6, QTZ_SITE_OUT_EMPTY = 7 };
 
 inline qtz_status qtz_cuda_fail(qtz_ctx* h, cudaError_t e, const char* what)
 {
