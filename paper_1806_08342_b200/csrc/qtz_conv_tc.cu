@@ -35,14 +35,15 @@ using namespace qtz_ptx;
 namespace {
 
 constexpr int kTileM = 128;          // rows of one accumulator (TMEM lanes)
-constexpr int kAccStride = 256;      // TMEM columns between the two accumulators
+constexpr int kMaxAcc = 4;           // accumulators in TMEM: as many as fit in its 512 columns, at most four
 constexpr int kTmemCols = 512;
-constexpr int kEpiGroups = 2;        // epilogue groups: group g drains accumulator g, so their tiles overlap
+constexpr int kEpiGroups = 2;        // epilogue groups: they take alternate tiles, so their drains overlap
 constexpr int kGroupThreads = 256;   // eight warps per group: two per TMEM lane quarter
 constexpr int kStoreWarp0 = 2 + kEpiGroups * kGroupThreads / 32;   // first of the store warps (one per group)
 constexpr int kThreadsTc = 64 + kEpiGroups * (kGroupThreads + 32);   // + producer warp, MMA warp, store warps
 constexpr int kMaxObuf = 4;
 constexpr int kMaxStages = 8;
+constexpr int kNumBarriers = 2 * kMaxStages + 2 * kMaxAcc + 2 * kEpiGroups * kMaxObuf;
 constexpr int kProducerLanes = 4;    // lanes of the producer warp that issue TMA copies side by side
 constexpr int kMaxCls = 16;
 constexpr int kSmemBudget = 227 * 1024 - 1024;  // leave room for the 1 KB alignment slack
@@ -83,6 +84,7 @@ struct TcArgs {
     int32_t kb_per_tap, c_pad;
     int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
     int32_t obuf;                           // staging boxes per epilogue group (1..4)
+    int32_t n_acc, acc_stride;              // accumulators in TMEM and the columns between them
     uint32_t idesc;
     const int32_t* bias;
     const int32_t* wsum;                    // [ncls][N]
@@ -117,7 +119,7 @@ __host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, in
     L.addhi_rel = L.sh_rel + BN * 4;
     L.tbl_stride = L.addhi_rel + BN * 4;
     L.bar_off = L.tbl_off + groups * L.tbl_stride;
-    L.total = L.bar_off + (2 * kMaxStages + 4 + 2 * kEpiGroups * kMaxObuf) * 8 + 16;
+    L.total = L.bar_off + kNumBarriers * 8 + 16;
     return L;
 }
 
@@ -229,11 +231,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t bar_full = base + L.bar_off;
     const uint32_t bar_empty = bar_full + 8 * kMaxStages;
     const uint32_t bar_tfull = bar_empty + 8 * kMaxStages;
-    const uint32_t bar_tempty = bar_tfull + 16;
-    const uint32_t bar_ofull = bar_tempty + 16;                               // [group][box]: box written
+    const uint32_t bar_tempty = bar_tfull + 8 * kMaxAcc;
+    const uint32_t bar_ofull = bar_tempty + 8 * kMaxAcc;                               // [group][box]: box written
     const uint32_t bar_oempty = bar_ofull + 8 * kEpiGroups * kMaxObuf;        // [group][box]: box read by its store
     volatile uint32_t* const tmem_slot =
-        reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + (2 * kMaxStages + 4 + 2 * kEpiGroups * kMaxObuf) * 8);
+        reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + kNumBarriers * 8);
     volatile uint32_t* const abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -243,7 +245,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kMaxAcc; ++i) {
             mbar_init(bar_tfull + 8 * i, 1);
             mbar_init(bar_tempty + 8 * i, kGroupThreads / 32);
         }
@@ -293,7 +295,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const uint32_t g = issued_before + static_cast<uint32_t>(kbl);
                     const uint32_t round = g / nstages, stage = g - round * nstages, phase = round & 1;
                     const int tap = kbl / a.kb_per_tap, kb = kbl - tap * a.kb_per_tap;
-                    if (mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget)) {
+                    if (mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget, 64u)) {
                         mbar_arrive_expect_tx(bar_full + 8 * stage, tx);
                         const uint32_t dst_a = base + L.a_off + stage * L.a_stage;
                         const uint32_t dst_b = base + L.b_off + stage * L.b_stage;
@@ -336,20 +338,19 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t a_step = L.a_stage >> 4, b_step = L.b_stage >> 4;   // descriptor address units
             const int mmas = a.BK / 32;          // each MMA consumes 32 bytes of K: advance 2 x 16 B
             uint32_t stage = 0, phase = 0;
-            uint32_t local = 0;
+            uint32_t acc = 0, acc_phase = 0;     // accumulators are used round robin
             bool ok = true;
             bool ready = mbar_try_wait(bar_full, 0);
-            for (uint32_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x, ++local) {
-                const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
-                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget)) {
+            for (uint32_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget, 128u)) {
                     report_timeout(a.status, QTZ_SITE_TMEM_EMPTY);
                     *abort_flag = 1;
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * kAccStride;
+                const uint32_t d_tmem = tmem_base + acc * a.acc_stride;
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!ready && !mbar_wait(bar_full + 8 * stage, phase, a.wait_budget)) {
+                    if (!ready && !mbar_wait(bar_full + 8 * stage, phase, a.wait_budget, 64u)) {
                         report_timeout(a.status, QTZ_SITE_TMA_FULL);
                         *abort_flag = 1;
                         ok = false;
@@ -368,6 +369,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     mma_commit(freed);           // frees the stage once these MMAs have read it
                 }
                 if (ok) mma_commit(bar_tfull + 8 * acc);
+                if (++acc == static_cast<uint32_t>(a.n_acc)) {
+                    acc = 0;
+                    acc_phase ^= 1;
+                }
             }
         }
     } else if (warp >= kStoreWarp0) {
@@ -389,7 +394,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 int w0, h0, b0;
                 tile_origin(a, m_tile, w0, h0, b0);
                 for (int nn = n_tile * a.BN, left = a.BN; left > 0 && nn < a.N; nn += a.out_box, left -= a.out_box) {
-                    if (!mbar_wait(ofull + 8 * slot, phase, a.wait_budget)) {
+                    if (!mbar_wait(ofull + 8 * slot, phase, a.wait_budget, 128u)) {
                         report_timeout(a.status, QTZ_SITE_OUT_FULL);
                         *abort_flag = 1;
                         ok = false;
@@ -443,7 +448,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint8_t* const out_s = smem + L.out_off + grp * a.obuf * box_bytes;          // this group's staging boxes
         const uint32_t ofull = bar_ofull + 8 * kMaxObuf * grp, oempty = bar_oempty + 8 * kMaxObuf * grp;
         uint32_t slot = 0, slot_phase = 0;                                           // box written next
-        const int boxes = a.BN / a.out_box;
+        const int boxes = (a.BN + a.out_box - 1) / a.out_box;
         const int half_cols = a.out_box >> 1;        // 32 or 64 columns per thread and box
         const int32_t span = a.act_max - a.act_min, off = a.zy - a.act_min;
         const uint32_t lo4 = 0x01010101u * static_cast<uint32_t>(a.act_min);
@@ -459,10 +464,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // so that nobody is left alone at one; everything else it would have signalled times out too.
         bool dead = false;
         // with two groups in use, group g takes every other tile (accumulator g); with one, group 0 takes all
-        uint32_t local = grp;
+        // the CTA's i-th tile lives in accumulator i mod n_acc
+        uint32_t next_acc = grp % a.n_acc, next_acc_phase = (grp / a.n_acc) & 1;
         uint32_t tile = grp < a.groups ? blockIdx.x + grp * gridDim.x : a.num_tiles;
-        for (; tile < a.num_tiles; tile += a.groups * gridDim.x, local += a.groups) {
-            const uint32_t acc = local & 1, acc_phase = (local >> 1) & 1;
+        for (; tile < a.num_tiles; tile += a.groups * gridDim.x) {
+            const uint32_t acc = next_acc, acc_phase = next_acc_phase;
+            next_acc += a.groups;
+            while (next_acc >= static_cast<uint32_t>(a.n_acc)) {
+                next_acc -= a.n_acc;
+                next_acc_phase ^= 1;
+            }
             int n_tile;
             uint32_t m_tile;
             decode_tile(a, tile, m_tile, n_tile);
@@ -523,7 +534,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int32_t* const corr_row = corr_s + cls * a.BN;
 
             // every lane polls the accumulator's barrier; the vote keeps the warp's decision uniform
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, a.wait_budget))) {
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * acc, acc_phase, a.wait_budget, 128u))) {
                 if (lane == 0) {
                     report_timeout(a.status, QTZ_SITE_TMEM_FULL);
                     *abort_flag = 1;
@@ -532,7 +543,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 continue;
             }
             tc_fence_after();
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kAccStride;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * a.acc_stride;
 
             if (a.raw) {
                 // int32 accumulators with the cross terms applied; the two warps of a quarter alternate 32-column chunks
@@ -560,7 +571,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (nn >= a.N) break;                // boxes entirely beyond the real channels
                 uint8_t* const dst = out_s + slot * box_bytes;
                 // the store that last used this box has read it
-                if (!__all_sync(0xffffffffu, mbar_wait(oempty + 8 * slot, slot_phase ^ 1, a.wait_budget))) {
+                if (!__all_sync(0xffffffffu, mbar_wait(oempty + 8 * slot, slot_phase ^ 1, a.wait_budget, 64u))) {
                     if (lane == 0) {
                         report_timeout(a.status, QTZ_SITE_OUT_EMPTY);
                         *abort_flag = 1;
@@ -900,8 +911,13 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.kb_per_tap = a.c_pad / a.BK;
     // N tiling: as few tiles as possible, each a multiple of 32 columns
     a.n_tiles = (d.n + 255) / 256;
-    a.BN = ((d.n + a.n_tiles - 1) / a.n_tiles + 63) / 64 * 64;
+    // (one tile: 32-column granularity, the TMA store clips what lies beyond the real channels;
+    //  several tiles: whole staging boxes, since a box must not spill into the next tile's columns)
+    a.BN = a.n_tiles == 1 ? (d.n + 31) / 32 * 32 : ((d.n + a.n_tiles - 1) / a.n_tiles + 63) / 64 * 64;
     a.out_box = (a.BN % 128 == 0) ? 128 : 64;
+    // every accumulator a tile ahead lets the MMA warp start a tile before an epilogue group is back
+    a.n_acc = std::min(kMaxAcc, kTmemCols / a.BN);
+    a.acc_stride = a.BN;
     t->n_pad = a.n_tiles * a.BN;
     a.ncls = pw ? 1 : kMaxCls;
 

@@ -47,29 +47,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return done != 0;
 }
 
-// Same test, but the hardware may park the thread for up to `hint_ns` nanoseconds while the phase is
-// still open; it resumes as soon as the phase completes.
-__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t hint_ns)
-{
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(bar), "r"(parity), "r"(hint_ns)
-        : "memory");
-    return done != 0;
-}
-
-// Waits for the phase with the given parity to complete; gives up after `budget` cycles.  The
-// waiting thread is parked by the barrier unit between polls, so a long wait costs few issue slots.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long budget)
+// Waits for the phase with the given parity to complete; gives up after `budget` cycles.  Between
+// polls the warp sleeps, for 32 ns at first and then twice as long each time up to `max_sleep_ns`,
+// so a long wait leaves the issue slots to the warps that have work; the cycle budget is looked at
+// on every eighth poll.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long budget, uint32_t max_sleep_ns = 32u)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
-    while (!mbar_try_wait_parked(bar, parity, 4000u)) {
-        if (clock64() - start > budget) return false;
+    uint32_t ns = 32u, polls = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++polls & 7u) == 0 && clock64() - start > budget) return false;
+        __nanosleep(ns);
+        if (ns < max_sleep_ns) ns <<= 1;
     }
     return true;
 }
