@@ -44,7 +44,6 @@ constexpr int kThreadsTc = 64 + kEpiGroups * (kGroupThreads + 32);   // + produc
 constexpr int kMaxObuf = 4;
 constexpr int kMaxStages = 8;
 constexpr int kNumBarriers = 2 * kMaxStages + 2 * kMaxAcc + 2 * kEpiGroups * kMaxObuf;
-constexpr int kProducerLanes = 4;    // lanes of the producer warp that issue TMA copies side by side
 constexpr int kMaxCls = 16;
 constexpr int kSmemBudget = 227 * 1024 - 1024;  // leave room for the 1 KB alignment slack
 
@@ -73,7 +72,7 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f)
 }
 
 struct TcArgs {
-    FastDiv dv_per_group, dv_group_m, dv_group_last, dv_tiles_w, dv_tiles_h;
+    FastDiv dv_per_group, dv_group_m, dv_group_last, dv_tiles_w, dv_tiles_h, dv_kb_per_tap, dv_kw;
     int32_t is4d;
     int32_t tw, th, tb, rows;               // pixel box of one tile and its row count (<= 128)
     int32_t tiles_w, tiles_h, n_tiles;
@@ -195,6 +194,11 @@ __device__ __forceinline__ void requant32(const uint32_t (&v)[32], const int32_t
 // that together fit in L2.
 __device__ __forceinline__ void decode_tile(const TcArgs& a, uint32_t tile, uint32_t& m_tile, int& n_tile)
 {
+    if (a.n_tiles == 1) {                   // the usual case for a convolution layer: one column tile
+        m_tile = tile;
+        n_tile = 0;
+        return;
+    }
     const uint32_t g = fdiv(tile, a.dv_per_group), r = tile - g * a.dv_per_group.d;
     const uint32_t m_first = g * static_cast<uint32_t>(a.group_m);
     const bool last = static_cast<uint32_t>(a.m_tiles) - m_first < static_cast<uint32_t>(a.group_m);   // a shorter final group
@@ -272,55 +276,60 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
-        // A single thread issuing one K block at a time spends several hundred cycles per block on
-        // its own dependent instructions (barrier poll, address arithmetic, two TMA issues).  Up to
-        // kProducerLanes lanes therefore run the loop in lockstep, lane l taking K blocks l, l+P, ...
-        // of the tile; every lane waits on and arms the barrier of its own stage.
-        const int P = min(min(kblocks, kProducerLanes), a.stages);   // never two lanes on one stage at a time
+        // The K blocks of all tiles of this CTA form one sequence; block g goes to ring stage g mod
+        // stages.  A single thread working through that sequence spends well over a thousand cycles per
+        // block on its own dependent instructions (tile decode, barrier poll, two TMA issues), which
+        // starves layers with a short reduction.  So one lane per stage runs the loop: lane l owns
+        // stage l and takes blocks l, l + stages, ...; a lane waits only on its own stage's barrier.
+        const uint32_t S = static_cast<uint32_t>(a.stages);
+        const uint32_t kbs = static_cast<uint32_t>(kblocks);
         const uint32_t tx = static_cast<uint32_t>(a.rows * a.BK + a.BN * a.BK);
-        const uint32_t nstages = static_cast<uint32_t>(a.stages);
-        uint32_t issued_before = 0;          // K blocks of earlier tiles
-        uint32_t last_stage = 0, last_phase = 0;
+        const uint32_t adv_t = S / kbs, adv_kb = S - adv_t * kbs;      // one trip moves every lane S blocks on
+        uint32_t t = static_cast<uint32_t>(lane) / kbs;                 // tile ordinal within this CTA
+        uint32_t kb = static_cast<uint32_t>(lane) - t * kbs;            // K block within the tile
+        const uint32_t stage = static_cast<uint32_t>(lane);
+        const uint32_t full = bar_full + 8 * stage, empty = bar_empty + 8 * stage;
+        const uint32_t dst_a = base + L.a_off + stage * L.a_stage;
+        const uint32_t dst_b = base + L.b_off + stage * L.b_stage;
+        uint32_t phase = 0;
         bool issued_any = false, failed = false;
-        for (uint32_t tile = blockIdx.x; tile < a.num_tiles; tile += gridDim.x) {
-            int n_tile;
-            uint32_t m_tile;
-            decode_tile(a, tile, m_tile, n_tile);
-            int w0, h0, b0;
-            tile_origin(a, m_tile, w0, h0, b0);
-            for (int kb0 = 0; kb0 < kblocks; kb0 += P) {
-                const int kbl = kb0 + lane;
-                const bool active = lane < P && kbl < kblocks;
-                if (active) {
-                    const uint32_t g = issued_before + static_cast<uint32_t>(kbl);
-                    const uint32_t round = g / nstages, stage = g - round * nstages, phase = round & 1;
-                    const int tap = kbl / a.kb_per_tap, kb = kbl - tap * a.kb_per_tap;
-                    if (mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget, 64u)) {
-                        mbar_arrive_expect_tx(bar_full + 8 * stage, tx);
-                        const uint32_t dst_a = base + L.a_off + stage * L.a_stage;
-                        const uint32_t dst_b = base + L.b_off + stage * L.b_stage;
-                        if (a.is4d) {
-                            const int ty = tap / a.kw;
-                            tma_load_4d(dst_a, &map_a, bar_full + 8 * stage, kb * a.BK, w0 + (tap - ty * a.kw) - a.pad,
-                                        h0 + ty - a.pad, b0);
-                        } else {
-                            tma_load_2d(dst_a, &map_a, bar_full + 8 * stage, kb * a.BK, w0);
-                        }
-                        tma_load_2d(dst_b, &map_b, bar_full + 8 * stage, tap * a.c_pad + kb * a.BK, n_tile * a.BN);
-                        last_stage = stage;
-                        last_phase = phase;
-                        issued_any = true;
+        for (;;) {
+            const uint64_t tile64 = blockIdx.x + static_cast<uint64_t>(t) * gridDim.x;
+            const bool active = static_cast<uint32_t>(lane) < S && tile64 < a.num_tiles;
+            if (active) {
+                int n_tile, w0, h0, b0;
+                uint32_t m_tile;
+                decode_tile(a, static_cast<uint32_t>(tile64), m_tile, n_tile);
+                tile_origin(a, m_tile, w0, h0, b0);
+                const uint32_t tap = fdiv(kb, a.dv_kb_per_tap);
+                const int kc = static_cast<int>(kb - tap * a.dv_kb_per_tap.d) * a.BK;    // channel offset inside the tap
+                if (mbar_wait(empty, phase ^ 1, a.wait_budget, 64u)) {
+                    mbar_arrive_expect_tx(full, tx);
+                    if (a.is4d) {
+                        const uint32_t ty = fdiv(tap, a.dv_kw);
+                        tma_load_4d(dst_a, &map_a, full, kc, w0 + static_cast<int>(tap - ty * a.dv_kw.d) - a.pad,
+                                    h0 + static_cast<int>(ty) - a.pad, b0);
                     } else {
-                        failed = true;
+                        tma_load_2d(dst_a, &map_a, full, kc, w0);
                     }
-                }
-                if (__any_sync(0xffffffffu, failed || *abort_flag != 0)) {
+                    tma_load_2d(dst_b, &map_b, full, static_cast<int>(tap) * a.c_pad + kc, n_tile * a.BN);
+                    issued_any = true;
+                } else {
                     failed = true;
-                    break;
                 }
             }
-            if (failed) break;
-            issued_before += static_cast<uint32_t>(kblocks);
+            if (__ballot_sync(0xffffffffu, failed || (lane == 0 && *abort_flag != 0)) != 0u) {
+                failed = true;
+                break;
+            }
+            if (!__any_sync(0xffffffffu, active)) break;      // lane 0 holds the earliest block: nothing left
+            t += adv_t;
+            kb += adv_kb;
+            if (kb >= kbs) {
+                kb -= kbs;
+                ++t;
+            }
+            phase ^= 1;
         }
         if (failed) {
             if (lane == 0) {
@@ -328,7 +337,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 *abort_flag = 1;
             }
             // drain: give this lane's last copy a bounded time to land before the CTA exits
-            if (issued_any) (void)mbar_wait(bar_full + 8 * last_stage, last_phase, a.wait_budget);
+            if (issued_any) (void)mbar_wait(full, phase, a.wait_budget);
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer --------------------------------
@@ -966,6 +975,8 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.dv_group_last = make_fastdiv(static_cast<uint32_t>(std::max(1, a.m_tiles % a.group_m)));
     a.dv_tiles_w = make_fastdiv(static_cast<uint32_t>(a.tiles_w));
     a.dv_tiles_h = make_fastdiv(static_cast<uint32_t>(std::max(1, a.tiles_h)));
+    a.dv_kb_per_tap = make_fastdiv(static_cast<uint32_t>(a.kb_per_tap));
+    a.dv_kw = make_fastdiv(static_cast<uint32_t>(a.kw));
     // shared-memory budget -> pipeline depth
     // worst case (all border classes) for the smem opt-in; every launch picks its own depth
     a.groups = kEpiGroups;
