@@ -237,10 +237,13 @@ def time_hbm_kernels(hq, qtz, torch, peaks):
 
 
 def time_layer(hq, qtz, torch, spec, reps=20):
-    """One convolution layer alone: spec = "batch,h,w,c,n,k,stride[,dw]" (profiling runs)."""
+    """One convolution layer alone: spec = "batch,h,w,c,n,k,stride[,dw][,full]" (profiling runs).
+    "full" = the zero points and clamp of a layer between two ReLU6 tensors (z_x = z_y = 0, clamp to
+    [0,255]); without it z_x = 7, z_y = 20 and the clamp is [20,255]."""
     v = spec.split(",")
     b, hh, ww, c, n, k, st = (int(x) for x in v[:7])
-    dw = len(v) > 7 and v[7] == "dw"
+    dw = "dw" in v[7:]
+    zargs = (0, 0, 0, 255) if "full" in v[7:] else (7, 20, 20, 255)
     pad = k // 2
     x = torch.randint(0, 256, (b, hh, ww, (c + 15) // 16 * 16), dtype=torch.uint8, device="cuda")
     w = torch.randint(-127, 128, (k, k, c) if dw else (n, k, k, c), dtype=torch.int8, device="cuda")
@@ -249,12 +252,12 @@ def time_layer(hq, qtz, torch, spec, reps=20):
                           np.full(n, r, np.int32), depthwise=dw)
     y = plan.empty_output("cuda")
     for _ in range(3):
-        plan(x, 7, 20, 20, 255, out=y)
+        plan(x, *zargs, out=y)
     torch.cuda.synchronize()
     s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s.record()
     for _ in range(reps):
-        plan(x, 7, 20, 20, 255, out=y)
+        plan(x, *zargs, out=y)
     e.record(); torch.cuda.synchronize()
     ms = s.elapsed_time(e) / reps
     oh, ow = plan.oh, plan.ow

@@ -147,7 +147,7 @@ __device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t col, uint32_t box
 //   kMode 0 (folded):  y - act_min = hi32(acc m + A) >> (r - 32), A = corr m + 2^(r-1) + (z_y - act_min) 2^r
 //   kMode 1 (general): the correction (border class, activation sums) is added to acc first
 //   kMode 2 (any shift): 64-bit shift and clamp
-template <int kMode>
+template <int kMode, bool kFullRange>
 __device__ __forceinline__ void requant32(const uint32_t (&v)[32], const int32_t* __restrict__ mult_s,
                                           const int32_t* __restrict__ sh_s, const int64_t* __restrict__ add64_s,
                                           const int32_t* __restrict__ corr_row, const int32_t* __restrict__ addhi_s,
@@ -166,7 +166,8 @@ __device__ __forceinline__ void requant32(const uint32_t (&v)[32], const int32_t
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int64_t prod = static_cast<int64_t>(static_cast<int32_t>(v[4 * q + e])) * mm[e] + aa[e];
-                y[e] = __vimin_s32_relu(static_cast<int32_t>(prod >> 32) >> ss[e], span);
+                const int32_t t = static_cast<int32_t>(prod >> 32) >> ss[e];
+                y[e] = kFullRange ? t : __vimin_s32_relu(t, span);     // [0,255]: the saturating pack clamps
             }
         } else {
             const int4 c4 = *reinterpret_cast<const int4*>(corr_row + 4 * q);
@@ -177,7 +178,8 @@ __device__ __forceinline__ void requant32(const uint32_t (&v)[32], const int32_t
                 const int32_t full = static_cast<int32_t>(v[4 * q + e]) + cc[e] + rowterm;
                 if (kMode == 1) {
                     const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(hh[e]) << 32);
-                    y[e] = __vimin_s32_relu(static_cast<int32_t>(prod >> 32) >> ss[e], span);
+                    const int32_t t = static_cast<int32_t>(prod >> 32) >> ss[e];
+                    y[e] = kFullRange ? t : __vimin_s32_relu(t, span);
                 } else {
                     const int64_t prod = static_cast<int64_t>(full) * mm[e] + (static_cast<int64_t>(1) << (ss[e] - 1));
                     const int64_t sh = (prod >> ss[e]) + off;
@@ -185,7 +187,7 @@ __device__ __forceinline__ void requant32(const uint32_t (&v)[32], const int32_t
                 }
             }
         }
-        packed[q] = pack_sat_u8(y[1], y[0], pack_sat_u8(y[3], y[2], 0u)) + lo4;
+        packed[q] = pack_sat_u8(y[1], y[0], pack_sat_u8(y[3], y[2], 0u)) + (kFullRange ? 0u : lo4);
     }
 }
 
@@ -463,6 +465,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t lo4 = 0x01010101u * static_cast<uint32_t>(a.act_min);
         const bool fold = a.fold != 0;
         const int mode = fold ? 0 : (a.fast_requant ? 1 : 2);
+        const bool full_range = a.act_min == 0 && a.act_max == 255;   // then saturation to a byte is the whole clamp
         const uint32_t bar_tbl = 1 + grp;
         // this thread's pixel inside a tile never changes
         const int dr_w = a.is4d ? row % a.tw : row;
@@ -594,12 +597,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     tmem_ld_32x32(taddr + j0, v);
                     tmem_ld_wait();
                     uint32_t packed[8];
-                    if (mode == 0)
-                        requant32<0>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
+                    if (mode == 0 && full_range)
+                        requant32<0, true>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
+                    else if (mode == 0)
+                        requant32<0, false>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
+                    else if (mode == 1 && full_range)
+                        requant32<1, true>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
                     else if (mode == 1)
-                        requant32<1>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
+                        requant32<1, false>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
                     else
-                        requant32<2>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
+                        requant32<2, false>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
                     *reinterpret_cast<uint4*>(dst + swz(row, col, a.out_box)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     *reinterpret_cast<uint4*>(dst + swz(row, col + 16, a.out_box)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
                 }
