@@ -35,12 +35,12 @@ using namespace qtz_ptx;
 namespace {
 
 constexpr int kTileM = 128;          // rows of one accumulator (TMEM lanes)
-constexpr int kMaxAcc = 4;           // accumulators in TMEM: as many as fit in its 512 columns, at most four
+constexpr int kMaxAcc = 8;           // accumulators in TMEM: as many as fit in its 512 columns, at most eight
 constexpr int kTmemCols = 512;
-constexpr int kEpiGroups = 2;        // epilogue groups: they take alternate tiles, so their drains overlap
-constexpr int kGroupThreads = 256;   // eight warps per group: two per TMEM lane quarter
-constexpr int kStoreWarp0 = 2 + kEpiGroups * kGroupThreads / 32;   // first of the store warps (one per group)
-constexpr int kThreadsTc = 64 + kEpiGroups * (kGroupThreads + 32);   // + producer warp, MMA warp, store warps
+constexpr int kEpiWarps = 16;        // epilogue warps: four groups of four or two groups of eight
+constexpr int kEpiGroups = 4;        // most epilogue groups; the groups take tiles in turn, so their drains overlap
+constexpr int kStoreWarp = 2 + kEpiWarps;            // its lane g issues the output stores of group g
+constexpr int kThreadsTc = 32 * (kStoreWarp + 1);    // producer warp, MMA warp, epilogue warps, store warp
 constexpr int kMaxObuf = 4;
 constexpr int kMaxStages = 8;
 constexpr int kNumBarriers = 2 * kMaxStages + 2 * kMaxAcc + 2 * kEpiGroups * kMaxObuf;
@@ -84,6 +84,7 @@ struct TcArgs {
     int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
     int32_t obuf;                           // staging boxes per epilogue group (1..4)
     int32_t n_acc, acc_stride;              // accumulators in TMEM and the columns between them
+    int32_t gwarps;                         // warps per epilogue group: 4 (up to four groups) or 8 (up to two)
     uint32_t idesc;
     const int32_t* bias;
     const int32_t* wsum;                    // [ncls][N]
@@ -253,10 +254,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int i = 0; i < kMaxAcc; ++i) {
             mbar_init(bar_tfull + 8 * i, 1);
-            mbar_init(bar_tempty + 8 * i, kGroupThreads / 32);
+            mbar_init(bar_tempty + 8 * i, a.gwarps);
         }
         for (int i = 0; i < kEpiGroups * kMaxObuf; ++i) {
-            mbar_init(bar_ofull + 8 * i, kGroupThreads / 32);
+            mbar_init(bar_ofull + 8 * i, a.gwarps);
             mbar_init(bar_oempty + 8 * i, 1);
         }
         *abort_flag = 0;
@@ -386,12 +387,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
             }
         }
-    } else if (warp >= kStoreWarp0) {
+    } else if (warp == kStoreWarp) {
         // ------------------------------ output stores ------------------------------
-        // One thread per epilogue group turns filled staging boxes into TMA stores and hands each box
+        // One lane per epilogue group turns filled staging boxes into TMA stores and hands each box
         // back once its store has read it, so the warps doing arithmetic never wait on a store.
-        const int grp = warp - kStoreWarp0;
-        if (lane == 0 && grp < a.groups && !a.raw) {
+        const int grp = lane;
+        if (grp < a.groups && !a.raw) {
             const uint32_t box_bytes = kTileM * a.out_box;
             const uint32_t out_addr = base + L.out_off + grp * a.obuf * box_bytes;
             const uint32_t ofull = bar_ofull + 8 * kMaxObuf * grp, oempty = bar_oempty + 8 * kMaxObuf * grp;
@@ -437,17 +438,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         // ------------------------------ epilogue ----------------------------------
-        // Two groups of eight warps.  Group g drains accumulator g (every other tile of this CTA), so
-        // the waits of one group overlap with the arithmetic of the other.  Inside a group a thread owns
-        // one accumulator row (one output pixel); the two warps of a TMEM lane quarter split the columns
-        // of every staging box in halves.  The warps of a group run free of one another: a warp waits
-        // for a staging box to be empty, fills its part and signals the box's barrier; the group's store
-        // thread issues the store once all eight warps have signalled.
+        // Sixteen warps as four groups of four (narrow tiles: more work per warp and tile, so the per-tile
+        // bookkeeping weighs less) or two groups of eight.  The groups take this CTA's tiles in turn, so
+        // the waits of one overlap with the arithmetic of the others.  Inside a group a thread owns one
+        // accumulator row (one output pixel); with eight warps the two warps of a TMEM lane quarter split
+        // the columns of every staging box in halves.  The warps of a group run free of one another: a
+        // warp waits for a staging box to be empty, fills its part and signals the box's barrier; the
+        // group's store lane issues the store once all warps of the group have signalled.
         const int et = threadIdx.x - 64;             // 0..511
-        const int grp = et >> 8;                     // epilogue group = accumulator index
-        const int gt = et & (kGroupThreads - 1);     // thread within the group
+        const int gthreads = 32 * a.gwarps;          // 128 or 256 threads per group
+        const int grp = et / gthreads;
+        const int gt = et - grp * gthreads;          // thread within the group
         const int quarter = warp & 3;                // TMEM lane quarter this warp may read
-        const int half = ((warp - 2) >> 2) & 1;      // which half of a box's columns
+        const int halves = a.gwarps >> 2;            // warps sharing a quarter split every box's columns between them
+        const int half = (gt >> 7) & (halves - 1);
         const int row = quarter * 32 + lane;         // accumulator row owned by this thread
         uint8_t* const tbl = smem + L.tbl_off + grp * L.tbl_stride;
         int32_t* const corr_s = reinterpret_cast<int32_t*>(tbl);                     // [ncls][BN] (general form)
@@ -460,7 +464,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t ofull = bar_ofull + 8 * kMaxObuf * grp, oempty = bar_oempty + 8 * kMaxObuf * grp;
         uint32_t slot = 0, slot_phase = 0;                                           // box written next
         const int boxes = (a.BN + a.out_box - 1) / a.out_box;
-        const int half_cols = a.out_box >> 1;        // 32 or 64 columns per thread and box
+        const int half_cols = a.out_box / halves;    // 32, 64 or 128 columns per thread and box
         const int32_t span = a.act_max - a.act_min, off = a.zy - a.act_min;
         const uint32_t lo4 = 0x01010101u * static_cast<uint32_t>(a.act_min);
         const bool fold = a.fold != 0;
@@ -494,8 +498,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (n_tile != staged_n_tile) {
                 // per-channel constants of this column tile: cross-term correction (Eq. 5-6), multiplier,
                 // shift, and the rounding constant with the output offset folded in
-                named_barrier(bar_tbl, kGroupThreads);       // everyone is done with the old tables
-                for (int j = gt; j < a.BN; j += kGroupThreads) {
+                named_barrier(bar_tbl, gthreads);            // everyone is done with the old tables
+                for (int j = gt; j < a.BN; j += gthreads) {
                     const int n = n0 + j;
                     const bool live = n < a.N;
                     const int32_t bias = live ? __ldg(a.bias + n) : 0;
@@ -517,7 +521,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                 }
                 staged_n_tile = n_tile;
-                named_barrier(bar_tbl, kGroupThreads);       // tables visible to the whole group
+                named_barrier(bar_tbl, gthreads);            // tables visible to the whole group
             }
             if (dead) continue;
 
@@ -559,7 +563,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
             if (a.raw) {
                 // int32 accumulators with the cross terms applied; the two warps of a quarter alternate 32-column chunks
-                for (int j0 = 32 * half; j0 < a.BN && n0 + j0 < a.N; j0 += 64) {
+                for (int j0 = 32 * half; j0 < a.BN && n0 + j0 < a.N; j0 += 32 * halves) {
                     uint32_t v[32];
                     tmem_ld_32x32(taddr + j0, v);
                     tmem_ld_wait();
@@ -986,7 +990,9 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.dv_kw = make_fastdiv(static_cast<uint32_t>(a.kw));
     // shared-memory budget -> pipeline depth
     // worst case (all border classes) for the smem opt-in; every launch picks its own depth
-    a.groups = kEpiGroups;
+    a.groups = 1;
+    a.gwarps = 8;
+    a.obuf = 1;
     a.stages = 2;
     if (make_layout(a.BK, a.BN, 2, a.ncls, a.out_box, 1, 1).total > static_cast<uint32_t>(kSmemBudget)) return QTZ_ERR_UNSUPPORTED;
 
@@ -1112,9 +1118,9 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     // with z_x = 0 the cross-term correction no longer depends on the border class: one class, small tables
     if (x_zp == 0) a.ncls = 1;
     // Shared memory is split between the operand ring, the epilogue groups and their staging boxes.
-    // Preference: two groups (overlapped tile drains) with two or three boxes each (the store of one box
+    // Preference: many groups (overlapped tile drains) with two or three boxes each (the store of one box
     // overlaps the arithmetic of the next), as long as the ring keeps four stages, or the whole
-    // reduction plus one block when that is shorter.
+    // reduction plus one block when that is shorter.  Four groups need four accumulators in TMEM.
     auto depth = [&](int groups, int obuf) {
         int st_ = kMaxStages;
         for (; st_ >= 2; --st_)
@@ -1123,10 +1129,11 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     };
     const int kblocks = a.taps * a.kb_per_tap;
     const int need = std::min(4, kblocks + 1);
-    static const int choice[5][2] = {{2, 3}, {2, 2}, {1, 2}, {2, 1}, {1, 1}};
+    static const int choice[7][2] = {{4, 3}, {4, 2}, {2, 3}, {2, 2}, {1, 2}, {2, 1}, {1, 1}};
     a.groups = 1;
     a.obuf = 1;
     for (const auto& c : choice) {
+        if (c[0] == 4 && a.n_acc < 4) continue;
         const int ob = a.raw ? 1 : c[1];             // the boxes rotate across tiles as well
         if (depth(c[0], ob) >= need) {
             a.groups = c[0];
@@ -1134,6 +1141,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
             break;
         }
     }
+    a.gwarps = a.groups == 4 ? 4 : 8;
     a.stages = depth(a.groups, a.obuf);
     if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
     const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf).total + 1024;
