@@ -40,7 +40,8 @@ constexpr int kTmemCols = 512;
 constexpr int kEpiWarps = 16;        // epilogue warps: four groups of four or two groups of eight
 constexpr int kEpiGroups = 4;        // most epilogue groups; the groups take tiles in turn, so their drains overlap
 constexpr int kStoreWarp = 2 + kEpiWarps;            // its lane g issues the output stores of group g
-constexpr int kThreadsTc = 32 * (kStoreWarp + 1);    // producer warp, MMA warp, epilogue warps, store warp
+constexpr int kMmaWarp2 = kStoreWarp + 1;            // second MMA-issuing warp (short reductions)
+constexpr int kThreadsTc = 32 * (kMmaWarp2 + 1);     // producer warp, MMA warp, epilogue warps, store warp, MMA warp
 constexpr int kMaxObuf = 4;
 constexpr int kMaxStages = 8;
 constexpr int kNumBarriers = 2 * kMaxStages + 2 * kMaxAcc + 2 * kEpiGroups * kMaxObuf;
@@ -85,6 +86,7 @@ struct TcArgs {
     int32_t obuf;                           // staging boxes per epilogue group (1..4)
     int32_t n_acc, acc_stride;              // accumulators in TMEM and the columns between them
     int32_t gwarps;                         // warps per epilogue group: 4 (up to four groups) or 8 (up to two)
+    int32_t mma_lanes;                      // MMA-issuing threads (1 or 2, each in its own warp)
     uint32_t idesc;
     const int32_t* bias;
     const int32_t* wsum;                    // [ncls][N]
@@ -342,18 +344,28 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // drain: give this lane's last copy a bounded time to land before the CTA exits
             if (issued_any) (void)mbar_wait(full, phase, a.wait_budget);
         }
-    } else if (warp == 1) {
-        // ------------------------------ MMA issuer --------------------------------
-        if (lane == 0) {
+    } else if (warp == 1 || warp == kMmaWarp2) {
+        // ------------------------------ MMA issuers -------------------------------
+        // One thread issues all MMAs of a tile.  With a short reduction its own dependent instructions
+        // (two barrier polls, descriptors, one or two MMAs, two commits) take longer per tile than the
+        // tensor core does, so when two whole tiles fit in the operand ring a second issuing thread, in a
+        // warp of its own, takes every other tile; every tile still has one issuing thread and its own
+        // accumulator.
+        const uint32_t P = static_cast<uint32_t>(a.mma_lanes);
+        const uint32_t me = warp == 1 ? 0u : 1u;
+        if (lane == 0 && me < P) {
             const uint64_t desc_a0 = make_kmajor_desc(base + L.a_off, a.BK);
             const uint64_t desc_b0 = make_kmajor_desc(base + L.b_off, a.BK);
             const uint32_t a_step = L.a_stage >> 4, b_step = L.b_stage >> 4;   // descriptor address units
             const int mmas = a.BK / 32;          // each MMA consumes 32 bytes of K: advance 2 x 16 B
-            uint32_t stage = 0, phase = 0;
-            uint32_t acc = 0, acc_phase = 0;     // accumulators are used round robin
+            const uint32_t S = static_cast<uint32_t>(a.stages), kbs = static_cast<uint32_t>(kblocks);
+            const uint32_t first = me * kbs;                                   // first K block of this thread's first tile
+            uint32_t stage = first % S, phase = (first / S) & 1;
+            const uint32_t skip = (P - 1) * kbs;                               // blocks of the other thread's tiles (< S)
+            uint32_t acc = me, acc_phase = 0;                                  // accumulators are used round robin (P <= n_acc)
             bool ok = true;
-            bool ready = mbar_try_wait(bar_full, 0);
-            for (uint32_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
+            bool ready = false;
+            for (uint32_t tile = blockIdx.x + me * gridDim.x; ok && tile < a.num_tiles; tile += P * gridDim.x) {
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget, 128u)) {
                     report_timeout(a.status, QTZ_SITE_TMEM_EMPTY);
                     *abort_flag = 1;
@@ -371,19 +383,25 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     tc_fence_after();
                     const uint64_t da = desc_a0 + stage * a_step, db = desc_b0 + stage * b_step;
                     const uint32_t freed = bar_empty + 8 * stage;
-                    if (++stage == static_cast<uint32_t>(a.stages)) {
+                    if (++stage == S) {
                         stage = 0;
                         phase ^= 1;
                     }
                     // poll the next stage now: the answer arrives while the MMAs below are being issued
-                    ready = mbar_try_wait(bar_full + 8 * stage, phase);
+                    ready = (kb + 1 < kblocks || P == 1) && mbar_try_wait(bar_full + 8 * stage, phase);
                     for (int k = 0; k < mmas; ++k) mma_i8(d_tmem, da + 2 * k, db + 2 * k, a.idesc, (kb > 0 || k > 0) ? 1u : 0u);
                     mma_commit(freed);           // frees the stage once these MMAs have read it
                 }
                 if (ok) mma_commit(bar_tfull + 8 * acc);
-                if (++acc == static_cast<uint32_t>(a.n_acc)) {
-                    acc = 0;
+                acc += P;
+                if (acc >= static_cast<uint32_t>(a.n_acc)) {
+                    acc -= a.n_acc;
                     acc_phase ^= 1;
+                }
+                stage += skip;
+                if (stage >= S) {
+                    stage -= S;
+                    phase ^= 1;
                 }
             }
         }
@@ -1144,6 +1162,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.gwarps = a.groups == 4 ? 4 : 8;
     a.stages = depth(a.groups, a.obuf);
     if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
+    a.mma_lanes = (a.n_acc >= 4 && a.stages >= 2 * kblocks) ? 2 : 1;
     const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf).total + 1024;
     a.fold = (a.fast_requant && a.ncls == 1 && a.zw == 0) ? 1 : 0;
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
