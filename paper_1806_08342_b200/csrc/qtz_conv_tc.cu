@@ -40,8 +40,7 @@ constexpr int kTmemCols = 512;
 constexpr int kEpiWarps = 16;        // epilogue warps: four groups of four or two groups of eight
 constexpr int kEpiGroups = 4;        // most epilogue groups; the groups take tiles in turn, so their drains overlap
 constexpr int kStoreWarp = 2 + kEpiWarps;            // its lane g issues the output stores of group g
-constexpr int kMmaWarp2 = kStoreWarp + 1;            // second MMA-issuing warp (short reductions)
-constexpr int kThreadsTc = 32 * (kMmaWarp2 + 1);     // producer warp, MMA warp, epilogue warps, store warp, MMA warp
+constexpr int kThreadsTc = 32 * (kStoreWarp + 1);    // producer warp, MMA warp, epilogue warps, store warp
 constexpr int kMaxObuf = 4;
 constexpr int kMaxStages = 8;
 constexpr int kNumBarriers = 2 * kMaxStages + 2 * kMaxAcc + 2 * kEpiGroups * kMaxObuf;
@@ -73,7 +72,7 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f)
 }
 
 struct TcArgs {
-    FastDiv dv_per_group, dv_group_m, dv_group_last, dv_tiles_w, dv_tiles_h, dv_kb_per_tap, dv_kw;
+    FastDiv dv_per_group, dv_group_m, dv_group_last, dv_tiles_w, dv_tiles_h;
     int32_t is4d;
     int32_t tw, th, tb, rows;               // pixel box of one tile and its row count (<= 128)
     int32_t tiles_w, tiles_h, n_tiles;
@@ -86,7 +85,6 @@ struct TcArgs {
     int32_t obuf;                           // staging boxes per epilogue group (1..4)
     int32_t n_acc, acc_stride;              // accumulators in TMEM and the columns between them
     int32_t gwarps;                         // warps per epilogue group: 4 (up to four groups) or 8 (up to two)
-    int32_t mma_lanes;                      // MMA-issuing threads (1 or 2, each in its own warp)
     uint32_t idesc;
     const int32_t* bias;
     const int32_t* wsum;                    // [ncls][N]
@@ -247,7 +245,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + kNumBarriers * 8);
     volatile uint32_t* const abort_flag = tmem_slot + 1;
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the shuffle tells the compiler that the warp index is the same in all lanes
+    const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < a.stages; ++s) {
@@ -275,134 +274,113 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
 
     const int kblocks = a.taps * a.kb_per_tap;
 
     if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
-        // The K blocks of all tiles of this CTA form one sequence; block g goes to ring stage g mod
-        // stages.  A single thread working through that sequence spends well over a thousand cycles per
-        // block on its own dependent instructions (tile decode, barrier poll, two TMA issues), which
-        // starves layers with a short reduction.  So one lane per stage runs the loop: lane l owns
-        // stage l and takes blocks l, l + stages, ...; a lane waits only on its own stage's barrier.
+        // The whole warp runs the loop in step, so every address, coordinate and counter is a
+        // warp-uniform value; one elected lane issues the copies.  (Letting a single lane run the loop
+        // alone makes each issue pay for moving its operands into uniform registers: hundreds of
+        // cycles per K block, which starves layers with a short reduction.)
         const uint32_t S = static_cast<uint32_t>(a.stages);
-        const uint32_t kbs = static_cast<uint32_t>(kblocks);
         const uint32_t tx = static_cast<uint32_t>(a.rows * a.BK + a.BN * a.BK);
-        const uint32_t adv_t = S / kbs, adv_kb = S - adv_t * kbs;      // one trip moves every lane S blocks on
-        uint32_t t = static_cast<uint32_t>(lane) / kbs;                 // tile ordinal within this CTA
-        uint32_t kb = static_cast<uint32_t>(lane) - t * kbs;            // K block within the tile
-        const uint32_t stage = static_cast<uint32_t>(lane);
-        const uint32_t full = bar_full + 8 * stage, empty = bar_empty + 8 * stage;
-        const uint32_t dst_a = base + L.a_off + stage * L.a_stage;
-        const uint32_t dst_b = base + L.b_off + stage * L.b_stage;
-        uint32_t phase = 0;
-        bool issued_any = false, failed = false;
-        for (;;) {
-            const uint64_t tile64 = blockIdx.x + static_cast<uint64_t>(t) * gridDim.x;
-            const bool active = static_cast<uint32_t>(lane) < S && tile64 < a.num_tiles;
-            if (active) {
-                int n_tile, w0, h0, b0;
-                uint32_t m_tile;
-                decode_tile(a, static_cast<uint32_t>(tile64), m_tile, n_tile);
-                tile_origin(a, m_tile, w0, h0, b0);
-                const uint32_t tap = fdiv(kb, a.dv_kb_per_tap);
-                const int kc = static_cast<int>(kb - tap * a.dv_kb_per_tap.d) * a.BK;    // channel offset inside the tap
-                if (mbar_wait(empty, phase ^ 1, a.wait_budget, 64u)) {
-                    mbar_arrive_expect_tx(full, tx);
-                    if (a.is4d) {
-                        const uint32_t ty = fdiv(tap, a.dv_kw);
-                        tma_load_4d(dst_a, &map_a, full, kc, w0 + static_cast<int>(tap - ty * a.dv_kw.d) - a.pad,
-                                    h0 + static_cast<int>(ty) - a.pad, b0);
-                    } else {
-                        tma_load_2d(dst_a, &map_a, full, kc, w0);
+        uint32_t stage = 0, phase = 0;
+        bool failed = false;
+        for (uint32_t tile = blockIdx.x; !failed && tile < a.num_tiles; tile += gridDim.x) {
+            int n_tile, w0, h0, b0;
+            uint32_t m_tile;
+            decode_tile(a, tile, m_tile, n_tile);
+            tile_origin(a, m_tile, w0, h0, b0);
+            const int nrow = n_tile * a.BN;
+            int tap_x = 0, tap_y = 0, kcol = 0;      // filter tap of the current K block and its first weight column
+            for (int tap = 0; tap < a.taps && !failed; ++tap) {
+                for (int kc = 0; kc < a.c_pad; kc += a.BK) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget, 64u)) ||
+                        *abort_flag != 0) {
+                        failed = true;
+                        break;
                     }
-                    tma_load_2d(dst_b, &map_b, full, static_cast<int>(tap) * a.c_pad + kc, n_tile * a.BN);
-                    issued_any = true;
-                } else {
-                    failed = true;
+                    if (elect_one()) {
+                        const uint32_t full = bar_full + 8 * stage;
+                        mbar_arrive_expect_tx(full, tx);
+                        if (a.is4d)
+                            tma_load_4d(base + L.a_off + stage * L.a_stage, &map_a, full, kc, w0 + tap_x - a.pad, h0 + tap_y - a.pad, b0);
+                        else
+                            tma_load_2d(base + L.a_off + stage * L.a_stage, &map_a, full, kc, w0);
+                        tma_load_2d(base + L.b_off + stage * L.b_stage, &map_b, full, kcol + kc, nrow);
+                    }
+                    __syncwarp();
+                    if (++stage == S) {
+                        stage = 0;
+                        phase ^= 1;
+                    }
+                }
+                kcol += a.c_pad;
+                if (++tap_x == a.kw) {
+                    tap_x = 0;
+                    ++tap_y;
                 }
             }
-            if (__ballot_sync(0xffffffffu, failed || (lane == 0 && *abort_flag != 0)) != 0u) {
-                failed = true;
-                break;
-            }
-            if (!__any_sync(0xffffffffu, active)) break;      // lane 0 holds the earliest block: nothing left
-            t += adv_t;
-            kb += adv_kb;
-            if (kb >= kbs) {
-                kb -= kbs;
-                ++t;
-            }
-            phase ^= 1;
         }
         if (failed) {
             if (lane == 0) {
                 report_timeout(a.status, QTZ_SITE_SMEM_EMPTY);
                 *abort_flag = 1;
             }
-            // drain: give this lane's last copy a bounded time to land before the CTA exits
-            if (issued_any) (void)mbar_wait(full, phase, a.wait_budget);
+            // drain: give the most recent copy (the others were issued before it) a bounded time to land
+            // before the CTA exits
+            const uint32_t last = stage == 0 ? S - 1 : stage - 1;
+            (void)mbar_wait(bar_full + 8 * last, stage == 0 ? phase ^ 1 : phase, 20000000LL);
         }
-    } else if (warp == 1 || warp == kMmaWarp2) {
-        // ------------------------------ MMA issuers -------------------------------
-        // One thread issues all MMAs of a tile.  With a short reduction its own dependent instructions
-        // (two barrier polls, descriptors, one or two MMAs, two commits) take longer per tile than the
-        // tensor core does, so when two whole tiles fit in the operand ring a second issuing thread, in a
-        // warp of its own, takes every other tile; every tile still has one issuing thread and its own
-        // accumulator.
-        const uint32_t P = static_cast<uint32_t>(a.mma_lanes);
-        const uint32_t me = warp == 1 ? 0u : 1u;
-        if (lane == 0 && me < P) {
-            const uint64_t desc_a0 = make_kmajor_desc(base + L.a_off, a.BK);
-            const uint64_t desc_b0 = make_kmajor_desc(base + L.b_off, a.BK);
-            const uint32_t a_step = L.a_stage >> 4, b_step = L.b_stage >> 4;   // descriptor address units
-            const int mmas = a.BK / 32;          // each MMA consumes 32 bytes of K: advance 2 x 16 B
-            const uint32_t S = static_cast<uint32_t>(a.stages), kbs = static_cast<uint32_t>(kblocks);
-            const uint32_t first = me * kbs;                                   // first K block of this thread's first tile
-            uint32_t stage = first % S, phase = (first / S) & 1;
-            const uint32_t skip = (P - 1) * kbs;                               // blocks of the other thread's tiles (< S)
-            uint32_t acc = me, acc_phase = 0;                                  // accumulators are used round robin (P <= n_acc)
-            bool ok = true;
-            bool ready = false;
-            for (uint32_t tile = blockIdx.x + me * gridDim.x; ok && tile < a.num_tiles; tile += P * gridDim.x) {
-                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget, 128u)) {
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer --------------------------------
+        // Again the whole warp runs the loop and one elected lane issues, so descriptors and TMEM
+        // addresses stay warp-uniform.  Only this warp ever issues MMAs.
+        const uint64_t desc_a0 = make_kmajor_desc(base + L.a_off, a.BK);
+        const uint64_t desc_b0 = make_kmajor_desc(base + L.b_off, a.BK);
+        const uint32_t a_step = L.a_stage >> 4, b_step = L.b_stage >> 4;   // descriptor address units
+        const int mmas = a.BK / 32;          // each MMA consumes 32 bytes of K: advance 2 x 16 B
+        const uint32_t S = static_cast<uint32_t>(a.stages);
+        uint32_t stage = 0, phase = 0;
+        uint32_t acc = 0, acc_phase = 0;     // accumulators are used round robin
+        bool ok = true;
+        for (uint32_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget, 128u))) {
+                if (lane == 0) {
                     report_timeout(a.status, QTZ_SITE_TMEM_EMPTY);
                     *abort_flag = 1;
+                }
+                break;
+            }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * a.acc_stride;
+            for (int kb = 0; kb < kblocks; ++kb) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8 * stage, phase, a.wait_budget, 64u))) {
+                    if (lane == 0) {
+                        report_timeout(a.status, QTZ_SITE_TMA_FULL);
+                        *abort_flag = 1;
+                    }
+                    ok = false;
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * a.acc_stride;
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!ready && !mbar_wait(bar_full + 8 * stage, phase, a.wait_budget, 64u)) {
-                        report_timeout(a.status, QTZ_SITE_TMA_FULL);
-                        *abort_flag = 1;
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after();
+                if (elect_one()) {
                     const uint64_t da = desc_a0 + stage * a_step, db = desc_b0 + stage * b_step;
-                    const uint32_t freed = bar_empty + 8 * stage;
-                    if (++stage == S) {
-                        stage = 0;
-                        phase ^= 1;
-                    }
-                    // poll the next stage now: the answer arrives while the MMAs below are being issued
-                    ready = (kb + 1 < kblocks || P == 1) && mbar_try_wait(bar_full + 8 * stage, phase);
                     for (int k = 0; k < mmas; ++k) mma_i8(d_tmem, da + 2 * k, db + 2 * k, a.idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                    mma_commit(freed);           // frees the stage once these MMAs have read it
+                    mma_commit(bar_empty + 8 * stage);                     // frees the stage once these MMAs have read it
+                    if (kb == kblocks - 1) mma_commit(bar_tfull + 8 * acc);
                 }
-                if (ok) mma_commit(bar_tfull + 8 * acc);
-                acc += P;
-                if (acc >= static_cast<uint32_t>(a.n_acc)) {
-                    acc -= a.n_acc;
-                    acc_phase ^= 1;
-                }
-                stage += skip;
-                if (stage >= S) {
-                    stage -= S;
+                __syncwarp();
+                if (++stage == S) {
+                    stage = 0;
                     phase ^= 1;
                 }
+            }
+            if (++acc == static_cast<uint32_t>(a.n_acc)) {
+                acc = 0;
+                acc_phase ^= 1;
             }
         }
     } else if (warp == kStoreWarp) {
@@ -1004,8 +982,6 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.dv_group_last = make_fastdiv(static_cast<uint32_t>(std::max(1, a.m_tiles % a.group_m)));
     a.dv_tiles_w = make_fastdiv(static_cast<uint32_t>(a.tiles_w));
     a.dv_tiles_h = make_fastdiv(static_cast<uint32_t>(std::max(1, a.tiles_h)));
-    a.dv_kb_per_tap = make_fastdiv(static_cast<uint32_t>(a.kb_per_tap));
-    a.dv_kw = make_fastdiv(static_cast<uint32_t>(a.kw));
     // shared-memory budget -> pipeline depth
     // worst case (all border classes) for the smem opt-in; every launch picks its own depth
     a.groups = 1;
@@ -1162,7 +1138,6 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.gwarps = a.groups == 4 ? 4 : 8;
     a.stages = depth(a.groups, a.obuf);
     if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
-    a.mma_lanes = (a.n_acc >= 4 && a.stages >= 2 * kblocks) ? 2 : 1;
     const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf).total + 1024;
     a.fold = (a.fast_requant && a.ncls == 1 && a.zw == 0) ? 1 : 0;
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
