@@ -43,7 +43,8 @@ constexpr int kStoreWarp = 2 + kEpiWarps;            // its lane g issues the ou
 constexpr int kThreadsTc = 32 * (kStoreWarp + 1);    // producer warp, MMA warp, epilogue warps, store warp
 constexpr int kMaxObuf = 4;
 constexpr int kMaxStages = 8;
-constexpr int kNumBarriers = 2 * kMaxStages + 2 * kMaxAcc + 2 * kEpiGroups * kMaxObuf;
+constexpr int kNumBarriers = 2 * kMaxStages + 2 * kMaxAcc + 2 * kEpiGroups * kMaxObuf + 1;
+constexpr int kResidentBMax = 80 * 1024;   // weights of a whole layer stay in shared memory up to this size
 constexpr int kMaxCls = 16;
 constexpr int kSmemBudget = 227 * 1024 - 1024;  // leave room for the 1 KB alignment slack
 
@@ -83,6 +84,7 @@ struct TcArgs {
     int32_t kb_per_tap, c_pad;
     int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
     int32_t obuf;                           // staging boxes per epilogue group (1..4)
+    int32_t bres;                           // weight K blocks kept resident in shared memory (0: weights go through the ring)
     int32_t n_acc, acc_stride;              // accumulators in TMEM and the columns between them
     int32_t gwarps;                         // warps per epilogue group: 4 (up to four groups) or 8 (up to two)
     uint32_t idesc;
@@ -104,15 +106,16 @@ struct SmemLayout {
     uint32_t a_stage, b_stage;
 };
 
-// Operand ring, one output staging box and one set of per-channel tables per epilogue group, barriers.
-__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int groups, int obuf)
+// Operand ring (activations, and weights unless all `bres` weight blocks of the layer stay resident),
+// output staging boxes and one set of per-channel tables per epilogue group, barriers.
+__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int groups, int obuf, int bres)
 {
     SmemLayout L;
     L.a_stage = kTileM * BK;
     L.b_stage = BN * BK;
     L.a_off = 0;
     L.b_off = L.a_off + stages * L.a_stage;
-    L.out_off = L.b_off + stages * L.b_stage;
+    L.out_off = L.b_off + (bres > 0 ? bres : stages) * L.b_stage;
     L.tbl_off = L.out_off + groups * obuf * kTileM * out_box;
     L.mult_rel = ncls > 1 ? ncls * BN * 4 : BN * 8;   // first table: [ncls][BN] int32, or [BN] int64 when folded
     L.sh_rel = L.mult_rel + BN * 4;
@@ -233,7 +236,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
-    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf);
+    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres);
 
     const uint32_t bar_full = base + L.bar_off;
     const uint32_t bar_empty = bar_full + 8 * kMaxStages;
@@ -241,6 +244,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t bar_tempty = bar_tfull + 8 * kMaxAcc;
     const uint32_t bar_ofull = bar_tempty + 8 * kMaxAcc;                               // [group][box]: box written
     const uint32_t bar_oempty = bar_ofull + 8 * kEpiGroups * kMaxObuf;        // [group][box]: box read by its store
+    const uint32_t bar_wres = bar_oempty + 8 * kEpiGroups * kMaxObuf;         // resident weights have landed
     volatile uint32_t* const tmem_slot =
         reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + kNumBarriers * 8);
     volatile uint32_t* const abort_flag = tmem_slot + 1;
@@ -261,6 +265,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             mbar_init(bar_ofull + 8 * i, a.gwarps);
             mbar_init(bar_oempty + 8 * i, 1);
         }
+        mbar_init(bar_wres, 1);
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_a);
@@ -285,9 +290,21 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // alone makes each issue pay for moving its operands into uniform registers: hundreds of
         // cycles per K block, which starves layers with a short reduction.)
         const uint32_t S = static_cast<uint32_t>(a.stages);
-        const uint32_t tx = static_cast<uint32_t>(a.rows * a.BK + a.BN * a.BK);
+        const bool wres = a.bres > 0;
+        const uint32_t tx = static_cast<uint32_t>(a.rows * a.BK + (wres ? 0 : a.BN * a.BK));
         uint32_t stage = 0, phase = 0;
         bool failed = false;
+        if (wres && blockIdx.x < a.num_tiles) {
+            // the layer's weights are small: fetch all of their K blocks once, they stay for every tile
+            if (elect_one()) {
+                mbar_arrive_expect_tx(bar_wres, static_cast<uint32_t>(a.bres) * L.b_stage);
+                int blk = 0;
+                for (int tap = 0; tap < a.taps; ++tap)
+                    for (int kc = 0; kc < a.c_pad; kc += a.BK, ++blk)
+                        tma_load_2d(base + L.b_off + blk * L.b_stage, &map_b, bar_wres, tap * a.c_pad + kc, 0);
+            }
+            __syncwarp();
+        }
         for (uint32_t tile = blockIdx.x; !failed && tile < a.num_tiles; tile += gridDim.x) {
             int n_tile, w0, h0, b0;
             uint32_t m_tile;
@@ -309,7 +326,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             tma_load_4d(base + L.a_off + stage * L.a_stage, &map_a, full, kc, w0 + tap_x - a.pad, h0 + tap_y - a.pad, b0);
                         else
                             tma_load_2d(base + L.a_off + stage * L.a_stage, &map_a, full, kc, w0);
-                        tma_load_2d(base + L.b_off + stage * L.b_stage, &map_b, full, kcol + kc, nrow);
+                        if (!wres) tma_load_2d(base + L.b_off + stage * L.b_stage, &map_b, full, kcol + kc, nrow);
                     }
                     __syncwarp();
                     if (++stage == S) {
@@ -346,6 +363,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t stage = 0, phase = 0;
         uint32_t acc = 0, acc_phase = 0;     // accumulators are used round robin
         bool ok = true;
+        const bool wres = a.bres > 0;
+        if (wres && blockIdx.x < a.num_tiles && !__all_sync(0xffffffffu, mbar_wait(bar_wres, 0, a.wait_budget, 64u))) {
+            if (lane == 0) {
+                report_timeout(a.status, QTZ_SITE_TMA_FULL);
+                *abort_flag = 1;
+            }
+            ok = false;
+        }
         for (uint32_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
             if (!__all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget, 128u))) {
                 if (lane == 0) {
@@ -367,7 +392,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 tc_fence_after();
                 if (elect_one()) {
-                    const uint64_t da = desc_a0 + stage * a_step, db = desc_b0 + stage * b_step;
+                    const uint64_t da = desc_a0 + stage * a_step, db = desc_b0 + (wres ? static_cast<uint32_t>(kb) : stage) * b_step;
                     for (int k = 0; k < mmas; ++k) mma_i8(d_tmem, da + 2 * k, db + 2 * k, a.idesc, (kb > 0 || k > 0) ? 1u : 0u);
                     mma_commit(bar_empty + 8 * stage);                     // frees the stage once these MMAs have read it
                     if (kb == kblocks - 1) mma_commit(bar_tfull + 8 * acc);
@@ -987,8 +1012,9 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.groups = 1;
     a.gwarps = 8;
     a.obuf = 1;
+    a.bres = 0;
     a.stages = 2;
-    if (make_layout(a.BK, a.BN, 2, a.ncls, a.out_box, 1, 1).total > static_cast<uint32_t>(kSmemBudget)) return QTZ_ERR_UNSUPPORTED;
+    if (make_layout(a.BK, a.BN, 2, a.ncls, a.out_box, 1, 1, 0).total > static_cast<uint32_t>(kSmemBudget)) return QTZ_ERR_UNSUPPORTED;
 
     // instruction descriptor: s32 accumulate, A = u8, B = s8, both K-major, N and M of the tile
     a.idesc = (2u << 4) | (0u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) |
@@ -1118,27 +1144,35 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     auto depth = [&](int groups, int obuf) {
         int st_ = kMaxStages;
         for (; st_ >= 2; --st_)
-            if (make_layout(a.BK, a.BN, st_, a.ncls, a.out_box, groups, obuf).total <= static_cast<uint32_t>(kSmemBudget)) break;
+            if (make_layout(a.BK, a.BN, st_, a.ncls, a.out_box, groups, obuf, a.bres).total <= static_cast<uint32_t>(kSmemBudget)) break;
         return st_;
     };
     const int kblocks = a.taps * a.kb_per_tap;
     const int need = std::min(4, kblocks + 1);
+    // weights of a single-column-tile layer stay resident when they are small: the ring then carries activations only
+    a.bres = (a.n_tiles == 1 && kblocks * a.BN * a.BK <= kResidentBMax) ? kblocks : 0;
     static const int choice[7][2] = {{4, 3}, {4, 2}, {2, 3}, {2, 2}, {1, 2}, {2, 1}, {1, 1}};
-    a.groups = 1;
-    a.obuf = 1;
-    for (const auto& c : choice) {
-        if (c[0] == 4 && a.n_acc < 4) continue;
-        const int ob = a.raw ? 1 : c[1];             // the boxes rotate across tiles as well
-        if (depth(c[0], ob) >= need) {
-            a.groups = c[0];
-            a.obuf = ob;
-            break;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        a.groups = 1;
+        a.obuf = 1;
+        bool found = false;
+        for (const auto& c : choice) {
+            if (c[0] == 4 && a.n_acc < 4) continue;
+            const int ob = a.raw ? 1 : c[1];         // the boxes rotate across tiles as well
+            if (depth(c[0], ob) >= need) {
+                a.groups = c[0];
+                a.obuf = ob;
+                found = true;
+                break;
+            }
         }
+        if (found || a.bres == 0) break;
+        a.bres = 0;                                  // no room beside resident weights: send them through the ring
     }
     a.gwarps = a.groups == 4 ? 4 : 8;
     a.stages = depth(a.groups, a.obuf);
     if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
-    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf).total + 1024;
+    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres).total + 1024;
     a.fold = (a.fast_requant && a.ncls == 1 && a.zw == 0) ? 1 : 0;
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
     conv_tc_kernel<<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, a);
