@@ -85,6 +85,7 @@ struct TcArgs {
     int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
     int32_t obuf;                           // staging boxes per epilogue group (1..4)
     int32_t bres;                           // weight K blocks kept resident in shared memory (0: weights go through the ring)
+    int32_t spb;                            // K blocks per ring stage (one barrier handshake covers them all)
     int32_t n_acc, acc_stride;              // accumulators in TMEM and the columns between them
     int32_t gwarps;                         // warps per epilogue group: 4 (up to four groups) or 8 (up to two)
     uint32_t idesc;
@@ -103,19 +104,21 @@ struct TcArgs {
 
 struct SmemLayout {
     uint32_t a_off, b_off, out_off, tbl_off, tbl_stride, mult_rel, sh_rel, addhi_rel, bar_off, total;
-    uint32_t a_stage, b_stage;
+    uint32_t a_stage, b_stage, a_blk, b_blk;
 };
 
 // Operand ring (activations, and weights unless all `bres` weight blocks of the layer stay resident),
 // output staging boxes and one set of per-channel tables per epilogue group, barriers.
-__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int groups, int obuf, int bres)
+__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int groups, int obuf, int bres, int spb)
 {
     SmemLayout L;
-    L.a_stage = kTileM * BK;
-    L.b_stage = BN * BK;
+    L.a_blk = kTileM * BK;                  // one K block of activations / of weights
+    L.b_blk = BN * BK;
+    L.a_stage = spb * L.a_blk;              // a ring stage holds spb consecutive K blocks
+    L.b_stage = spb * L.b_blk;
     L.a_off = 0;
     L.b_off = L.a_off + stages * L.a_stage;
-    L.out_off = L.b_off + (bres > 0 ? bres : stages) * L.b_stage;
+    L.out_off = L.b_off + (bres > 0 ? bres * L.b_blk : stages * L.b_stage);
     L.tbl_off = L.out_off + groups * obuf * kTileM * out_box;
     L.mult_rel = ncls > 1 ? ncls * BN * 4 : BN * 8;   // first table: [ncls][BN] int32, or [BN] int64 when folded
     L.sh_rel = L.mult_rel + BN * 4;
@@ -236,7 +239,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
-    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres);
+    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb);
 
     const uint32_t bar_full = base + L.bar_off;
     const uint32_t bar_empty = bar_full + 8 * kMaxStages;
@@ -291,17 +294,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // cycles per K block, which starves layers with a short reduction.)
         const uint32_t S = static_cast<uint32_t>(a.stages);
         const bool wres = a.bres > 0;
-        const uint32_t tx = static_cast<uint32_t>(a.rows * a.BK + (wres ? 0 : a.BN * a.BK));
+        const uint32_t tx = static_cast<uint32_t>(a.spb) * static_cast<uint32_t>(a.rows * a.BK + (wres ? 0 : a.BN * a.BK));
+        const int nst = kblocks / a.spb;         // ring stages per tile
         uint32_t stage = 0, phase = 0;
         bool failed = false;
         if (wres && blockIdx.x < a.num_tiles) {
             // the layer's weights are small: fetch all of their K blocks once, they stay for every tile
             if (elect_one()) {
-                mbar_arrive_expect_tx(bar_wres, static_cast<uint32_t>(a.bres) * L.b_stage);
+                mbar_arrive_expect_tx(bar_wres, static_cast<uint32_t>(a.bres) * L.b_blk);
                 int blk = 0;
                 for (int tap = 0; tap < a.taps; ++tap)
                     for (int kc = 0; kc < a.c_pad; kc += a.BK, ++blk)
-                        tma_load_2d(base + L.b_off + blk * L.b_stage, &map_b, bar_wres, tap * a.c_pad + kc, 0);
+                        tma_load_2d(base + L.b_off + blk * L.b_blk, &map_b, bar_wres, tap * a.c_pad + kc, 0);
             }
             __syncwarp();
         }
@@ -311,33 +315,39 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             decode_tile(a, tile, m_tile, n_tile);
             tile_origin(a, m_tile, w0, h0, b0);
             const int nrow = n_tile * a.BN;
-            int tap_x = 0, tap_y = 0, kcol = 0;      // filter tap of the current K block and its first weight column
-            for (int tap = 0; tap < a.taps && !failed; ++tap) {
-                for (int kc = 0; kc < a.c_pad; kc += a.BK) {
-                    if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget, 64u)) ||
-                        *abort_flag != 0) {
-                        failed = true;
-                        break;
-                    }
-                    if (elect_one()) {
-                        const uint32_t full = bar_full + 8 * stage;
-                        mbar_arrive_expect_tx(full, tx);
+            int tap_x = 0, tap_y = 0, kcol = 0, kc = 0;   // filter tap of the next K block, its first weight column, channel offset
+            for (int st = 0; st < nst; ++st) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget, 64u)) ||
+                    *abort_flag != 0) {
+                    failed = true;
+                    break;
+                }
+                const bool leader = elect_one();
+                const uint32_t full = bar_full + 8 * stage;
+                if (leader) mbar_arrive_expect_tx(full, tx);
+                for (int j = 0; j < a.spb; ++j) {
+                    if (leader) {
+                        const uint32_t dst_a = base + L.a_off + stage * L.a_stage + j * L.a_blk;
                         if (a.is4d)
-                            tma_load_4d(base + L.a_off + stage * L.a_stage, &map_a, full, kc, w0 + tap_x - a.pad, h0 + tap_y - a.pad, b0);
+                            tma_load_4d(dst_a, &map_a, full, kc, w0 + tap_x - a.pad, h0 + tap_y - a.pad, b0);
                         else
-                            tma_load_2d(base + L.a_off + stage * L.a_stage, &map_a, full, kc, w0);
-                        if (!wres) tma_load_2d(base + L.b_off + stage * L.b_stage, &map_b, full, kcol + kc, nrow);
+                            tma_load_2d(dst_a, &map_a, full, kc, w0);
+                        if (!wres) tma_load_2d(base + L.b_off + stage * L.b_stage + j * L.b_blk, &map_b, full, kcol + kc, nrow);
                     }
-                    __syncwarp();
-                    if (++stage == S) {
-                        stage = 0;
-                        phase ^= 1;
+                    kc += a.BK;
+                    if (kc == a.c_pad) {             // next filter tap
+                        kc = 0;
+                        kcol += a.c_pad;
+                        if (++tap_x == a.kw) {
+                            tap_x = 0;
+                            ++tap_y;
+                        }
                     }
                 }
-                kcol += a.c_pad;
-                if (++tap_x == a.kw) {
-                    tap_x = 0;
-                    ++tap_y;
+                __syncwarp();
+                if (++stage == S) {
+                    stage = 0;
+                    phase ^= 1;
                 }
             }
         }
@@ -358,6 +368,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint64_t desc_a0 = make_kmajor_desc(base + L.a_off, a.BK);
         const uint64_t desc_b0 = make_kmajor_desc(base + L.b_off, a.BK);
         const uint32_t a_step = L.a_stage >> 4, b_step = L.b_stage >> 4;   // descriptor address units
+        const uint32_t a_blk = L.a_blk >> 4, b_blk = L.b_blk >> 4;
+        const int nst = kblocks / a.spb;         // ring stages per tile
         const int mmas = a.BK / 32;          // each MMA consumes 32 bytes of K: advance 2 x 16 B
         const uint32_t S = static_cast<uint32_t>(a.stages);
         uint32_t stage = 0, phase = 0;
@@ -381,7 +393,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * a.acc_stride;
-            for (int kb = 0; kb < kblocks; ++kb) {
+            for (int st = 0; st < nst; ++st) {
                 if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8 * stage, phase, a.wait_budget, 64u))) {
                     if (lane == 0) {
                         report_timeout(a.status, QTZ_SITE_TMA_FULL);
@@ -392,10 +404,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 tc_fence_after();
                 if (elect_one()) {
-                    const uint64_t da = desc_a0 + stage * a_step, db = desc_b0 + (wres ? static_cast<uint32_t>(kb) : stage) * b_step;
-                    for (int k = 0; k < mmas; ++k) mma_i8(d_tmem, da + 2 * k, db + 2 * k, a.idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    for (int j = 0; j < a.spb; ++j) {
+                        const uint32_t kb = static_cast<uint32_t>(st * a.spb + j);
+                        const uint64_t da = desc_a0 + stage * a_step + j * a_blk;
+                        const uint64_t db = desc_b0 + (wres ? kb * b_blk : stage * b_step + j * b_blk);
+                        for (int k = 0; k < mmas; ++k) mma_i8(d_tmem, da + 2 * k, db + 2 * k, a.idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    }
                     mma_commit(bar_empty + 8 * stage);                     // frees the stage once these MMAs have read it
-                    if (kb == kblocks - 1) mma_commit(bar_tfull + 8 * acc);
+                    if (st == nst - 1) mma_commit(bar_tfull + 8 * acc);
                 }
                 __syncwarp();
                 if (++stage == S) {
@@ -1013,8 +1029,9 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.gwarps = 8;
     a.obuf = 1;
     a.bres = 0;
+    a.spb = 1;
     a.stages = 2;
-    if (make_layout(a.BK, a.BN, 2, a.ncls, a.out_box, 1, 1, 0).total > static_cast<uint32_t>(kSmemBudget)) return QTZ_ERR_UNSUPPORTED;
+    if (make_layout(a.BK, a.BN, 2, a.ncls, a.out_box, 1, 1, 0, 1).total > static_cast<uint32_t>(kSmemBudget)) return QTZ_ERR_UNSUPPORTED;
 
     // instruction descriptor: s32 accumulate, A = u8, B = s8, both K-major, N and M of the tile
     a.idesc = (2u << 4) | (0u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) |
@@ -1144,13 +1161,22 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     auto depth = [&](int groups, int obuf) {
         int st_ = kMaxStages;
         for (; st_ >= 2; --st_)
-            if (make_layout(a.BK, a.BN, st_, a.ncls, a.out_box, groups, obuf, a.bres).total <= static_cast<uint32_t>(kSmemBudget)) break;
+            if (make_layout(a.BK, a.BN, st_, a.ncls, a.out_box, groups, obuf, a.bres, a.spb).total <= static_cast<uint32_t>(kSmemBudget)) break;
         return st_;
     };
     const int kblocks = a.taps * a.kb_per_tap;
-    const int need = std::min(4, kblocks + 1);
     // weights of a single-column-tile layer stay resident when they are small: the ring then carries activations only
     a.bres = (a.n_tiles == 1 && kblocks * a.BN * a.BK <= kResidentBMax) ? kblocks : 0;
+    // several K blocks share a ring stage (one barrier handshake for all of them) while the stage stays within 32 KB
+    auto blocks_per_stage = [&]() {
+        const int blk = kTileM * a.BK + (a.bres > 0 ? 0 : a.BN * a.BK);
+        int best = 1;
+        for (int c = 2; c <= 4; ++c)
+            if (kblocks % c == 0 && c * blk <= 32 * 1024) best = c;
+        return best;
+    };
+    a.spb = blocks_per_stage();
+    int need = std::min(4, kblocks / a.spb + 1);
     static const int choice[7][2] = {{4, 3}, {4, 2}, {2, 3}, {2, 2}, {1, 2}, {2, 1}, {1, 1}};
     for (int attempt = 0; attempt < 2; ++attempt) {
         a.groups = 1;
@@ -1168,11 +1194,13 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
         }
         if (found || a.bres == 0) break;
         a.bres = 0;                                  // no room beside resident weights: send them through the ring
+        a.spb = blocks_per_stage();
+        need = std::min(4, kblocks / a.spb + 1);
     }
     a.gwarps = a.groups == 4 ? 4 : 8;
     a.stages = depth(a.groups, a.obuf);
     if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
-    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres).total + 1024;
+    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb).total + 1024;
     a.fold = (a.fast_requant && a.ncls == 1 && a.zw == 0) ? 1 : 0;
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
     conv_tc_kernel<<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, a);
