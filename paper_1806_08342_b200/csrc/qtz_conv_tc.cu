@@ -544,11 +544,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const int32_t r = (live && !a.raw) ? __ldg(a.rshift + n) : 40;
                     const int32_t addhi = a.fast_requant ? (2 * off + 1) * (1 << (r - 33)) : 0;
                     mult_s[j] = m;
-                    sh_s[j] = a.fast_requant ? r - 32 : r;
+                    sh_s[j] = (fold || a.fast_requant) ? r - 32 : r;
                     if (fold) {
+                        // rounding constant 2^(r-1) and the output offset (z_y - act_min) 2^r in one 64-bit addend
                         const int32_t ws = live ? __ldg(a.wsum + n) : 0;
                         const int32_t corr = bias - a.zx * ws;
-                        add64_s[j] = static_cast<int64_t>(corr) * m + (static_cast<int64_t>(addhi) << 32);
+                        add64_s[j] = static_cast<int64_t>(corr) * m + (static_cast<int64_t>(2 * off + 1) << (r - 1));
                     } else {
                         addhi_s[j] = addhi;
                         for (int c = 0; c < a.ncls; ++c) {
@@ -1070,7 +1071,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.zw = p->w_zp_signed;
     a.raw = d.outkind == QTZ_OUT_S32_RAW;
     a.fast_requant = (!a.raw && p->rshift_min >= 33 && p->rshift_max <= 53) ? 1 : 0;
-    a.fold = (a.fast_requant && a.ncls == 1 && a.zw == 0) ? 1 : 0;
+    a.fold = 0;                             // decided per launch (it depends on the zero points)
     a.status = h->status_dev;
     a.wait_budget = 2000000000LL;  // about one second of SM clocks
     t->grid = static_cast<int>(std::min<int64_t>(a.num_tiles, h->num_sms));
@@ -1201,7 +1202,8 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.stages = depth(a.groups, a.obuf);
     if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
     const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb).total + 1024;
-    a.fold = (a.fast_requant && a.ncls == 1 && a.zw == 0) ? 1 : 0;
+    // folded form: shifts 32..53 (the high word of the 64-bit sum, shifted on by r - 32)
+    a.fold = (!a.raw && a.ncls == 1 && a.zw == 0 && p->rshift_min >= 32 && p->rshift_max <= 53) ? 1 : 0;
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
     conv_tc_kernel<<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, a);
     QTZ_LAUNCH_CHECK(h, "conv_tc_kernel");

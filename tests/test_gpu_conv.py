@@ -27,14 +27,14 @@ def make_weights(wkind, shape, seed):
     return None, codes, None                                        # packed by the caller (layout differs)
 
 
-def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=0, expect_kernel=None):
+def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=0, expect_kernel=None, real_m=None, bias_range=20000):
     x = synth.uniform_u8((b, h, w, c), seed, 1)
     xp = pitched(x)
     api_w, codes, zw = make_weights(wkind, (n, k, k, c), seed)
     if wkind == qtz.W_S4_PACKED_PER_CHANNEL_SYM:
         api_w = oracle.pack_s4(codes.reshape(n, -1))
     g = synth.rng(seed, 71)
-    bias = g.integers(-20000, 20000, size=n).astype(np.int32)
+    bias = g.integers(-bias_range, bias_range, size=n).astype(np.int32)
     z_x = int(g.integers(64, 192))
     z_w = None if zw is None else np.full(n, zw, np.int32)
     acc = oracle.conv2d_acc(xp, z_x, codes, z_w, bias, stride, pad, c=c)
@@ -49,7 +49,8 @@ def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=0, 
         return
     # per-channel multipliers spread over two decades so that outputs use the whole code range
     span = np.abs(acc).reshape(-1, n).max(axis=0).astype(np.float64) + 1.0
-    real_m = 100.0 / span * np.exp(g.uniform(-1.0, 1.0, size=n))
+    if real_m is None:
+        real_m = 100.0 / span * np.exp(g.uniform(-1.0, 1.0, size=n))
     mr = [oracle.quantize_multiplier(float(v)) for v in real_m]
     mult = np.array([m for m, _ in mr], np.int32)
     rsh = np.array([r for _, r in mr], np.int32)
@@ -123,6 +124,19 @@ def test_conv_tensor_core_shapes(hq, shape, wkind):
 @pytest.mark.parametrize("shape", TC_SHAPES[:5])
 def test_conv_tensor_core_raw(hq, shape):
     conv_case(hq, *shape, qtz.W_U8_PER_LAYER_ASYM, seed=300 + shape[3], raw=True, expect_kernel="tcgen05")
+
+
+@pytest.mark.parametrize("lo_m,hi_m", [(0.26, 0.49), (0.13, 0.49), (0.26, 0.99), (0.3, 3.0)])
+def test_conv_large_multipliers(hq, lo_m, hi_m):
+    # Real multipliers near 1 (4-bit weights make them large): right shifts of 32 (still the folded
+    # fast form), mixed 32/33+, 31 and below (the general 64-bit form).  One input channel keeps the
+    # accumulators small enough for the outputs to spread over the code range.
+    n = 40
+    real_m = np.exp(np.linspace(np.log(lo_m), np.log(hi_m), n))
+    shifts = {oracle.quantize_multiplier(float(v))[1] for v in real_m}
+    assert (min(shifts) <= 32) and (hi_m < 0.5 or min(shifts) <= 31)
+    conv_case(hq, 3, 20, 20, 1, n, 1, 1, 0, qtz.W_S4_PACKED_PER_CHANNEL_SYM, seed=401, real_m=real_m, expect_kernel="tcgen05", bias_range=60)
+    conv_case(hq, 2, 13, 13, 2, n, 3, 1, 1, qtz.W_S8_PER_CHANNEL_SYM, seed=402, real_m=real_m / 40.0 if hi_m > 1 else real_m / 64.0, bias_range=2000)
 
 
 def test_extreme_zero_points_and_codes(hq):
