@@ -404,11 +404,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 tc_fence_after();
                 if (elect_one()) {
-                    for (int j = 0; j < a.spb; ++j) {
-                        const uint32_t kb = static_cast<uint32_t>(st * a.spb + j);
-                        const uint64_t da = desc_a0 + stage * a_step + j * a_blk;
-                        const uint64_t db = desc_b0 + (wres ? kb * b_blk : stage * b_step + j * b_blk);
-                        for (int k = 0; k < mmas; ++k) mma_i8(d_tmem, da + 2 * k, db + 2 * k, a.idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    uint64_t da = desc_a0 + stage * a_step;
+                    uint64_t db = desc_b0 + (wres ? static_cast<uint32_t>(st * a.spb) * b_blk : stage * b_step);
+                    uint32_t accumulate = st > 0 ? 1u : 0u;      // the tile's first MMA overwrites the accumulator
+                    for (int j = 0; j < a.spb; ++j, da += a_blk, db += b_blk) {
+                        mma_i8(d_tmem, da, db, a.idesc, accumulate);
+                        if (mmas >= 2) mma_i8(d_tmem, da + 2, db + 2, a.idesc, 1u);
+                        if (mmas == 4) {
+                            mma_i8(d_tmem, da + 4, db + 4, a.idesc, 1u);
+                            mma_i8(d_tmem, da + 6, db + 6, a.idesc, 1u);
+                        }
+                        accumulate = 1u;
                     }
                     mma_commit(bar_empty + 8 * stage);                     // frees the stage once these MMAs have read it
                     if (st == nst - 1) mma_commit(bar_tfull + 8 * acc);
