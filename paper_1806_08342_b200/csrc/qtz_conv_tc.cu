@@ -154,6 +154,7 @@ __device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t col, uint32_t box
 //   kMode 0 (folded):  y - act_min = hi32(acc m + A) >> (r - 32), A = corr m + 2^(r-1) + (z_y - act_min) 2^r
 //   kMode 1 (general): the correction (border class, activation sums) is added to acc first
 //   kMode 2 (any shift): 64-bit shift and clamp
+//   kMode 3 (folded, any shift r >= 1 whose result is known to fit 32 bits): low word of (acc m + A) >> r
 template <int kMode, bool kFullRange>
 __device__ __forceinline__ void requant32(const uint32_t (&v)[32], const int32_t* __restrict__ mult_s,
                                           const int32_t* __restrict__ sh_s, const int64_t* __restrict__ add64_s,
@@ -166,14 +167,22 @@ __device__ __forceinline__ void requant32(const uint32_t (&v)[32], const int32_t
         const int4 s4 = *reinterpret_cast<const int4*>(sh_s + 4 * q);
         const int32_t mm[4] = {m4.x, m4.y, m4.z, m4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
         int32_t y[4];
-        if (kMode == 0) {
+        if (kMode == 0 || kMode == 3) {
             const longlong2 a01 = *reinterpret_cast<const longlong2*>(add64_s + 4 * q);
             const longlong2 a23 = *reinterpret_cast<const longlong2*>(add64_s + 4 * q + 2);
             const int64_t aa[4] = {a01.x, a01.y, a23.x, a23.y};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int64_t prod = static_cast<int64_t>(static_cast<int32_t>(v[4 * q + e])) * mm[e] + aa[e];
-                const int32_t t = static_cast<int32_t>(prod >> 32) >> ss[e];
+                int32_t t;
+                if (kMode == 0) {
+                    t = static_cast<int32_t>(prod >> 32) >> ss[e];
+                } else {
+                    // ss = r; the funnel shift stops at 32, the shift by max(r - 32, 0) does the rest
+                    const int4 h4 = *reinterpret_cast<const int4*>(addhi_s + 4 * q);
+                    const int32_t s2[4] = {h4.x, h4.y, h4.z, h4.w};
+                    t = static_cast<int32_t>(__funnelshift_rc(static_cast<uint32_t>(prod), static_cast<uint32_t>(prod >> 32), ss[e])) >> s2[e];
+                }
                 y[e] = kFullRange ? t : __vimin_s32_relu(t, span);     // [0,255]: the saturating pack clamps
             }
         } else {
@@ -511,7 +520,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int32_t span = a.act_max - a.act_min, off = a.zy - a.act_min;
         const uint32_t lo4 = 0x01010101u * static_cast<uint32_t>(a.act_min);
         const bool fold = a.fold != 0;
-        const int mode = fold ? 0 : (a.fast_requant ? 1 : 2);
+        const int mode = a.fold == 1 ? 0 : (a.fold == 2 ? 3 : (a.fast_requant ? 1 : 2));
         const bool full_range = a.act_min == 0 && a.act_max == 255;   // then saturation to a byte is the whole clamp
         const uint32_t bar_tbl = 1 + grp;
         // this thread's pixel inside a tile never changes
@@ -550,12 +559,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const int32_t r = (live && !a.raw) ? __ldg(a.rshift + n) : 40;
                     const int32_t addhi = a.fast_requant ? (2 * off + 1) * (1 << (r - 33)) : 0;
                     mult_s[j] = m;
-                    sh_s[j] = (fold || a.fast_requant) ? r - 32 : r;
+                    sh_s[j] = (a.fold == 1 || a.fast_requant) ? r - 32 : r;
                     if (fold) {
                         // rounding constant 2^(r-1) and the output offset (z_y - act_min) 2^r in one 64-bit addend
                         const int32_t ws = live ? __ldg(a.wsum + n) : 0;
                         const int32_t corr = bias - a.zx * ws;
                         add64_s[j] = static_cast<int64_t>(corr) * m + (static_cast<int64_t>(2 * off + 1) << (r - 1));
+                        addhi_s[j] = r > 32 ? r - 32 : 0;
                     } else {
                         addhi_s[j] = addhi;
                         for (int c = 0; c < a.ncls; ++c) {
@@ -649,6 +659,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         requant32<0, true>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
                     else if (mode == 0)
                         requant32<0, false>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
+                    else if (mode == 3 && full_range)
+                        requant32<3, true>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
+                    else if (mode == 3)
+                        requant32<3, false>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
                     else if (mode == 1 && full_range)
                         requant32<1, true>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
                     else if (mode == 1)
@@ -1209,7 +1223,10 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
     const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb).total + 1024;
     // folded form: shifts 32..53 (the high word of the 64-bit sum, shifted on by r - 32)
-    a.fold = (!a.raw && a.ncls == 1 && a.zw == 0 && p->rshift_min >= 32 && p->rshift_max <= 53) ? 1 : 0;
+    // (2: shifts below 32 as well, given that no requantised value can leave 32 bits)
+    a.fold = 0;
+    if (!a.raw && a.ncls == 1 && a.zw == 0 && p->rshift_max <= 53)
+        a.fold = p->rshift_min >= 32 ? 1 : (p->narrow_ok ? 2 : 0);
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
     conv_tc_kernel<<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, a);
     QTZ_LAUNCH_CHECK(h, "conv_tc_kernel");

@@ -134,7 +134,7 @@ __device__ __forceinline__ void mac_row(const RowState<kStride>& r, const uint32
 struct Requant {
     int32_t m[8];
     int32_t sh[8];      // fast form: r - 32;  general form: r
-    int32_t addhi[8];   // fast form: high word of 2^(r-1) + ((z_y - act_min) << r) (its low word is zero for r >= 33)
+    int64_t add[8];     // fast form: 2^(r-1) + ((z_y - act_min) << r)
     uint32_t lo4;       // act_min in every byte
     int32_t span;       // act_max - act_min
     int32_t zy, lo;
@@ -149,8 +149,8 @@ __device__ __forceinline__ uint2 requant_pixel(const int32_t (&v)[8], const Requ
     int32_t y[8];
 #pragma unroll
     for (int ch = 0; ch < 8; ++ch) {
-        if (kFast) {   // 33 <= r <= 53: floor((v m + addend) / 2^r) = hi32(v m + addend) >> (r - 32)
-            const int64_t p = static_cast<int64_t>(v[ch]) * q.m[ch] + (static_cast<int64_t>(q.addhi[ch]) << 32);
+        if (kFast) {   // 32 <= r <= 53: floor((v m + addend) / 2^r) = hi32(v m + addend) >> (r - 32)
+            const int64_t p = static_cast<int64_t>(v[ch]) * q.m[ch] + q.add[ch];
             y[ch] = __vimin_s32_relu(static_cast<int32_t>(p >> 32) >> q.sh[ch], q.span);
         } else {
             const int64_t p = static_cast<int64_t>(v[ch]) * q.m[ch] + (static_cast<int64_t>(1) << (q.sh[ch] - 1));
@@ -249,7 +249,7 @@ depthwise3x3_kernel(const __grid_constant__ CUtensorMap map_x, const DwArgs a)
                 const int32_t r = a.y_raw ? 40 : __ldg(a.rshift + c0 + ch);   // raw output has no multipliers
                 rq.m[ch] = a.y_raw ? 0 : __ldg(a.mult + c0 + ch);
                 rq.sh[ch] = kFast ? r - 32 : r;
-                rq.addhi[ch] = kFast ? (2 * (a.zy - a.act_min) + 1) * (1 << (r - 33)) : 0;
+                rq.add[ch] = kFast ? static_cast<int64_t>(2 * (a.zy - a.act_min) + 1) << (r - 1) : 0;
                 base[ch] = __ldg(a.bias + c0 + ch) - a.zx * __ldg(a.wsum + c0 + ch) + 9 * a.zx * a.zw;
             }
             loaded_cc = t.cc;
@@ -477,7 +477,7 @@ qtz_status qtz_depthwise_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, uin
         p->h->last_error = "cuTensorMapEncodeTiled failed for the depthwise input";
         return QTZ_ERR_CUDA;
     }
-    const bool fast = !raw && p->rshift_min >= 33 && p->rshift_max <= 53;
+    const bool fast = !raw && p->rshift_min >= 32 && p->rshift_max <= 53;
     const bool asym = p->w_zp_signed != 0;
     if (p->ev_start) QTZ_CUDA(p->h, cudaEventRecord(p->ev_start, st));
     const unsigned blocks = static_cast<unsigned>(p->dw->grid);

@@ -1,6 +1,7 @@
 // Per-layer preparation (weights are constant at inference, Section 2.1) and dispatch of
 // the convolution entry points.
 #include <algorithm>
+#include <cstdlib>
 #include <new>
 #include <vector>
 
@@ -190,6 +191,20 @@ extern "C" qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, i
     PLAN_CUDA(cudaMemsetAsync(p->bias, 0, nb_alloc, st));
     if (bias_q_dev) PLAN_CUDA(cudaMemcpyAsync(p->bias, bias_q_dev, nb, cudaMemcpyDeviceToDevice, st));
     if (!raw) {
+        // Largest accumulator any input can produce, and with it the largest requantised value: when
+        // that stays inside 32 bits for every channel, the epilogue may narrow before it clamps.
+        std::vector<int32_t> bias_host(static_cast<size_t>(d.n), 0);
+        if (bias_q_dev) {
+            PLAN_CUDA(cudaMemcpyAsync(bias_host.data(), bias_q_dev, nb, cudaMemcpyDeviceToHost, st));
+            PLAN_CUDA(cudaStreamSynchronize(st));
+        }
+        const int64_t wmax = d.wkind == QTZ_W_S4_PACKED_PER_CHANNEL_SYM ? 8 : (d.wkind == QTZ_W_S8_PER_CHANNEL_SYM ? 128 : 255);
+        p->narrow_ok = true;
+        for (int i = 0; i < d.n; ++i) {
+            const int64_t bound = static_cast<int64_t>(p->k_total) * 255 * wmax + std::llabs(static_cast<long long>(bias_host[i]));
+            const unsigned __int128 scaled = (static_cast<unsigned __int128>(bound) * static_cast<uint32_t>(mult_host[i])) >> rshift_host[i];
+            if (scaled > static_cast<unsigned __int128>(0x7fffffff - 1024)) p->narrow_ok = false;
+        }
         PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->mult), nb_alloc));
         PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->rshift), nb_alloc));
         PLAN_CUDA(cudaMemsetAsync(p->mult, 0, nb_alloc, st));

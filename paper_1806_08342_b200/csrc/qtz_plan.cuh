@@ -21,6 +21,7 @@ struct qtz_plan {
     int n_padded = 0;     // rows of w_direct (multiple of 64)
     int rshift_max = 1;
     int rshift_min = 62;  // smallest per-channel right shift (selects the epilogue's requantise form)
+    bool narrow_ok = false;  // every requantised value provably fits 32 bits before the clamp (any accumulator, any shift)
     int w_zp_signed = 0;  // weight zero point after moving codes to int8 (z_w - 128 for uint8 weights)
 
     int8_t* w_direct = nullptr;   // [n_padded][k_padded] int8, zero padded       (direct path)

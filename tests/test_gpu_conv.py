@@ -259,6 +259,16 @@ DW_SHAPES = [(2, 14, 14, 32, 1), (1, 15, 13, 64, 2), (3, 7, 7, 24, 1), (1, 9, 10
 @pytest.mark.parametrize("wkind", [qtz.W_S8_PER_CHANNEL_SYM, qtz.W_U8_PER_LAYER_ASYM,
                                    qtz.W_S4_PACKED_PER_CHANNEL_SYM])
 def test_depthwise(hq, shape, wkind):
+    depthwise_case(hq, shape, wkind, 150.0)
+
+
+@pytest.mark.parametrize("gain", [4000.0, 30000.0])
+def test_depthwise_large_multipliers(hq, gain):
+    # multipliers around 0.3 (right shift 32, still the fast form) and above 1 (general form)
+    depthwise_case(hq, (2, 12, 12, 40, 1), qtz.W_S4_PACKED_PER_CHANNEL_SYM, gain)
+
+
+def depthwise_case(hq, shape, wkind, gain):
     b, h, w, c, stride = shape
     x = pitched(synth.uniform_u8((b, h, w, c), 31, c))
     api_w, codes, zw = make_weights(wkind, (3, 3, c), 31 + c)
@@ -270,9 +280,11 @@ def test_depthwise(hq, shape, wkind):
     z_w = None if zw is None else np.full(c, zw, np.int32)
     acc = oracle.depthwise_acc(x, z_x, codes, z_w, bias, stride, 1, c=c)
     span = np.abs(acc).reshape(-1, c).max(axis=0).astype(np.float64) + 1.0
-    mr = [oracle.quantize_multiplier(float(v)) for v in 150.0 / span]
+    mr = [oracle.quantize_multiplier(float(v)) for v in gain / span]
     mult = np.array([m for m, _ in mr], np.int32)
     rsh = np.array([r for _, r in mr], np.int32)
+    if gain > 1000.0:
+        assert rsh.min() <= 32
     z_y = 30
     want = oracle.requantize(acc, mult, rsh, z_y, z_y, 255)
     desc = qtz.conv_desc(b, h, w, c, c, 3, 3, stride, 1, wkind)
