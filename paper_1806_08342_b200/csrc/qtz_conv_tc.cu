@@ -710,16 +710,27 @@ __device__ __forceinline__ int32_t api_code_s8(const void* w, int wkind, int64_t
     return static_cast<int32_t>(nib << 28) >> 28;
 }
 
-// OHWI codes -> int8 [n_pad][taps][c_pad], zero padded (K-major rows for the B operand).
+// OHWI codes -> int8 [n_pad][taps][c_pad], zero padded (K-major rows for the B operand).  The c
+// positions of a tap are c / cs runs of cs bytes, of which the first c_src come from the source
+// tensor (layers run over an im2col matrix pad every source tap from c_src to cs bytes; otherwise
+// cs = c_src = c).
 __global__ void __launch_bounds__(kPrepThreads)
-prepack_tc_kernel(const void* __restrict__ w, int wkind, int n, int taps, int c, int n_pad, int c_pad, int8_t* __restrict__ out)
+prepack_tc_kernel(const void* __restrict__ w, int wkind, int n, int taps, int c, int n_pad, int c_pad, int8_t* __restrict__ out,
+                  int cs, int c_src)
 {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
     const int64_t row_len = static_cast<int64_t>(taps) * c_pad;
     if (i >= n_pad * row_len) return;
     const int64_t row = i / row_len, rem = i - row * row_len;
     const int tap = static_cast<int>(rem / c_pad), ch = static_cast<int>(rem - static_cast<int64_t>(tap) * c_pad);
-    out[i] = (row < n && ch < c) ? static_cast<int8_t>(api_code_s8(w, wkind, row, static_cast<int64_t>(tap) * c + ch, static_cast<int64_t>(taps) * c)) : 0;
+    int8_t v = 0;
+    if (row < n && ch < c) {
+        const int runs = c / cs, sub = ch / cs, cc = ch - sub * cs;
+        if (cc < c_src)
+            v = static_cast<int8_t>(api_code_s8(w, wkind, row, (static_cast<int64_t>(tap) * runs + sub) * c_src + cc,
+                                                static_cast<int64_t>(taps) * runs * c_src));
+    }
+    out[i] = v;
 }
 
 // Weight sums per border class.  Class = 4 * rowclass + colclass, each a 2-bit mask
@@ -798,42 +809,88 @@ stride_gather_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, i
 }
 
 // Explicit im2col for layers with a short reduction (3-channel stem convolutions, strided 3x3):
-// row p of `out` holds the kh*kw*c window bytes of output pixel p in OHWI order, out-of-image taps
-// as the code z_x (real zero, Section 2.1) and the tail up to the pitch as 0.  The layer then runs
-// as a pointwise layer over this matrix on the tensor cores.  One thread per 16 output bytes;
-// `lut[k]` gives (dy << 24 | dx << 16 | channel) for window byte k.
+// row p of `out` holds the window of output pixel p, filter rows first, then filter columns, then
+// `cs` bytes per tap: the c channels and, where c is not a multiple of 4, padding bytes up to
+// cs = roundup4(c) (the weights of the padding positions are zero).  Out-of-image taps and the
+// padding bytes hold the code z_x (real zero, Section 2.1); the tail of the row up to its pitch is 0.
+// The layer then runs as a pointwise layer over this matrix on the tensor cores.
+//
+// One CTA makes the rows of `tp` consecutive output pixels of one output row.  It first copies the
+// kh input rows it needs into shared memory, cs bytes per pixel; a window is then kh contiguous runs
+// of kw*cs bytes there, and every 32-bit word of an output row is one aligned word of shared memory.
+// The CTA writes its rows with fully coalesced 16-byte stores.
 __global__ void __launch_bounds__(kPrepThreads)
-im2col_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, const uint32_t* __restrict__ lut, int h, int w,
-              int pitch, int stride, int pad, int oh, int ow, int64_t pixels, int k_total, int k_pitch, int zx)
+im2col_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, int h, int w, int c, int cs, int pitch, int kh,
+              int kw, int stride, int pad, int oh, int ow, int tp, int k_total, int k_pitch, int zx)
 {
-    extern __shared__ uint32_t lut_s[];
-    for (int i = threadIdx.x; i < k_pitch; i += kPrepThreads) lut_s[i] = i < k_total ? lut[i] : 0u;
-    __syncthreads();
-    const int chunks = k_pitch >> 4;
-    const int64_t t = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
-    if (t >= pixels * chunks) return;
-    const int ck = static_cast<int>(t % chunks);
-    int64_t p = t / chunks;
-    const int ox = static_cast<int>(p % ow); p /= ow;
-    const int oy = static_cast<int>(p % oh);
-    const int64_t b = p / oh;
-    const int iy0 = oy * stride - pad, ix0 = ox * stride - pad;
-    const uint8_t* img = x + b * h * w * pitch;
-    uint32_t words[4] = {0, 0, 0, 0};
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        const int k = 16 * ck + j;
-        uint32_t v = 0;
-        if (k < k_total) {
-            const uint32_t e = lut_s[k];
-            const int iy = iy0 + static_cast<int>(e >> 24), ix = ix0 + static_cast<int>((e >> 16) & 0xff);
-            v = (iy >= 0 && iy < h && ix >= 0 && ix < w)
-                    ? img[(static_cast<int64_t>(iy) * w + ix) * pitch + (e & 0xffff)]
-                    : static_cast<uint32_t>(zx);
-        }
-        words[j >> 2] |= v << (8 * (j & 3));
+    extern __shared__ __align__(16) uint8_t im_s[];
+    const int kwords = k_pitch >> 2;
+    uint16_t* const off_s = reinterpret_cast<uint16_t*>(im_s);          // [kwords] word offset of output word k in the staged rows
+    uint32_t* const rows_s = reinterpret_cast<uint32_t*>(im_s + ((2 * kwords + 15) & ~15));   // [kh][wt][cs / 4]
+    const int wq = cs >> 2;                                              // words per pixel
+    const int wt = (tp - 1) * stride + kw;                               // input pixels per staged row
+    const int seg_w = (ow + tp - 1) / tp;
+    int blk = blockIdx.x;
+    const int seg = blk % seg_w; blk /= seg_w;
+    const int oy = blk % oh;
+    const int64_t b = blk / oh;
+    const int ox0 = seg * tp;
+    const int npx = min(tp, ow - ox0);
+    const int iy0 = oy * stride - pad, ix0 = ox0 * stride - pad;
+    const uint32_t zx4 = 0x01010101u * static_cast<uint32_t>(zx);
+
+    const int run = kw * wq;                                             // words of one filter row
+    for (int k = threadIdx.x; k < kwords; k += kPrepThreads) {
+        const int dy = k / run;
+        off_s[k] = static_cast<uint16_t>(4 * k < k_total ? dy * wt * wq + (k - dy * run) : 0);
     }
-    reinterpret_cast<uint4*>(out)[t] = make_uint4(words[0], words[1], words[2], words[3]);
+    // stage the input rows: one thread per word
+    const uint8_t* const img = x + b * h * w * pitch;
+    const int row_words = wt * wq;
+    for (int dy = 0; dy < kh; ++dy) {
+        const int iy = iy0 + dy;
+        const bool row_in = iy >= 0 && iy < h;
+        for (int e = threadIdx.x; e < row_words; e += kPrepThreads) {
+            const int px = wq == 1 ? e : e / wq, q = e - px * wq;
+            const int ix = ix0 + px;
+            uint32_t v = zx4;
+            if (row_in && ix >= 0 && ix < w) {
+                v = __ldg(reinterpret_cast<const uint32_t*>(img + (static_cast<int64_t>(iy) * w + ix) * pitch) + q);
+                const int live = c - 4 * q;                              // real channel bytes in this word
+                if (live < 4) {
+                    const uint32_t keep = 0xffffffffu >> (8 * (4 - live));
+                    v = (v & keep) | (zx4 & ~keep);
+                }
+            }
+            rows_s[dy * row_words + e] = v;
+        }
+    }
+    __syncthreads();
+
+    const int chunks = k_pitch >> 4;
+    const int64_t row0 = (b * oh + oy) * ow + ox0;
+    uint4* const dst = reinterpret_cast<uint4*>(out + row0 * k_pitch);
+    const int tail_words = (k_total >> 2);                               // words at and beyond this index are zero
+    int ck = threadIdx.x % chunks, p = threadIdx.x / chunks;
+    const int step_p = kPrepThreads / chunks, step_ck = kPrepThreads - step_p * chunks;
+    for (int i = threadIdx.x; i < npx * chunks; i += kPrepThreads) {
+        const uint32_t* const win = rows_s + p * stride * wq;
+        const uint2 o = *reinterpret_cast<const uint2*>(off_s + 4 * ck);
+        uint32_t w0 = win[o.x & 0xffffu], w1 = win[o.x >> 16], w2 = win[o.y & 0xffffu], w3 = win[o.y >> 16];
+        if (4 * ck + 4 > tail_words) {                                   // the row's last chunk: zero tail
+            if (4 * ck + 0 >= tail_words) w0 = 0;
+            if (4 * ck + 1 >= tail_words) w1 = 0;
+            if (4 * ck + 2 >= tail_words) w2 = 0;
+            if (4 * ck + 3 >= tail_words) w3 = 0;
+        }
+        dst[i] = make_uint4(w0, w1, w2, w3);
+        p += step_p;
+        ck += step_ck;
+        if (ck >= chunks) {
+            ck -= chunks;
+            ++p;
+        }
+    }
 }
 
 }  // namespace
@@ -845,7 +902,7 @@ struct qtz_tc_state {
     TcArgs args{};
     qtz_conv_desc eff{};       // the layer as the kernel sees it (im2col layers become pointwise over the window matrix)
     bool im2col = false;
-    uint32_t* lut = nullptr;   // im2col: window byte -> (dy, dx, channel)
+    int cs = 0;                // im2col: bytes per tap in the window matrix (channels rounded up to 4)
     CUtensorMap map_b{};
     int8_t* w_packed = nullptr;
     int32_t* xsum = nullptr;
@@ -936,7 +993,6 @@ void qtz_tc_release(qtz_plan* p)
 {
     if (!p->tc) return;
     cudaFree(p->tc->w_packed);
-    cudaFree(p->tc->lut);
     cudaFree(p->tc->xsum);
     delete p->tc;
     p->tc = nullptr;
@@ -956,18 +1012,11 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     t->im2col = wants_im2col(p->d);
     if (t->im2col) {
         const qtz_conv_desc& o = p->d;
-        const int k_total = o.kh * o.kw * o.c;
+        t->cs = (o.c + 3) / 4 * 4;
+        const int k_total = o.kh * o.kw * t->cs;
         t->eff.h = p->oh; t->eff.w = p->ow;
         t->eff.c = k_total; t->eff.c_pitch_in = (k_total + 15) / 16 * 16;
         t->eff.kh = t->eff.kw = 1; t->eff.stride = 1; t->eff.pad = 0;
-        std::vector<uint32_t> lut(static_cast<size_t>(k_total));
-        for (int k = 0; k < k_total; ++k) {
-            const int tap = k / o.c, ch = k - tap * o.c;
-            lut[k] = (static_cast<uint32_t>(tap / o.kw) << 24) | (static_cast<uint32_t>(tap % o.kw) << 16) | static_cast<uint32_t>(ch);
-        }
-        QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->lut), sizeof(uint32_t) * lut.size()));
-        QTZ_CUDA(h, cudaMemcpyAsync(t->lut, lut.data(), sizeof(uint32_t) * lut.size(), cudaMemcpyHostToDevice, st));
-        QTZ_CUDA(h, cudaStreamSynchronize(st));   // the staging vector goes out of scope
     }
     const qtz_conv_desc& d = t->eff;
     TcArgs& a = t->args;
@@ -1062,7 +1111,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     const int64_t wbytes = static_cast<int64_t>(t->n_pad) * a.taps * a.c_pad;
     QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->w_packed), static_cast<size_t>(wbytes)));
     prepack_tc_kernel<<<static_cast<unsigned>((wbytes + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
-        w_q_dev, d.wkind, d.n, a.taps, d.c, t->n_pad, a.c_pad, t->w_packed);
+        w_q_dev, d.wkind, d.n, a.taps, d.c, t->n_pad, a.c_pad, t->w_packed, t->im2col ? t->cs : d.c, t->im2col ? p->d.c : d.c);
     QTZ_LAUNCH_CHECK(h, "prepack_tc_kernel");
     QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->wsum), sizeof(int32_t) * a.ncls * d.n));
     class_sums_kernel<<<d.n, kPrepThreads, 0, st>>>(t->w_packed, d.n, a.taps, a.kw, a.c_pad, a.ncls, p->wsum);
@@ -1116,10 +1165,14 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     const uint8_t* xin = x;
     if (t->im2col) {
         const qtz_conv_desc& o = p->d;
-        const int64_t work = t->in_pixels * (d.c_pitch_in >> 4);
-        im2col_kernel<<<static_cast<unsigned>((work + kPrepThreads - 1) / kPrepThreads), kPrepThreads,
-                        sizeof(uint32_t) * d.c_pitch_in, st>>>(x, p->x_gather, t->lut, o.h, o.w, o.c_pitch_in, o.stride, o.pad,
-                                                               p->oh, p->ow, t->in_pixels, d.c, d.c_pitch_in, x_zp);
+        // pixels per CTA: as many as keep the staged input rows within 40 KB
+        int tp = 64;
+        while (tp > 8 && static_cast<int64_t>(o.kh) * ((tp - 1) * o.stride + o.kw) * t->cs > 40 * 1024) tp >>= 1;
+        const size_t smem = ((static_cast<size_t>(d.c_pitch_in) / 2 + 15) & ~static_cast<size_t>(15)) +
+                            static_cast<size_t>(o.kh) * ((tp - 1) * o.stride + o.kw) * t->cs;
+        const int64_t blocks = static_cast<int64_t>(o.batch) * p->oh * ((p->ow + tp - 1) / tp);
+        im2col_kernel<<<static_cast<unsigned>(blocks), kPrepThreads, smem, st>>>(
+            x, p->x_gather, o.h, o.w, o.c, t->cs, o.c_pitch_in, o.kh, o.kw, o.stride, o.pad, p->oh, p->ow, tp, d.c, d.c_pitch_in, x_zp);
         QTZ_LAUNCH_CHECK(h, "im2col_kernel");
         xin = p->x_gather;
     } else if (pw && d.stride > 1) {
