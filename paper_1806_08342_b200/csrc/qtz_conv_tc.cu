@@ -80,7 +80,7 @@ struct TcArgs {
     int32_t m_tiles, group_m;               // rasterisation: groups of group_m pixel tiles x all n tiles
     uint32_t num_tiles;
     int32_t W, H, B;                        // output extent (2-D case: W = number of pixels)
-    int32_t taps, kw, pad;
+    int32_t taps, kw, pad, cstride;          // cstride: input steps per output pixel (row-window layers; else 1)
     int32_t kb_per_tap, c_pad;
     int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
     int32_t obuf;                           // staging boxes per epilogue group (1..4)
@@ -338,7 +338,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (leader) {
                         const uint32_t dst_a = base + L.a_off + stage * L.a_stage + j * L.a_blk;
                         if (a.is4d)
-                            tma_load_4d(dst_a, &map_a, full, kc, w0 + tap_x - a.pad, h0 + tap_y - a.pad, b0);
+                            tma_load_4d(dst_a, &map_a, full, kc, w0 * a.cstride + tap_x - a.pad, h0 * a.cstride + tap_y - a.pad, b0);
                         else
                             tma_load_2d(dst_a, &map_a, full, kc, w0);
                         if (!wres) tma_load_2d(base + L.b_off + stage * L.b_stage + j * L.b_blk, &map_b, full, kcol + kc, nrow);
@@ -808,6 +808,58 @@ stride_gather_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, i
     reinterpret_cast<uint4*>(out)[t] = v;
 }
 
+// Row-window layers (kw pixels of at most 16 channel bytes each: image stems).  The input is copied
+// once into a frame of z_x codes (real zero, Section 2.1) with 16 bytes per pixel; eight consecutive
+// pixels of a frame row are then 128 contiguous bytes, i.e. one filter row of an output pixel's
+// window plus zero-weight positions, and a tensor map whose pixel dimension overlaps itself hands
+// those runs to the tensor cores as K-major operand rows.  No border classes: padding is data.
+__global__ void __launch_bounds__(kPrepThreads)
+pad_copy_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ xp, int batch, int h, int w, int c, int hp, int wp,
+                int pad, int zx)
+{
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
+    if (i >= static_cast<int64_t>(batch) * hp * wp) return;
+    const int xq = static_cast<int>(i % wp);
+    const int64_t r = i / wp;
+    const int yp = static_cast<int>(r % hp);
+    const int64_t b = r / hp;
+    const int iy = yp - pad, ix = xq - pad;
+    const uint32_t zx4 = 0x01010101u * static_cast<uint32_t>(zx);
+    uint4 v = make_uint4(zx4, zx4, zx4, zx4);
+    if (iy >= 0 && iy < h && ix >= 0 && ix < w) {
+        const uint4 s = __ldg(reinterpret_cast<const uint4*>(x) + (b * h + iy) * w + ix);
+        uint32_t words[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int live = c - 4 * q;              // real channel bytes in this word
+            if (live <= 0) words[q] = zx4;
+            else if (live < 4) {
+                const uint32_t keep = 0xffffffffu >> (8 * (4 - live));
+                words[q] = (words[q] & keep) | (zx4 & ~keep);
+            }
+        }
+        v = make_uint4(words[0], words[1], words[2], words[3]);
+    }
+    reinterpret_cast<uint4*>(xp)[i] = v;
+}
+
+// OHWI codes -> int8 [n_pad][kh][8 pixels][16 bytes]: filter row dy of output channel `row` laid over
+// the 128-byte run of frame pixels it meets; positions beyond kw pixels or c channels weigh zero.
+__global__ void __launch_bounds__(kPrepThreads)
+prepack_rowwin_kernel(const void* __restrict__ w, int wkind, int n, int kh, int kw, int c, int n_pad, int8_t* __restrict__ out)
+{
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
+    if (i >= static_cast<int64_t>(n_pad) * kh * 128) return;
+    const int byte = static_cast<int>(i & 127);
+    const int dy = static_cast<int>((i >> 7) % kh);
+    const int64_t row = (i >> 7) / kh;
+    const int px = byte >> 4, ch = byte & 15;
+    int8_t v = 0;
+    if (row < n && px < kw && ch < c)
+        v = static_cast<int8_t>(api_code_s8(w, wkind, row, (static_cast<int64_t>(dy) * kw + px) * c + ch, static_cast<int64_t>(kh) * kw * c));
+    out[i] = v;
+}
+
 // Explicit im2col for layers with a short reduction (3-channel stem convolutions, strided 3x3):
 // row p of `out` holds the window of output pixel p, filter rows first, then filter columns, then
 // `cs` bytes per tap: the c channels and, where c is not a multiple of 4, padding bytes up to
@@ -902,6 +954,8 @@ struct qtz_tc_state {
     TcArgs args{};
     qtz_conv_desc eff{};       // the layer as the kernel sees it (im2col layers become pointwise over the window matrix)
     bool im2col = false;
+    bool rowwin = false;       // row-window layer: padded frame + overlapping tensor map (see pad_copy_kernel)
+    int hp = 0, wp = 0;        // its frame extent
     int cs = 0;                // im2col: bytes per tap in the window matrix (channels rounded up to 4)
     CUtensorMap map_b{};
     int8_t* w_packed = nullptr;
@@ -952,6 +1006,29 @@ bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims
 
 bool is_pointwise(const qtz_conv_desc& d) { return d.kh == 1 && d.kw == 1 && d.pad == 0; }
 bool is_3x3(const qtz_conv_desc& d) { return d.kh == 3 && d.kw == 3 && d.pad == 1 && d.stride == 1; }
+
+// Row-window layers: see pad_copy_kernel.  Symmetric weights only (a zero-weight position must also
+// be a zero in the integer arithmetic).
+bool wants_rowwin(const qtz_conv_desc& d, int w_zp_signed)
+{
+    if (is_pointwise(d) || (is_3x3(d) && d.c >= 8)) return false;
+    return d.c_pitch_in == 16 && d.kw <= 8 && d.kh <= 16 && d.stride <= 4 && w_zp_signed == 0;
+}
+
+// Tensor map of the padded frame [batch][hp][wp][16 B]: dimension 0 is a run of 128 bytes (eight
+// pixels), dimension 1 the pixel the run starts at (16-byte steps, so consecutive runs overlap),
+// then frame rows and images.  The box takes every `stride`-th run and row.
+bool encode_rowwin_map(CUtensorMap* m, const void* base, int batch, int hp, int wp, int stride, int tw, int th, int tb)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t gd[4] = {128, static_cast<cuuint64_t>(wp - 7), static_cast<cuuint64_t>(hp), static_cast<cuuint64_t>(batch)};
+    cuuint64_t gs[3] = {16, static_cast<cuuint64_t>(wp) * 16, static_cast<cuuint64_t>(hp) * wp * 16};
+    cuuint32_t bx[4] = {128, static_cast<cuuint32_t>(tw * stride), static_cast<cuuint32_t>(th * stride), static_cast<cuuint32_t>(tb)};
+    cuuint32_t es[4] = {1, static_cast<cuuint32_t>(stride), static_cast<cuuint32_t>(stride), 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 }  // namespace
 
@@ -1009,7 +1086,8 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     if (!t) return QTZ_ERR_INVALID_ARG;
     p->tc = t;
     t->eff = p->d;
-    t->im2col = wants_im2col(p->d);
+    t->rowwin = wants_rowwin(p->d, p->w_zp_signed);
+    t->im2col = !t->rowwin && wants_im2col(p->d);
     if (t->im2col) {
         const qtz_conv_desc& o = p->d;
         t->cs = (o.c + 3) / 4 * 4;
@@ -1021,9 +1099,15 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     const qtz_conv_desc& d = t->eff;
     TcArgs& a = t->args;
     const bool pw = is_pointwise(d);
-    a.taps = pw ? 1 : 9;
-    a.kw = pw ? 1 : 3;
-    a.pad = pw ? 0 : 1;
+    const bool rw = t->rowwin;
+    a.taps = rw ? d.kh : (pw ? 1 : 9);       // row-window layers: one "tap" per filter row
+    a.kw = (pw || rw) ? 1 : 3;
+    a.pad = (pw || rw) ? 0 : 1;
+    a.cstride = rw ? d.stride : 1;
+    if (rw) {
+        t->hp = d.h + 2 * d.pad;
+        t->wp = std::max(d.w + 2 * d.pad, (p->ow - 1) * d.stride + 8);
+    }
     a.N = d.n;
     a.B = d.batch;
     a.H = p->oh;
@@ -1033,8 +1117,8 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     t->in_pixels = static_cast<int64_t>(d.batch) * p->oh * p->ow;
 
     // K blocking: the widest swizzle the channel count fills reasonably
-    a.BK = d.c > 64 ? 128 : (d.c > 32 ? 64 : 32);
-    a.c_pad = (d.c + a.BK - 1) / a.BK * a.BK;
+    a.BK = (rw || d.c > 64) ? 128 : (d.c > 32 ? 64 : 32);
+    a.c_pad = rw ? 128 : (d.c + a.BK - 1) / a.BK * a.BK;
     a.kb_per_tap = a.c_pad / a.BK;
     // N tiling: as few tiles as possible, each a multiple of 32 columns
     a.n_tiles = (d.n + 255) / 256;
@@ -1046,7 +1130,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.n_acc = std::min(kMaxAcc, kTmemCols / a.BN);
     a.acc_stride = a.BN;
     t->n_pad = a.n_tiles * a.BN;
-    a.ncls = pw ? 1 : kMaxCls;
+    a.ncls = (pw || rw) ? 1 : kMaxCls;
 
     // pixel tiling
     if (pw) {
@@ -1064,8 +1148,9 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     } else {
         a.is4d = 1;
         int64_t best_tiles = INT64_MAX;
-        for (int tw = 1; tw <= std::min(a.W, kTileM); ++tw)
-            for (int th = 1; th <= std::min(a.H, kTileM / tw); ++th) {
+        const int box_max = 256 / a.cstride;     // a box dimension holds at most 256 elements, strided ones included
+        for (int tw = 1; tw <= std::min(std::min(a.W, kTileM), box_max); ++tw)
+            for (int th = 1; th <= std::min(std::min(a.H, kTileM / tw), box_max); ++th) {
                 const int tb = std::min(a.B, kTileM / (tw * th));
                 const int64_t tiles = static_cast<int64_t>((a.W + tw - 1) / tw) * ((a.H + th - 1) / th) * ((a.B + tb - 1) / tb);
                 if (tiles < best_tiles || (tiles == best_tiles && tw > a.tw)) {
@@ -1110,17 +1195,32 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     // weights: re-lay, then the per-class sums
     const int64_t wbytes = static_cast<int64_t>(t->n_pad) * a.taps * a.c_pad;
     QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->w_packed), static_cast<size_t>(wbytes)));
-    prepack_tc_kernel<<<static_cast<unsigned>((wbytes + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
-        w_q_dev, d.wkind, d.n, a.taps, d.c, t->n_pad, a.c_pad, t->w_packed, t->im2col ? t->cs : d.c, t->im2col ? p->d.c : d.c);
+    if (rw)
+        prepack_rowwin_kernel<<<static_cast<unsigned>((wbytes + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
+            w_q_dev, d.wkind, d.n, d.kh, d.kw, d.c, t->n_pad, t->w_packed);
+    else
+        prepack_tc_kernel<<<static_cast<unsigned>((wbytes + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
+            w_q_dev, d.wkind, d.n, a.taps, d.c, t->n_pad, a.c_pad, t->w_packed, t->im2col ? t->cs : d.c, t->im2col ? p->d.c : d.c);
     QTZ_LAUNCH_CHECK(h, "prepack_tc_kernel");
     QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->wsum), sizeof(int32_t) * a.ncls * d.n));
-    class_sums_kernel<<<d.n, kPrepThreads, 0, st>>>(t->w_packed, d.n, a.taps, a.kw, a.c_pad, a.ncls, p->wsum);
+    if (rw)   // one class, the whole packed row as a single run
+        class_sums_kernel<<<d.n, kPrepThreads, 0, st>>>(t->w_packed, d.n, 1, 1, a.taps * a.c_pad, 1, p->wsum);
+    else
+        class_sums_kernel<<<d.n, kPrepThreads, 0, st>>>(t->w_packed, d.n, a.taps, a.kw, a.c_pad, a.ncls, p->wsum);
     QTZ_LAUNCH_CHECK(h, "class_sums_kernel");
 
     if (p->w_zp_signed != 0)
         QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->xsum), sizeof(int32_t) * static_cast<size_t>(t->in_pixels)));
     if ((pw && d.stride > 1) || t->im2col)
         QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->x_gather), static_cast<size_t>(t->in_pixels) * d.c_pitch_in));
+    if (rw) {
+        QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->x_gather), static_cast<size_t>(d.batch) * t->hp * t->wp * 16));
+        CUtensorMap probe;
+        if (!encode_rowwin_map(&probe, p->x_gather, d.batch, t->hp, t->wp, d.stride, a.tw, a.th, a.tb)) {
+            h->last_error = "cuTensorMapEncodeTiled refused the overlapping row-window map";
+            return QTZ_ERR_UNSUPPORTED;
+        }
+    }
 
     // the weight map never changes
     {
@@ -1163,7 +1263,13 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     const bool pw = is_pointwise(d);
 
     const uint8_t* xin = x;
-    if (t->im2col) {
+    if (t->rowwin) {
+        const int64_t work = static_cast<int64_t>(d.batch) * t->hp * t->wp;
+        pad_copy_kernel<<<static_cast<unsigned>((work + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
+            x, p->x_gather, d.batch, d.h, d.w, d.c, t->hp, t->wp, d.pad, x_zp);
+        QTZ_LAUNCH_CHECK(h, "pad_copy_kernel");
+        xin = p->x_gather;
+    } else if (t->im2col) {
         const qtz_conv_desc& o = p->d;
         // pixels per CTA: as many as keep the staged input rows within 40 KB
         int tp = 64;
@@ -1190,7 +1296,9 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
 
     CUtensorMap map_a, map_y;
     const uint64_t pitch = static_cast<uint64_t>(d.c_pitch_in);
-    if (pw) {
+    if (t->rowwin) {
+        if (!encode_rowwin_map(&map_a, xin, d.batch, t->hp, t->wp, d.stride, a.tw, a.th, a.tb)) return QTZ_ERR_CUDA;
+    } else if (pw) {
         const uint64_t dims[2] = {static_cast<uint64_t>(d.c), static_cast<uint64_t>(t->in_pixels)};
         const uint64_t strides[1] = {pitch};
         const uint32_t box[2] = {static_cast<uint32_t>(a.BK), static_cast<uint32_t>(kTileM)};
