@@ -80,7 +80,7 @@ struct TcArgs {
     int32_t m_tiles, group_m;               // rasterisation: groups of group_m pixel tiles x all n tiles
     uint32_t num_tiles;
     int32_t W, H, B;                        // output extent (2-D case: W = number of pixels)
-    int32_t taps, kw, pad, cstride;          // cstride: input steps per output pixel (row-window layers; else 1)
+    int32_t taps, kw, pad, cstride;          // cstride > 0: row-window layer with that convolution stride (else 0)
     int32_t kb_per_tap, c_pad;
     int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
     int32_t obuf;                           // staging boxes per epilogue group (1..4)
@@ -325,6 +325,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             tile_origin(a, m_tile, w0, h0, b0);
             const int nrow = n_tile * a.BN;
             int tap_x = 0, tap_y = 0, kcol = 0, kc = 0;   // filter tap of the next K block, its first weight column, channel offset
+            int row_q = 0, row_r = 0;                     // row-window layers: tap_y split by the stride
             for (int st = 0; st < nst; ++st) {
                 if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget, 64u)) ||
                     *abort_flag != 0) {
@@ -338,7 +339,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (leader) {
                         const uint32_t dst_a = base + L.a_off + stage * L.a_stage + j * L.a_blk;
                         if (a.is4d)
-                            tma_load_4d(dst_a, &map_a, full, kc, w0 * a.cstride + tap_x - a.pad, h0 * a.cstride + tap_y - a.pad, b0);
+                            if (a.cstride > 0)   // frame row tap_y = cstride * row_q + row_r; the map splits rows the same way
+                                tma_load_5d(dst_a, &map_a, full, 0, w0, h0 + row_q, row_r, b0);
+                            else
+                                tma_load_4d(dst_a, &map_a, full, kc, w0 + tap_x - a.pad, h0 + tap_y - a.pad, b0);
                         else
                             tma_load_2d(dst_a, &map_a, full, kc, w0);
                         if (!wres) tma_load_2d(base + L.b_off + stage * L.b_stage + j * L.b_blk, &map_b, full, kcol + kc, nrow);
@@ -350,6 +354,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         if (++tap_x == a.kw) {
                             tap_x = 0;
                             ++tap_y;
+                            if (++row_r == a.cstride) {
+                                row_r = 0;
+                                ++row_q;
+                            }
                         }
                     }
                 }
@@ -1015,18 +1023,21 @@ bool wants_rowwin(const qtz_conv_desc& d, int w_zp_signed)
     return d.c_pitch_in == 16 && d.kw <= 8 && d.kh <= 16 && d.stride <= 4 && w_zp_signed == 0;
 }
 
-// Tensor map of the padded frame [batch][hp][wp][16 B]: dimension 0 is a run of 128 bytes (eight
-// pixels), dimension 1 the pixel the run starts at (16-byte steps, so consecutive runs overlap),
-// then frame rows and images.  The box takes every `stride`-th run and row.
+// Tensor map of the padded frame [batch][hp][wp][16 B] for convolution stride s: dimension 0 is a
+// run of 128 bytes (eight pixels), dimension 1 the output column (its run starts s pixels after the
+// previous one, so runs overlap), dimension 2 frame row / s, dimension 3 frame row mod s, dimension
+// 4 the image.  hp is a multiple of s.
 bool encode_rowwin_map(CUtensorMap* m, const void* base, int batch, int hp, int wp, int stride, int tw, int th, int tb)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    cuuint64_t gd[4] = {128, static_cast<cuuint64_t>(wp - 7), static_cast<cuuint64_t>(hp), static_cast<cuuint64_t>(batch)};
-    cuuint64_t gs[3] = {16, static_cast<cuuint64_t>(wp) * 16, static_cast<cuuint64_t>(hp) * wp * 16};
-    cuuint32_t bx[4] = {128, static_cast<cuuint32_t>(tw * stride), static_cast<cuuint32_t>(th * stride), static_cast<cuuint32_t>(tb)};
-    cuuint32_t es[4] = {1, static_cast<cuuint32_t>(stride), static_cast<cuuint32_t>(stride), 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    const cuuint64_t s = static_cast<cuuint64_t>(stride);
+    cuuint64_t gd[5] = {128, static_cast<cuuint64_t>((wp - 8) / stride + 1), static_cast<cuuint64_t>(hp / stride), s,
+                        static_cast<cuuint64_t>(batch)};
+    cuuint64_t gs[4] = {s * 16, s * wp * 16, static_cast<cuuint64_t>(wp) * 16, static_cast<cuuint64_t>(hp) * wp * 16};
+    cuuint32_t bx[5] = {128, static_cast<cuuint32_t>(tw), static_cast<cuuint32_t>(th), 1, static_cast<cuuint32_t>(tb)};
+    cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 5, const_cast<void*>(base), gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -1103,9 +1114,9 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.taps = rw ? d.kh : (pw ? 1 : 9);       // row-window layers: one "tap" per filter row
     a.kw = (pw || rw) ? 1 : 3;
     a.pad = (pw || rw) ? 0 : 1;
-    a.cstride = rw ? d.stride : 1;
+    a.cstride = rw ? d.stride : 0;
     if (rw) {
-        t->hp = d.h + 2 * d.pad;
+        t->hp = (d.h + 2 * d.pad + d.stride - 1) / d.stride * d.stride;
         t->wp = std::max(d.w + 2 * d.pad, (p->ow - 1) * d.stride + 8);
     }
     a.N = d.n;
@@ -1148,9 +1159,8 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     } else {
         a.is4d = 1;
         int64_t best_tiles = INT64_MAX;
-        const int box_max = 256 / a.cstride;     // a box dimension holds at most 256 elements, strided ones included
-        for (int tw = 1; tw <= std::min(std::min(a.W, kTileM), box_max); ++tw)
-            for (int th = 1; th <= std::min(std::min(a.H, kTileM / tw), box_max); ++th) {
+        for (int tw = 1; tw <= std::min(a.W, kTileM); ++tw)
+            for (int th = 1; th <= std::min(a.H, kTileM / tw); ++th) {
                 const int tb = std::min(a.B, kTileM / (tw * th));
                 const int64_t tiles = static_cast<int64_t>((a.W + tw - 1) / tw) * ((a.H + th - 1) / th) * ((a.B + tb - 1) / tb);
                 if (tiles < best_tiles || (tiles == best_tiles && tw > a.tw)) {
