@@ -134,7 +134,8 @@ __device__ __forceinline__ void mac_row(const RowState<kStride>& r, const uint32
 struct Requant {
     int32_t m[8];
     int32_t sh[8];      // fast form: r - 32;  general form: r
-    int64_t add[8];     // fast form: 2^(r-1) + ((z_y - act_min) << r)
+    int32_t addhi[8];   // fast form, r >= 33: high word of 2^(r-1) + ((z_y - act_min) << r) (its low word is zero)
+    int64_t add[8];     // fast form, r >= 32: the same constant in full
     uint32_t lo4;       // act_min in every byte
     int32_t span;       // act_max - act_min
     int32_t zy, lo;
@@ -143,14 +144,15 @@ struct Requant {
 // Requantises 8 channels of one pixel and returns them as two packed words.  The clamp is done
 // relative to act_min: max(min(y - act_min, span), 0) is a single instruction, act_min is added
 // back to all four bytes of a packed word at once.
-template <bool kFast>
+template <int kFast>
 __device__ __forceinline__ uint2 requant_pixel(const int32_t (&v)[8], const Requant& q)
 {
     int32_t y[8];
 #pragma unroll
     for (int ch = 0; ch < 8; ++ch) {
-        if (kFast) {   // 32 <= r <= 53: floor((v m + addend) / 2^r) = hi32(v m + addend) >> (r - 32)
-            const int64_t p = static_cast<int64_t>(v[ch]) * q.m[ch] + q.add[ch];
+        if (kFast != 0) {   // 32 (33) <= r <= 53: floor((v m + addend) / 2^r) = hi32(v m + addend) >> (r - 32)
+            const int64_t p = static_cast<int64_t>(v[ch]) * q.m[ch] +
+                              (kFast == 1 ? static_cast<int64_t>(q.addhi[ch]) << 32 : q.add[ch]);
             y[ch] = __vimin_s32_relu(static_cast<int32_t>(p >> 32) >> q.sh[ch], q.span);
         } else {
             const int64_t p = static_cast<int64_t>(v[ch]) * q.m[ch] + (static_cast<int64_t>(1) << (q.sh[ch] - 1));
@@ -178,7 +180,7 @@ __device__ __forceinline__ TileCoord decode_tile(const DwArgs& a, int64_t tile)
     return t;
 }
 
-template <int kStride, bool kAsym, bool kFast>
+template <int kStride, bool kAsym, int kFast>
 __global__ void __launch_bounds__(kDwThreads, 2)
 depthwise3x3_kernel(const __grid_constant__ CUtensorMap map_x, const DwArgs a)
 {
@@ -248,8 +250,9 @@ depthwise3x3_kernel(const __grid_constant__ CUtensorMap map_x, const DwArgs a)
             for (int ch = 0; ch < 8; ++ch) {
                 const int32_t r = a.y_raw ? 40 : __ldg(a.rshift + c0 + ch);   // raw output has no multipliers
                 rq.m[ch] = a.y_raw ? 0 : __ldg(a.mult + c0 + ch);
-                rq.sh[ch] = kFast ? r - 32 : r;
-                rq.add[ch] = kFast ? static_cast<int64_t>(2 * (a.zy - a.act_min) + 1) << (r - 1) : 0;
+                rq.sh[ch] = kFast != 0 ? r - 32 : r;
+                if (kFast == 1) rq.addhi[ch] = (2 * (a.zy - a.act_min) + 1) * (1 << (r - 33));
+                if (kFast == 2) rq.add[ch] = static_cast<int64_t>(2 * (a.zy - a.act_min) + 1) << (r - 1);
                 base[ch] = __ldg(a.bias + c0 + ch) - a.zx * __ldg(a.wsum + c0 + ch) + 9 * a.zx * a.zw;
             }
             loaded_cc = t.cc;
@@ -368,21 +371,26 @@ depthwise3x3_kernel(const __grid_constant__ CUtensorMap map_x, const DwArgs a)
 }
 
 template <int kStride, bool kAsym>
-void launch_variant(bool fast, unsigned blocks, size_t smem, cudaStream_t st, const CUtensorMap& map, const DwArgs& a)
+void launch_variant(int fast, unsigned blocks, size_t smem, cudaStream_t st, const CUtensorMap& map, const DwArgs& a)
 {
-    if (fast)
-        depthwise3x3_kernel<kStride, kAsym, true><<<blocks, kDwThreads, smem, st>>>(map, a);
+    if (fast == 1)
+        depthwise3x3_kernel<kStride, kAsym, 1><<<blocks, kDwThreads, smem, st>>>(map, a);
+    else if (fast == 2)
+        depthwise3x3_kernel<kStride, kAsym, 2><<<blocks, kDwThreads, smem, st>>>(map, a);
     else
-        depthwise3x3_kernel<kStride, kAsym, false><<<blocks, kDwThreads, smem, st>>>(map, a);
+        depthwise3x3_kernel<kStride, kAsym, 0><<<blocks, kDwThreads, smem, st>>>(map, a);
 }
 
 template <int kStride, bool kAsym>
 cudaError_t allow_smem()
 {
-    cudaError_t e = cudaFuncSetAttribute(depthwise3x3_kernel<kStride, kAsym, true>,
+    cudaError_t e = cudaFuncSetAttribute(depthwise3x3_kernel<kStride, kAsym, 0>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemLimit);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(depthwise3x3_kernel<kStride, kAsym, false>,
+        e = cudaFuncSetAttribute(depthwise3x3_kernel<kStride, kAsym, 1>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemLimit);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(depthwise3x3_kernel<kStride, kAsym, 2>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemLimit);
     return e;
 }
@@ -477,7 +485,8 @@ qtz_status qtz_depthwise_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, uin
         p->h->last_error = "cuTensorMapEncodeTiled failed for the depthwise input";
         return QTZ_ERR_CUDA;
     }
-    const bool fast = !raw && p->rshift_min >= 32 && p->rshift_max <= 53;
+    // requantisation form: 1 for right shifts 33..53, 2 for 32..53 (64-bit rounding constant), 0 for any shift
+    const int fast = (raw || p->rshift_max > 53 || p->rshift_min < 32) ? 0 : (p->rshift_min >= 33 ? 1 : 2);
     const bool asym = p->w_zp_signed != 0;
     if (p->ev_start) QTZ_CUDA(p->h, cudaEventRecord(p->ev_start, st));
     const unsigned blocks = static_cast<unsigned>(p->dw->grid);
