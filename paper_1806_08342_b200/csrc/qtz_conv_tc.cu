@@ -81,6 +81,10 @@ struct TcArgs {
     uint32_t num_tiles;
     int32_t W, H, B;                        // output extent (2-D case: W = number of pixels)
     int32_t taps, kw, pad, cstride;          // cstride > 0: row-window layer with that convolution stride (else 0)
+    const uint8_t* frame;                    // row-window layers: the padded frame, its row pitch and rows per image,
+    int64_t frame_row;                       // and the bytes one tile takes from a frame row
+    int32_t frame_rows, seg_bytes;
+    int32_t a_blk;                           // bytes of one activation K block in the ring (0: 128 rows of BK bytes)
     int32_t kb_per_tap, c_pad;
     int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
     int32_t obuf;                           // staging boxes per epilogue group (1..4)
@@ -109,12 +113,13 @@ struct SmemLayout {
 
 // Operand ring (activations, and weights unless all `bres` weight blocks of the layer stay resident),
 // output staging boxes and one set of per-channel tables per epilogue group, barriers.
-__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int groups, int obuf, int bres, int spb)
+__host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int groups, int obuf, int bres, int spb,
+                                                  int a_blk = 0)
 {
     SmemLayout L;
-    L.a_blk = kTileM * BK;                  // one K block of activations / of weights
+    L.a_blk = a_blk > 0 ? a_blk : kTileM * BK;   // one K block of activations (row-window layers: one run of the frame) / of weights
     L.b_blk = BN * BK;
-    L.a_stage = spb * L.a_blk;              // a ring stage holds spb consecutive K blocks
+    L.a_stage = (spb * L.a_blk + 1023u) & ~1023u;   // a ring stage holds spb consecutive K blocks; swizzled tiles behind the ring need 1 KB alignment
     L.b_stage = spb * L.b_blk;
     L.a_off = 0;
     L.b_off = L.a_off + stages * L.a_stage;
@@ -248,7 +253,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
-    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb);
+    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb, a.a_blk);
 
     const uint32_t bar_full = base + L.bar_off;
     const uint32_t bar_empty = bar_full + 8 * kMaxStages;
@@ -303,7 +308,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // cycles per K block, which starves layers with a short reduction.)
         const uint32_t S = static_cast<uint32_t>(a.stages);
         const bool wres = a.bres > 0;
-        const uint32_t tx = static_cast<uint32_t>(a.spb) * static_cast<uint32_t>(a.rows * a.BK + (wres ? 0 : a.BN * a.BK));
+        const uint32_t tx = static_cast<uint32_t>(a.spb) *
+                            static_cast<uint32_t>((a.cstride > 0 ? a.seg_bytes : a.rows * a.BK) + (wres ? 0 : a.BN * a.BK));
         const int nst = kblocks / a.spb;         // ring stages per tile
         uint32_t stage = 0, phase = 0;
         bool failed = false;
@@ -325,7 +331,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             tile_origin(a, m_tile, w0, h0, b0);
             const int nrow = n_tile * a.BN;
             int tap_x = 0, tap_y = 0, kcol = 0, kc = 0;   // filter tap of the next K block, its first weight column, channel offset
-            int row_q = 0, row_r = 0;                     // row-window layers: tap_y split by the stride
+            // row-window layers: the tile is a run of output columns of one output row; filter row tap_y
+            // reads frame row h0 * cstride + tap_y from the byte where the window of column w0 starts
+            const uint8_t* const frame_at =
+                a.cstride > 0 ? a.frame + (static_cast<int64_t>(b0) * a.frame_rows + h0 * a.cstride) * a.frame_row + 16 * w0
+                              : nullptr;
             for (int st = 0; st < nst; ++st) {
                 if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget, 64u)) ||
                     *abort_flag != 0) {
@@ -339,8 +349,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (leader) {
                         const uint32_t dst_a = base + L.a_off + stage * L.a_stage + j * L.a_blk;
                         if (a.is4d)
-                            if (a.cstride > 0)   // frame row tap_y = cstride * row_q + row_r; the map splits rows the same way
-                                tma_load_5d(dst_a, &map_a, full, 0, w0, h0 + row_q, row_r, b0);
+                            if (a.cstride > 0)
+                                bulk_load(dst_a, frame_at + tap_y * a.frame_row, static_cast<uint32_t>(a.seg_bytes), full);
                             else
                                 tma_load_4d(dst_a, &map_a, full, kc, w0 + tap_x - a.pad, h0 + tap_y - a.pad, b0);
                         else
@@ -354,10 +364,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         if (++tap_x == a.kw) {
                             tap_x = 0;
                             ++tap_y;
-                            if (++row_r == a.cstride) {
-                                row_r = 0;
-                                ++row_q;
-                            }
                         }
                     }
                 }
@@ -382,7 +388,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------ MMA issuer --------------------------------
         // Again the whole warp runs the loop and one elected lane issues, so descriptors and TMEM
         // addresses stay warp-uniform.  Only this warp ever issues MMAs.
-        const uint64_t desc_a0 = make_kmajor_desc(base + L.a_off, a.BK);
+        const uint64_t desc_a0 = a.cstride > 0 ? make_sliding_desc(base + L.a_off) : make_kmajor_desc(base + L.a_off, a.BK);
         const uint64_t desc_b0 = make_kmajor_desc(base + L.b_off, a.BK);
         const uint32_t a_step = L.a_stage >> 4, b_step = L.b_stage >> 4;   // descriptor address units
         const uint32_t a_blk = L.a_blk >> 4, b_blk = L.b_blk >> 4;
@@ -817,51 +823,61 @@ stride_gather_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, i
 }
 
 // Row-window layers (kw pixels of at most 16 channel bytes each: image stems).  The input is copied
-// once into a frame of z_x codes (real zero, Section 2.1) with 16 bytes per pixel; eight consecutive
-// pixels of a frame row are then 128 contiguous bytes, i.e. one filter row of an output pixel's
-// window plus zero-weight positions, and a tensor map whose pixel dimension overlaps itself hands
-// those runs to the tensor cores as K-major operand rows.  No border classes: padding is data.
+// once into a frame of z_x codes (real zero, Section 2.1) with fp = 4, 8 or 16 bytes per pixel (the
+// smallest that holds the channels and makes the step between output columns, stride * fp, a
+// multiple of 16 bytes -- here exactly 16); rb / fp consecutive pixels of a frame row (rb = 32, 64
+// or 128 bytes) are then one filter row of an output pixel's window plus zero-weight positions, and
+// the window of the next output column starts 16 bytes later.  A tile (128 output columns of one
+// output row) therefore needs, per filter row, one contiguous run of 16 * 127 + rb frame bytes in
+// shared memory, and the tensor cores read their K-major operand rows straight out of that run
+// through an unswizzled descriptor with a 16-byte row pitch (make_sliding_desc): no window matrix is
+// ever materialised.  No border classes: padding is data.  One thread writes 16 bytes of the frame.
 __global__ void __launch_bounds__(kPrepThreads)
 pad_copy_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ xp, int batch, int h, int w, int c, int hp, int wp,
-                int pad, int zx)
+                int pad, int zx, int fp)
 {
+    const int ppc = 16 / fp;                         // pixels per 16-byte chunk
+    const int chunks = wp / ppc;                     // wp is a multiple of ppc
     const int64_t i = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
-    if (i >= static_cast<int64_t>(batch) * hp * wp) return;
-    const int xq = static_cast<int>(i % wp);
-    const int64_t r = i / wp;
+    if (i >= static_cast<int64_t>(batch) * hp * chunks) return;
+    const int xc = static_cast<int>(i % chunks);
+    const int64_t r = i / chunks;
     const int yp = static_cast<int>(r % hp);
     const int64_t b = r / hp;
-    const int iy = yp - pad, ix = xq - pad;
+    const int iy = yp - pad;
     const uint32_t zx4 = 0x01010101u * static_cast<uint32_t>(zx);
-    uint4 v = make_uint4(zx4, zx4, zx4, zx4);
-    if (iy >= 0 && iy < h && ix >= 0 && ix < w) {
-        const uint4 s = __ldg(reinterpret_cast<const uint4*>(x) + (b * h + iy) * w + ix);
-        uint32_t words[4] = {s.x, s.y, s.z, s.w};
+    uint32_t words[4] = {zx4, zx4, zx4, zx4};
+    const int wpp = fp >> 2;                         // words per frame pixel
+    if (iy >= 0 && iy < h) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int k = 0; k < 4; ++k) {                // word k of the chunk: pixel k / wpp, channel word k % wpp
+            const int j = k / wpp, q = k - j * wpp;
+            const int ix = xc * ppc + j - pad;
             const int live = c - 4 * q;              // real channel bytes in this word
-            if (live <= 0) words[q] = zx4;
-            else if (live < 4) {
+            if (ix < 0 || ix >= w || live <= 0) continue;
+            uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(x) + ((b * h + iy) * w + ix) * 4 + q);   // input pitch: 16 bytes
+            if (live < 4) {
                 const uint32_t keep = 0xffffffffu >> (8 * (4 - live));
-                words[q] = (words[q] & keep) | (zx4 & ~keep);
+                v = (v & keep) | (zx4 & ~keep);
             }
+            words[k] = v;
         }
-        v = make_uint4(words[0], words[1], words[2], words[3]);
     }
-    reinterpret_cast<uint4*>(xp)[i] = v;
+    reinterpret_cast<uint4*>(xp)[i] = make_uint4(words[0], words[1], words[2], words[3]);
 }
 
-// OHWI codes -> int8 [n_pad][kh][8 pixels][16 bytes]: filter row dy of output channel `row` laid over
-// the 128-byte run of frame pixels it meets; positions beyond kw pixels or c channels weigh zero.
+// OHWI codes -> int8 [n_pad][kh][rb / fp pixels][fp bytes]: filter row dy of output channel `row` laid
+// over the rb-byte run of frame pixels it meets; positions beyond kw pixels or c channels weigh zero.
 __global__ void __launch_bounds__(kPrepThreads)
-prepack_rowwin_kernel(const void* __restrict__ w, int wkind, int n, int kh, int kw, int c, int n_pad, int8_t* __restrict__ out)
+prepack_rowwin_kernel(const void* __restrict__ w, int wkind, int n, int kh, int kw, int c, int n_pad, int fp, int rb,
+                      int8_t* __restrict__ out)
 {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
-    if (i >= static_cast<int64_t>(n_pad) * kh * 128) return;
-    const int byte = static_cast<int>(i & 127);
-    const int dy = static_cast<int>((i >> 7) % kh);
-    const int64_t row = (i >> 7) / kh;
-    const int px = byte >> 4, ch = byte & 15;
+    if (i >= static_cast<int64_t>(n_pad) * kh * rb) return;
+    const int byte = static_cast<int>(i % rb);
+    const int dy = static_cast<int>((i / rb) % kh);
+    const int64_t row = (i / rb) / kh;
+    const int px = byte / fp, ch = byte % fp;
     int8_t v = 0;
     if (row < n && px < kw && ch < c)
         v = static_cast<int8_t>(api_code_s8(w, wkind, row, (static_cast<int64_t>(dy) * kw + px) * c + ch, static_cast<int64_t>(kh) * kw * c));
@@ -964,6 +980,7 @@ struct qtz_tc_state {
     bool im2col = false;
     bool rowwin = false;       // row-window layer: padded frame + overlapping tensor map (see pad_copy_kernel)
     int hp = 0, wp = 0;        // its frame extent
+    int fp = 16, rb = 128;     // bytes per frame pixel, bytes of one filter-row run
     int cs = 0;                // im2col: bytes per tap in the window matrix (channels rounded up to 4)
     CUtensorMap map_b{};
     int8_t* w_packed = nullptr;
@@ -1016,29 +1033,28 @@ bool is_pointwise(const qtz_conv_desc& d) { return d.kh == 1 && d.kw == 1 && d.p
 bool is_3x3(const qtz_conv_desc& d) { return d.kh == 3 && d.kw == 3 && d.pad == 1 && d.stride == 1; }
 
 // Row-window layers: see pad_copy_kernel.  Symmetric weights only (a zero-weight position must also
-// be a zero in the integer arithmetic).
+// be a zero in the integer arithmetic).  Frame pixel size: the smallest of 4, 8, 16 bytes that holds
+// the channels and makes stride * fp exactly 16 (the row pitch of the sliding operand descriptor).
+int rowwin_pixel_bytes(const qtz_conv_desc& d)
+{
+    for (int fp = 4; fp <= 16; fp *= 2)
+        if (fp >= d.c && d.stride * fp == 16) return fp;
+    return 0;
+}
+
+int rowwin_run_bytes(const qtz_conv_desc& d)
+{
+    const int fp = rowwin_pixel_bytes(d);
+    if (fp == 0) return 0;
+    for (int rb = 32; rb <= 128; rb *= 2)
+        if (rb >= d.kw * fp) return rb;
+    return 0;
+}
+
 bool wants_rowwin(const qtz_conv_desc& d, int w_zp_signed)
 {
     if (is_pointwise(d) || (is_3x3(d) && d.c >= 8)) return false;
-    return d.c_pitch_in == 16 && d.kw <= 8 && d.kh <= 16 && d.stride <= 4 && w_zp_signed == 0;
-}
-
-// Tensor map of the padded frame [batch][hp][wp][16 B] for convolution stride s: dimension 0 is a
-// run of 128 bytes (eight pixels), dimension 1 the output column (its run starts s pixels after the
-// previous one, so runs overlap), dimension 2 frame row / s, dimension 3 frame row mod s, dimension
-// 4 the image.  hp is a multiple of s.
-bool encode_rowwin_map(CUtensorMap* m, const void* base, int batch, int hp, int wp, int stride, int tw, int th, int tb)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t s = static_cast<cuuint64_t>(stride);
-    cuuint64_t gd[5] = {128, static_cast<cuuint64_t>((wp - 8) / stride + 1), static_cast<cuuint64_t>(hp / stride), s,
-                        static_cast<cuuint64_t>(batch)};
-    cuuint64_t gs[4] = {s * 16, s * wp * 16, static_cast<cuuint64_t>(wp) * 16, static_cast<cuuint64_t>(hp) * wp * 16};
-    cuuint32_t bx[5] = {128, static_cast<cuuint32_t>(tw), static_cast<cuuint32_t>(th), 1, static_cast<cuuint32_t>(tb)};
-    cuuint32_t es[5] = {1, 1, 1, 1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 5, const_cast<void*>(base), gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return d.c_pitch_in == 16 && rowwin_run_bytes(d) != 0 && d.kh <= 16 && d.stride <= 4 && w_zp_signed == 0;
 }
 
 }  // namespace
@@ -1116,8 +1132,11 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.pad = (pw || rw) ? 0 : 1;
     a.cstride = rw ? d.stride : 0;
     if (rw) {
+        t->fp = rowwin_pixel_bytes(d);
+        t->rb = rowwin_run_bytes(d);
+        const int ppc = 16 / t->fp;               // frame rows are whole 16-byte chunks
         t->hp = (d.h + 2 * d.pad + d.stride - 1) / d.stride * d.stride;
-        t->wp = std::max(d.w + 2 * d.pad, (p->ow - 1) * d.stride + 8);
+        t->wp = (std::max(d.w + 2 * d.pad, (p->ow - 1) * d.stride + t->rb / t->fp) + ppc - 1) / ppc * ppc;
     }
     a.N = d.n;
     a.B = d.batch;
@@ -1128,8 +1147,8 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     t->in_pixels = static_cast<int64_t>(d.batch) * p->oh * p->ow;
 
     // K blocking: the widest swizzle the channel count fills reasonably
-    a.BK = (rw || d.c > 64) ? 128 : (d.c > 32 ? 64 : 32);
-    a.c_pad = rw ? 128 : (d.c + a.BK - 1) / a.BK * a.BK;
+    a.BK = rw ? t->rb : (d.c > 64 ? 128 : (d.c > 32 ? 64 : 32));
+    a.c_pad = rw ? t->rb : (d.c + a.BK - 1) / a.BK * a.BK;
     a.kb_per_tap = a.c_pad / a.BK;
     // N tiling: as few tiles as possible, each a multiple of 32 columns
     a.n_tiles = (d.n + 255) / 256;
@@ -1159,15 +1178,22 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     } else {
         a.is4d = 1;
         int64_t best_tiles = INT64_MAX;
-        for (int tw = 1; tw <= std::min(a.W, kTileM); ++tw)
-            for (int th = 1; th <= std::min(a.H, kTileM / tw); ++th) {
-                const int tb = std::min(a.B, kTileM / (tw * th));
-                const int64_t tiles = static_cast<int64_t>((a.W + tw - 1) / tw) * ((a.H + th - 1) / th) * ((a.B + tb - 1) / tb);
-                if (tiles < best_tiles || (tiles == best_tiles && tw > a.tw)) {
-                    best_tiles = tiles;
-                    a.tw = tw; a.th = th; a.tb = tb;
+        if (rw) {
+            // a tile is a run of 128 output columns of one output row (columns beyond the image are
+            // computed from whatever follows in the frame and clipped by the store)
+            a.tw = kTileM; a.th = 1; a.tb = 1;
+            best_tiles = static_cast<int64_t>((a.W + kTileM - 1) / kTileM) * a.H * a.B;
+        } else {
+            for (int tw = 1; tw <= std::min(a.W, kTileM); ++tw)
+                for (int th = 1; th <= std::min(a.H, kTileM / tw); ++th) {
+                    const int tb = std::min(a.B, kTileM / (tw * th));
+                    const int64_t tiles = static_cast<int64_t>((a.W + tw - 1) / tw) * ((a.H + th - 1) / th) * ((a.B + tb - 1) / tb);
+                    if (tiles < best_tiles || (tiles == best_tiles && tw > a.tw)) {
+                        best_tiles = tiles;
+                        a.tw = tw; a.th = th; a.tb = tb;
+                    }
                 }
-            }
+        }
         a.rows = a.tw * a.th * a.tb;
         a.tiles_w = (a.W + a.tw - 1) / a.tw;
         a.tiles_h = (a.H + a.th - 1) / a.th;
@@ -1207,7 +1233,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->w_packed), static_cast<size_t>(wbytes)));
     if (rw)
         prepack_rowwin_kernel<<<static_cast<unsigned>((wbytes + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
-            w_q_dev, d.wkind, d.n, d.kh, d.kw, d.c, t->n_pad, t->w_packed);
+            w_q_dev, d.wkind, d.n, d.kh, d.kw, d.c, t->n_pad, t->fp, t->rb, t->w_packed);
     else
         prepack_tc_kernel<<<static_cast<unsigned>((wbytes + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
             w_q_dev, d.wkind, d.n, a.taps, d.c, t->n_pad, a.c_pad, t->w_packed, t->im2col ? t->cs : d.c, t->im2col ? p->d.c : d.c);
@@ -1224,12 +1250,14 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     if ((pw && d.stride > 1) || t->im2col)
         QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->x_gather), static_cast<size_t>(t->in_pixels) * d.c_pitch_in));
     if (rw) {
-        QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->x_gather), static_cast<size_t>(d.batch) * t->hp * t->wp * 16));
-        CUtensorMap probe;
-        if (!encode_rowwin_map(&probe, p->x_gather, d.batch, t->hp, t->wp, d.stride, a.tw, a.th, a.tb)) {
-            h->last_error = "cuTensorMapEncodeTiled refused the overlapping row-window map";
-            return QTZ_ERR_UNSUPPORTED;
-        }
+        // the last tiles of a row read past its end (into the next row, or into this slack after the last one)
+        a.frame_row = static_cast<int64_t>(t->wp) * t->fp;
+        a.frame_rows = t->hp;
+        a.seg_bytes = 16 * (kTileM - 1) + t->rb;
+        a.a_blk = (a.seg_bytes + 127) / 128 * 128;
+        const size_t slack = static_cast<size_t>(a.tiles_w) * kTileM * 16 + 256;
+        QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->x_gather), static_cast<size_t>(d.batch) * t->hp * a.frame_row + slack));
+        QTZ_CUDA(h, cudaMemsetAsync(p->x_gather, 0, static_cast<size_t>(d.batch) * t->hp * a.frame_row + slack, st));
     }
 
     // the weight map never changes
@@ -1274,9 +1302,9 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
 
     const uint8_t* xin = x;
     if (t->rowwin) {
-        const int64_t work = static_cast<int64_t>(d.batch) * t->hp * t->wp;
+        const int64_t work = static_cast<int64_t>(d.batch) * t->hp * (t->wp * t->fp / 16);
         pad_copy_kernel<<<static_cast<unsigned>((work + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
-            x, p->x_gather, d.batch, d.h, d.w, d.c, t->hp, t->wp, d.pad, x_zp);
+            x, p->x_gather, d.batch, d.h, d.w, d.c, t->hp, t->wp, d.pad, x_zp, t->fp);
         QTZ_LAUNCH_CHECK(h, "pad_copy_kernel");
         xin = p->x_gather;
     } else if (t->im2col) {
@@ -1307,7 +1335,8 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     CUtensorMap map_a, map_y;
     const uint64_t pitch = static_cast<uint64_t>(d.c_pitch_in);
     if (t->rowwin) {
-        if (!encode_rowwin_map(&map_a, xin, d.batch, t->hp, t->wp, d.stride, a.tw, a.th, a.tb)) return QTZ_ERR_CUDA;
+        map_a = t->map_b;   // unused: the producer copies runs of the frame with plain bulk copies
+        a.frame = xin;
     } else if (pw) {
         const uint64_t dims[2] = {static_cast<uint64_t>(d.c), static_cast<uint64_t>(t->in_pixels)};
         const uint64_t strides[1] = {pitch};
@@ -1353,7 +1382,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     auto depth = [&](int groups, int obuf) {
         int st_ = kMaxStages;
         for (; st_ >= 2; --st_)
-            if (make_layout(a.BK, a.BN, st_, a.ncls, a.out_box, groups, obuf, a.bres, a.spb).total <= static_cast<uint32_t>(kSmemBudget)) break;
+            if (make_layout(a.BK, a.BN, st_, a.ncls, a.out_box, groups, obuf, a.bres, a.spb, a.a_blk).total <= static_cast<uint32_t>(kSmemBudget)) break;
         return st_;
     };
     const int kblocks = a.taps * a.kb_per_tap;
@@ -1361,9 +1390,9 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.bres = (a.n_tiles == 1 && kblocks * a.BN * a.BK <= kResidentBMax) ? kblocks : 0;
     // several K blocks share a ring stage (one barrier handshake for all of them) while the stage stays within 32 KB
     auto blocks_per_stage = [&]() {
-        const int blk = kTileM * a.BK + (a.bres > 0 ? 0 : a.BN * a.BK);
+        const int blk = (a.a_blk > 0 ? a.a_blk : kTileM * a.BK) + (a.bres > 0 ? 0 : a.BN * a.BK);
         int best = 1;
-        for (int c = 2; c <= 4; ++c)
+        for (int c = 2; c <= (a.a_blk > 0 ? 8 : 4); ++c)
             if (kblocks % c == 0 && c * blk <= 32 * 1024) best = c;
         return best;
     };
@@ -1392,7 +1421,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.gwarps = a.groups == 4 ? 4 : 8;
     a.stages = depth(a.groups, a.obuf);
     if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
-    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb).total + 1024;
+    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb, a.a_blk).total + 1024;
     // folded form: shifts 32..53 (the high word of the 64-bit sum, shifted on by r - 32)
     // (2: shifts below 32 as well, given that no requantised value can leave 32 bits)
     a.fold = 0;

@@ -82,6 +82,15 @@ __device__ __forceinline__ void prefetch_tensormap(const void* tmap)
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
 
+// Plain (untiled) bulk copy of `bytes` contiguous bytes from global to shared memory; both addresses
+// 16-byte aligned, the size a multiple of 16.  Completes on the mbarrier like a tensor copy.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, uint32_t bar, int x, int y)
 {
     asm volatile(
@@ -233,6 +242,20 @@ __device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t smem_addr, uint32_
     d |= static_cast<uint64_t>(1) << 46;                            // descriptor version of this architecture
     d |= layout << 61;
     return d;
+}
+
+// Descriptor of a K-major operand without swizzle whose row m starts 16 bytes after row m - 1:
+// overlapping rows read straight out of one contiguous run of bytes (element (m, k) at 16 m + k).
+// In the unswizzled canonical layout a core matrix is 8 rows of 16 bytes at a 16-byte pitch; the
+// next core matrix along K lies `leading` bytes on (16 here), the next 8 rows `stride` bytes on (128).
+__device__ __forceinline__ uint64_t make_sliding_desc(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);        // start address, 16-byte units
+    d |= static_cast<uint64_t>(16 >> 4) << 16;                      // leading offset: next 16 bytes of K
+    d |= static_cast<uint64_t>(128 >> 4) << 32;                     // stride offset between 8-row groups
+    d |= static_cast<uint64_t>(1) << 46;                            // descriptor version of this architecture
+    return d;                                                       // layout field 0: no swizzle
 }
 
 }  // namespace qtz_ptx
