@@ -17,7 +17,7 @@ import subprocess
 import numpy as np
 
 _DIR = os.path.dirname(os.path.abspath(__file__))
-_SOURCES = ["qtz_oracle.c", "qtz_oracle_conv.c", "qtz_oracle_ops.c"]
+_SOURCES = ["qtz_oracle.c", "qtz_oracle_conv.c", "qtz_oracle_ops.c", "qtz_oracle_sim.c"]
 _LIB_PATH = os.path.join(_DIR, "liboracle.so")
 _lib = None
 
@@ -284,3 +284,53 @@ def global_avgpool_u8(x, z_x, mult, rshift, z_y, c=None):
     _chk(lib().orc_global_avgpool_u8(_p(x), I32(z_x), I32(b), I32(h * w), I32(c), I32(xp),
                                      I32(mult), I32(rshift), I32(z_y), I32(xp), _p(y)))
     return y
+
+
+def simquant(x, params, axis, qmin, qmax):
+    """SimQuant (Section 2.4): quantize then de-quantize, fp32 in and out."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    params = np.ascontiguousarray(np.atleast_1d(params), dtype=QPARAMS)
+    o, a, i = _view(x.shape, axis)
+    assert params.shape[0] == a
+    y = np.empty(x.shape, np.float32)
+    _chk(lib().orc_simquant(_p(x), I64(o), I64(a), I64(i), _p(params), I32(qmin), I32(qmax), _p(y)))
+    return y
+
+
+def sqnr(w, w_hat, axis=None):
+    """SQNR in dB (Appendix A) per index of `axis`, or of the whole tensor (axis=None)."""
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    w_hat = np.ascontiguousarray(w_hat, dtype=np.float32)
+    assert w.shape == w_hat.shape
+    o, a, i = _view(w.shape, axis)
+    out = np.empty(a, np.float64)
+    _chk(lib().orc_sqnr(_p(w), _p(w_hat), I64(o), I64(a), I64(i), _p(out)))
+    return out
+
+
+def ema_update(state_lo, state_hi, batch_lo, batch_hi, decay, initialised):
+    """Moving average of per-batch ranges (Section 2.5); updates the fp64 state arrays in place and
+    returns the new `initialised` flag."""
+    assert state_lo.dtype == np.float64 and state_hi.dtype == np.float64
+    batch_lo = np.ascontiguousarray(batch_lo, dtype=np.float32)
+    batch_hi = np.ascontiguousarray(batch_hi, dtype=np.float32)
+    flag = I32(int(bool(initialised)))
+    _chk(lib().orc_ema_update(_p(state_lo), _p(state_hi), _p(batch_lo), _p(batch_hi), I64(state_lo.size),
+                              ctypes.c_double(decay), ctypes.byref(flag)))
+    return bool(flag.value)
+
+
+def rescale_u8(x, z_x, mult, rshift, z_y, act_min=0, act_max=255, c=None, out=None, out_offset=0):
+    """uint8 tensor to another quantizer (concat, Section 3.2.1).  x: [..., pitch]; the result goes to
+    `out[..., out_offset:out_offset + c]` when `out` is given (a channel slice of a concatenation)."""
+    x = np.ascontiguousarray(x, dtype=np.uint8)
+    xp = x.shape[-1]
+    c = xp if c is None else c
+    if out is None:
+        out = np.zeros_like(x)
+    assert out.flags["C_CONTIGUOUS"] and out.dtype == np.uint8
+    yp = out.shape[-1]
+    dst = ctypes.c_void_p(out.ctypes.data + out_offset)
+    _chk(lib().orc_rescale_u8(_p(x), I64(x.size // xp), I32(c), I32(xp), I32(z_x), I32(mult), I32(rshift),
+                              I32(z_y), I32(act_min), I32(act_max), dst, I32(yp)))
+    return out

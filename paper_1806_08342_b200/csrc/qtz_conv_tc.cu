@@ -15,6 +15,9 @@
 //               the warps signal each filled box on an mbarrier and never wait for one another
 //   warps 18,19 one store thread per group: TMA store of every filled box (which also clips ragged
 //               tile edges), box handed back once the store has read it
+// Image stems (few channels, wide filters) run as "row-window" layers: a frame of the input padded
+// with z_x is staged one contiguous run per filter row by plain bulk copies, and the MMA reads the
+// overlapping windows of 128 neighbouring output columns straight out of that run (pad_copy_kernel).
 // Zero filling stands for padding, so the -z_x sum(w) term must skip the padded taps as well:
 // the weight sums are tabulated per border class (which filter rows / columns are cut) and each
 // epilogue thread, owning one output pixel, picks its class.
@@ -978,7 +981,7 @@ struct qtz_tc_state {
     TcArgs args{};
     qtz_conv_desc eff{};       // the layer as the kernel sees it (im2col layers become pointwise over the window matrix)
     bool im2col = false;
-    bool rowwin = false;       // row-window layer: padded frame + overlapping tensor map (see pad_copy_kernel)
+    bool rowwin = false;       // row-window layer: padded frame read through a sliding operand descriptor (see pad_copy_kernel)
     int hp = 0, wp = 0;        // its frame extent
     int fp = 16, rb = 128;     // bytes per frame pixel, bytes of one filter-row run
     int cs = 0;                // im2col: bytes per tap in the window matrix (channels rounded up to 4)
