@@ -39,6 +39,27 @@ def step_ops(sizes=None):
     return float(sum(2.0 * s * s * s for s in (SIZES if sizes is None else sizes)))
 
 
+# DRAM traffic of the dominant kernel, from one ncu capture of a timed step of the full sweep
+# (dram__bytes_read.sum + dram__bytes_write.sum over the five conv_tc_kernel launches, divided by five;
+# the summary is profiles/conv_tc_kernel_gemm_8192.md).  It is reported only while the kernel's sources
+# are the ones the counters were taken from.
+KERNEL_TRAFFIC = {"bytes_per_launch": 87.89e6,
+                  "sources": ("paper_1806_08342_b200/csrc/qtz_conv_tc.cu", "paper_1806_08342_b200/csrc/qtz_ptx.cuh"),
+                  "sha256": "f2cd2f4adadece37731e928a2148a3470bbca39773206cae45605aced04cd8b1"}
+
+
+def kernel_traffic():
+    import hashlib
+    h = hashlib.sha256()
+    try:
+        for f in KERNEL_TRAFFIC["sources"]:
+            with open(os.path.join(ROOT, f), "rb") as fh:
+                h.update(fh.read())
+    except OSError:
+        return None
+    return KERNEL_TRAFFIC["bytes_per_launch"] if h.hexdigest() == KERNEL_TRAFFIC["sha256"] and len(SIZES) == 5 else None
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -449,7 +470,8 @@ def run_ours(args, rank, world, local_rank):
                 "d2h_bytes_per_step": int(sum(c.y_host.numel() for c in cases)), "steps": e2e_steps},
         "gpu_launches": 2 * len(cases) * args.steps,
         "roofline": {"bound": "tensor", "kernel": "conv_tc_kernel", "achieved": kernel_tops, "peak": int8_peak,
-                     "unit": UNIT, "frac": kernel_tops / int8_peak, "traffic": None,
+                     "unit": UNIT, "frac": kernel_tops / int8_peak, "traffic": kernel_traffic(),
+                     "traffic_unit": "bytes per launch (algorithmic: 53.7e6)",
                      "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_burst']} TFLOP/s x 2 (int8:bf16 nominal ratio)",
                      "frac_of_sustained_peak": kernel_tops / (2.0 * peaks["bf16_sustained"]),
                      "frac_of_nominal_4500": kernel_tops / 4500.0},

@@ -170,6 +170,46 @@ QTZ_API qtz_status qtz_dequantize(qtz_handle h, const void* q_dev, int32_t in_dt
                           int64_t axis_len, int64_t inner, const qtz_qparams* params_host,
                           float* x_dev, void* stream);
 
+/* ---- simulated quantization, SQNR, range averaging, rescale ------------------------------ */
+
+/* SimQuant (Section 2.4): a quantizer followed by a de-quantizer,
+ *   y = (clamp(round(x / Delta) + z, qmin, qmax) - z) * Delta
+ * with exactly the fp32 steps of qtz_quantize_tensor and qtz_dequantize (the paper prints the
+ * formula with the sign of z flipped; this is Eq. 3 applied to Eq. 1-2).  fp32 in, fp32 out,
+ * same view and parameter conventions; code_dtype (QTZ_U8 / QTZ_S8 / QTZ_S4_PACKED) and
+ * restrict_range only select the code range [qmin, qmax].  y_dev may alias x_dev.           */
+QTZ_API qtz_status qtz_simquant(qtz_handle h, const float* x_dev, int64_t outer, int64_t axis_len,
+                                int64_t inner, const qtz_qparams* params_host, int32_t code_dtype,
+                                int32_t restrict_range, float* y_dev, void* stream);
+
+/* Signal-to-quantization-noise ratio (Appendix A),
+ *   SQNR = 10 log10( sum w^2 / sum (w - w_hat)^2 )   in dB,
+ * one value per index of the middle axis (per output feature map), or of the whole tensor with
+ * axis_len == 1.  Sums are accumulated in fp64; no noise at all gives +infinity.  Writes axis_len
+ * doubles to sqnr_db_host and BLOCKS until `stream` has finished.  axis_len <= 65535.        */
+QTZ_API qtz_status qtz_sqnr(qtz_handle h, const float* w_dev, const float* w_hat_dev, int64_t outer,
+                            int64_t axis_len, int64_t inner, double* sqnr_db_host, void* stream);
+
+/* Host-only: the moving average of per-batch ranges that Section 2.5 prescribes for
+ * activations.  The paper names no weighting; this is the exponential average
+ *   state <- decay * state + (1 - decay) * batch      (0 <= decay < 1, fp64)
+ * applied to n (lo, hi) pairs, e.g. the output of qtz_minmax.  While *initialised is 0 the batch
+ * values are copied instead and the flag is set.  Feed (float)state to qtz_params_from_range.
+ * Errors: QTZ_ERR_NONFINITE if a batch value is NaN/Inf (the state is then untouched).        */
+QTZ_API qtz_status qtz_ema_update(double* state_lo_host, double* state_hi_host, const float* batch_lo_host,
+                                  const float* batch_hi_host, int64_t n, double decay, int32_t* initialised);
+
+/* A uint8 tensor re-expressed in another quantizer -- what the inputs of a concatenation need
+ * so that they share the output's scale and zero point (Section 3.2.1):
+ *   y = clamp(y_zp + floor(((x - x_zp) mult + 2^(rshift-1)) / 2^rshift), act_min, act_max)
+ * with (mult, rshift) = qtz_quantize_multiplier(Delta_x / Delta_y).  x is [pixels][c] with pitch
+ * x_pitch, y likewise with y_pitch; to fill a channel slice of a concatenated tensor pass
+ * y_dev = base + channel offset and the pitch of the whole.  Pointers and pitches need no
+ * particular alignment (rows that are 4-byte aligned on both sides take a faster path).     */
+QTZ_API qtz_status qtz_rescale_u8(qtz_handle h, const uint8_t* x_dev, int32_t x_zp, int32_t mult, int32_t rshift,
+                                  uint8_t* y_dev, int32_t y_zp, int32_t act_min, int32_t act_max, int64_t pixels,
+                                  int32_t c, int32_t x_pitch, int32_t y_pitch, void* stream);
+
 /* ---- batch-norm folding (Eq. 20-21) ------------------------------------------------------ */
 
 /* W_inf[n][:] = gamma[n] W[n][:] / sigma[n],  Bias_inf[n] = beta[n] + gamma[n] (b[n] - mu[n]) /

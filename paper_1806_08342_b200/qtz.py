@@ -69,6 +69,11 @@ SIGNATURES = {
     "qtz_depthwise_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p]),
     "qtz_add_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p,
                              c_int32, c_int32, c_int32, c_int64, c_int32, c_int32, c_void_p]),
+    "qtz_simquant": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int32, c_int32, c_void_p, c_void_p]),
+    "qtz_sqnr": (c_int32, [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p]),
+    "qtz_ema_update": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_double, POINTER(c_int32)]),
+    "qtz_rescale_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_int32, c_int32, c_int32, c_int64,
+                                 c_int32, c_int32, c_int32, c_void_p]),
     "qtz_maxpool_u8": (c_int32, [c_void_p, c_void_p, c_void_p] + [c_int32] * 8 + [c_void_p]),
     "qtz_global_avgpool_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p] + [c_int32] * 7 + [c_void_p]),
 }
@@ -138,6 +143,21 @@ def add_params(a_scale, b_scale, y_scale):
     if rc:
         raise QtzError(rc, "qtz_add_params")
     return ma.value, mb.value, r.value
+
+
+def ema_update(state_lo, state_hi, batch_lo, batch_hi, decay, initialised):
+    """Moving average of per-batch ranges (Section 2.5): updates the fp64 state arrays in place and
+    returns the new `initialised` flag."""
+    assert state_lo.dtype == np.float64 and state_hi.dtype == np.float64 and state_lo.shape == state_hi.shape
+    batch_lo = np.ascontiguousarray(batch_lo, dtype=np.float32)
+    batch_hi = np.ascontiguousarray(batch_hi, dtype=np.float32)
+    assert batch_lo.size == state_lo.size and batch_hi.size == state_lo.size
+    flag = c_int32(int(bool(initialised)))
+    rc = load_library().qtz_ema_update(_np(state_lo), _np(state_hi), _np(batch_lo), _np(batch_hi), state_lo.size,
+                                       float(decay), ctypes.byref(flag))
+    if rc != 0:
+        raise QtzError(rc, "qtz_ema_update")
+    return bool(flag.value)
 
 
 def params_from_range(lo, hi, bits=8, symmetric=False):
@@ -241,6 +261,42 @@ class Handle:
             out = torch.empty(shape, dtype=torch.float32, device=q.device)
         self._chk(self.lib.qtz_dequantize(self.h, _ptr(q), in_dtype, o, a, i, _np(params), _ptr(out), _stream()),
                   "qtz_dequantize")
+        return out
+
+    def simquant(self, x, params, axis=None, code_dtype=U8, restrict_range=False, out=None):
+        """SimQuant (Section 2.4): quantize then de-quantize, fp32 in and out."""
+        _check_dev(x, out)
+        assert x.dtype == torch.float32
+        params = np.ascontiguousarray(np.atleast_1d(params), dtype=QPARAMS)
+        o, a, i = _view(x.shape, axis)
+        assert params.shape[0] == a
+        if out is None:
+            out = torch.empty_like(x)
+        self._chk(self.lib.qtz_simquant(self.h, _ptr(x), o, a, i, _np(params), code_dtype, int(restrict_range),
+                                        _ptr(out), _stream()), "qtz_simquant")
+        return out
+
+    def sqnr(self, w, w_hat, axis=None):
+        """SQNR in dB (Appendix A) per index of `axis`, or of the whole tensor."""
+        _check_dev(w, w_hat)
+        assert w.dtype == torch.float32 and w_hat.dtype == torch.float32 and w.shape == w_hat.shape
+        o, a, i = _view(w.shape, axis)
+        out = np.zeros(a, np.float64)
+        self._chk(self.lib.qtz_sqnr(self.h, _ptr(w), _ptr(w_hat), o, a, i, _np(out), _stream()), "qtz_sqnr")
+        return out
+
+    def rescale_u8(self, x, x_zp, mult, rshift, y_zp, act_min=0, act_max=255, c=None, out=None, out_offset=0):
+        """uint8 tensor to another quantizer (concat, Section 3.2.1); with `out`, fills the channel
+        slice [out_offset, out_offset + c) of that wider tensor."""
+        _check_dev(x, out)
+        xp = x.shape[-1]
+        c = xp if c is None else c
+        if out is None:
+            out = torch.zeros_like(x)
+        yp = out.shape[-1]
+        dst = c_void_p(out.data_ptr() + out_offset)
+        self._chk(self.lib.qtz_rescale_u8(self.h, _ptr(x), x_zp, mult, rshift, dst, y_zp, act_min, act_max,
+                                          x.numel() // xp, c, xp, yp, _stream()), "qtz_rescale_u8")
         return out
 
     def fold_batchnorm(self, w, conv_bias, gamma, beta, mean, var, eps):

@@ -84,3 +84,29 @@ def test_params_from_range_matches_oracle(qtz):
             assert a.tobytes() == b.tobytes(), (lo, hi, bits, a, b)
             a, b = qtz.params_from_range(lo, hi, bits, True), oracle.symmetric_params(lo, hi, bits)
             assert a.tobytes() == b.tobytes()
+
+
+def test_ema_update_matches_oracle_bit_for_bit(qtz):
+    g = np.random.default_rng(11)
+    n = 7
+    lo_a, hi_a, lo_b, hi_b = np.zeros(n), np.zeros(n), np.zeros(n), np.zeros(n)
+    init_a = init_b = False
+    for step in range(40):
+        blo = (g.normal(-1.0, 0.3, n)).astype(np.float32)
+        bhi = (g.normal(4.0, 0.5, n)).astype(np.float32)
+        decay = [0.9, 0.99, 0.0, 0.5][step % 4]
+        init_a = qtz.ema_update(lo_a, hi_a, blo, bhi, decay, init_a)
+        init_b = oracle.ema_update(lo_b, hi_b, blo, bhi, decay, init_b)
+        assert init_a and init_b
+        assert np.array_equal(lo_a.view(np.uint64), lo_b.view(np.uint64))
+        assert np.array_equal(hi_a.view(np.uint64), hi_b.view(np.uint64))
+    with pytest.raises(qtz.QtzError) as e:
+        qtz.ema_update(lo_a, hi_a, np.full(n, np.nan, np.float32), np.ones(n, np.float32), 0.9, True)
+    assert e.value.code == -5
+    with pytest.raises(qtz.QtzError):
+        qtz.ema_update(lo_a, hi_a, np.zeros(n, np.float32), np.ones(n, np.float32), 1.0, True)
+    # parameters from the averaged range, same rules on both sides
+    for i in range(n):
+        a = qtz.params_from_range(np.float32(lo_a[i]), np.float32(hi_a[i]))
+        b = oracle.affine_params(np.float32(lo_b[i]), np.float32(hi_b[i]))
+        assert a["zero_point"] == b["zero_point"] and a["scale"] == b["scale"]
