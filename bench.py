@@ -60,6 +60,9 @@ def kernel_traffic():
     return KERNEL_TRAFFIC["bytes_per_launch"] if h.hexdigest() == KERNEL_TRAFFIC["sha256"] and len(SIZES) == 5 else None
 
 
+DW_CLOCK_GHZ = 1.94   # SM clock ncu reports while the depthwise kernel runs (no tensor work, no power cap)
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -237,17 +240,27 @@ def time_hbm_kernels(hq, qtz, torch, peaks):
     entry("minmax_f32 (4 B/elem)", timed(lambda: hq.minmax(x)), 4.0 * n)
     entry("quantize_f32_to_u8 (5 B/elem)", timed(lambda: hq.quantize_tensor(x, p, out=q)), 5.0 * n)
     entry("dequantize_u8_to_f32 (5 B/elem)", timed(lambda: hq.dequantize(q, p, out=x)), 5.0 * n)
-    del x, q
-    # MobileNet-v1 depthwise layers at batch 128: (H, C, stride)
-    for hh, c, stride in [(112, 64, 2), (56, 128, 1), (14, 512, 1)]:
+    y = torch.empty_like(x)
+    entry("simquant_f32 (8 B/elem)", timed(lambda: hq.simquant(x, p, out=y)), 8.0 * n)
+    del x, q, y
+    # MobileNet-v1 depthwise layers at batch 128: (H, C, stride, zero points and clamp).  "ranged": z_x = 3,
+    # z_y = 10, clamp [10,255] (border cells refilled with z_x, explicit clamp); "relu6": the case between two
+    # ReLU6 tensors, z_x = z_y = 0 and the whole byte as the range.  The kernel is bound by integer issue, not by
+    # HBM: per output 3 dp4a (2 issue cycles each per warp) and one 32x32->64 multiply (4 cycles), i.e. 10 cycles
+    # per warp of 32 outputs on each of the 4 schedulers of an SM -- the ALU peak the fraction refers to.
+    alu_peak = 148 * 4 * 32 / 10.0 * DW_CLOCK_GHZ * 1e9                  # outputs per second
+    for hh, c, stride, name, z in [(112, 64, 2, "ranged", (3, 10, 10, 255)), (56, 128, 1, "ranged", (3, 10, 10, 255)),
+                                   (56, 128, 1, "relu6", (0, 0, 0, 255)), (14, 512, 1, "ranged", (3, 10, 10, 255))]:
         xin = torch.randint(0, 256, (128, hh, hh, c), dtype=torch.uint8, device="cuda")
         w = torch.randint(-127, 128, (3, 3, c), dtype=torch.int8, device="cuda")
         m, r = qtz.quantize_multiplier(1.0 / 600.0)
         plan = hq.conv_create(qtz.conv_desc(128, hh, hh, c, c, 3, 3, stride, 1), w, None, None,
                               np.full(c, m, np.int32), np.full(c, r, np.int32), depthwise=True)
         y = plan.empty_output("cuda")
-        secs = timed(lambda: plan(xin, 3, 10, 10, 255, out=y), reps=10)
-        entry(f"depthwise3x3 128x{hh}x{hh}x{c} s{stride}", secs, float(xin.numel() + y.numel()))
+        secs = timed(lambda: plan(xin, *z, out=y), reps=10)
+        key = f"depthwise3x3 128x{hh}x{hh}x{c} s{stride} {name}"
+        entry(key, secs, float(xin.numel() + y.numel()))
+        res[key]["frac_of_alu_peak"] = round(y.numel() / secs / alu_peak, 3)
         plan.close()
     a = torch.randint(0, 256, (1 << 28,), dtype=torch.uint8, device="cuda").view(-1, 64)
     b = torch.randint(0, 256, (1 << 28,), dtype=torch.uint8, device="cuda").view(-1, 64)
