@@ -376,6 +376,21 @@ def time_networks(hq, qtz, torch, reps=10, detail=False):
     return res
 
 
+def max_over_ranks(values, dist, device):
+    """The slowest rank's value of each entry (device-timed durations): replicas run side by side and the
+    job is done when the last one is."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_value(ops_per_rank_step, steps, world, ms):
+    """Aggregate throughput of `world` replicas (weak scaling: every rank does the full step)."""
+    return world * ops_per_rank_step * steps / (ms * 1e-3) / 1e12
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     from paper_1806_08342_b200 import build as qbuild
@@ -454,16 +469,13 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, e2e_ms = float(t[0]), float(t[1])
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], dist, "cuda")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
     ops = step_ops()
-    value = world * ops * args.steps / (ms * 1e-3) / 1e12
+    value = whole_job_value(ops, args.steps, world, ms)
     int8_peak = 2.0 * peaks["bf16_burst"]          # dense int8 : bf16 is 2 : 1 on this part (4.5 vs 2.25 POP/s nominal)
     kernel_tops = ops / (sum(per_size_ms) * 1e-3) / 1e12
     sweep = {str(c.size): {"kernel_ms": round(per_size_ms[i], 4),

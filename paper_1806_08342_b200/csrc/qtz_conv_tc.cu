@@ -841,12 +841,11 @@ pad_copy_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ xp, int bat
 {
     const int ppc = 16 / fp;                         // pixels per 16-byte chunk
     const int chunks = wp / ppc;                     // wp is a multiple of ppc
-    const int64_t i = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
-    if (i >= static_cast<int64_t>(batch) * hp * chunks) return;
-    const int xc = static_cast<int>(i % chunks);
-    const int64_t r = i / chunks;
-    const int yp = static_cast<int>(r % hp);
-    const int64_t b = r / hp;
+    const int xc = blockIdx.x * blockDim.x + threadIdx.x;      // grid: (chunks of a row, frame rows, images)
+    if (xc >= chunks) return;
+    const int yp = blockIdx.y;
+    const int64_t b = blockIdx.z;
+    const int64_t i = (b * hp + yp) * chunks + xc;
     const int iy = yp - pad;
     const uint32_t zx4 = 0x01010101u * static_cast<uint32_t>(zx);
     uint32_t words[4] = {zx4, zx4, zx4, zx4};
@@ -1305,8 +1304,11 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
 
     const uint8_t* xin = x;
     if (t->rowwin) {
-        const int64_t work = static_cast<int64_t>(d.batch) * t->hp * (t->wp * t->fp / 16);
-        pad_copy_kernel<<<static_cast<unsigned>((work + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
+        const int chunks = t->wp * t->fp / 16;
+        if (t->hp > 65535 || d.batch > 65535) return QTZ_ERR_UNSUPPORTED;
+        const int threads = std::min(kPrepThreads, (chunks + 31) / 32 * 32);
+        pad_copy_kernel<<<dim3(static_cast<unsigned>((chunks + threads - 1) / threads), static_cast<unsigned>(t->hp),
+                               static_cast<unsigned>(d.batch)), threads, 0, st>>>(
             x, p->x_gather, d.batch, d.h, d.w, d.c, t->hp, t->wp, d.pad, x_zp, t->fp);
         QTZ_LAUNCH_CHECK(h, "pad_copy_kernel");
         xin = p->x_gather;
