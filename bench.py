@@ -453,18 +453,51 @@ def run_ours(args, rank, world, local_rank):
     per_size_ms = [float(np.mean([kev[st][i][0].elapsed_time(kev[st][i][1]) for st in range(args.steps)]))
                    for i in range(len(cases))]
 
-    # end to end: host buffers in, host buffers out, copies inside the timed region
+    # end to end: host buffers in, host buffers out, every copy inside the timed region.  A user with pinned
+    # buffers overlaps the three legs: uploads, kernels and downloads run on a stream each (all library
+    # calls stay on ONE stream, as the handle requires) and events order them per tensor -- an input is
+    # not overwritten before the kernel that read it is done, an output not before its download is.
     e2e_steps = max(1, min(args.steps, 5))
-    for c in cases:
-        c.a.copy_(c.a_host, non_blocking=True); c.run(); c.y_host.copy_(c.y, non_blocking=True)
+    cur = torch.cuda.current_stream()
+    up, run, down = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+
+    def e2e_pass(steps):
+        a_free = [None] * len(cases)
+        y_free = [None] * len(cases)
+        for _ in range(steps):
+            for i, c in enumerate(cases):
+                with torch.cuda.stream(up):
+                    if a_free[i] is not None:
+                        up.wait_event(a_free[i])
+                    c.a.copy_(c.a_host, non_blocking=True)
+                    a_ready = torch.cuda.Event(); a_ready.record(up)
+                with torch.cuda.stream(run):
+                    run.wait_event(a_ready)
+                    if y_free[i] is not None:
+                        run.wait_event(y_free[i])
+                    c.run()
+                    done = torch.cuda.Event(); done.record(run)
+                    a_free[i] = done
+                with torch.cuda.stream(down):
+                    down.wait_event(done)
+                    c.y_host.copy_(c.y, non_blocking=True)
+                    y_free[i] = torch.cuda.Event(); y_free[i].record(down)
+
+    def fork():
+        ev = torch.cuda.Event(); ev.record(cur)
+        for st in (up, run, down):
+            st.wait_event(ev)
+
+    def join():
+        for st in (up, run, down):
+            ev = torch.cuda.Event(); ev.record(st)
+            cur.wait_event(ev)
+
+    fork(); e2e_pass(1); join()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(e2e_steps):
-        for c in cases:
-            c.a.copy_(c.a_host, non_blocking=True)
-            c.run()
-            c.y_host.copy_(c.y, non_blocking=True)
+    fork(); e2e_pass(e2e_steps); join()
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
@@ -492,7 +525,8 @@ def run_ours(args, rank, world, local_rank):
         "clocks": clocks,
         "e2e": {"value": world * ops * e2e_steps / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                 "h2d_bytes_per_step": int(sum(c.a_host.numel() for c in cases)),
-                "d2h_bytes_per_step": int(sum(c.y_host.numel() for c in cases)), "steps": e2e_steps},
+                "d2h_bytes_per_step": int(sum(c.y_host.numel() for c in cases)), "steps": e2e_steps,
+                "how": "pinned host buffers; upload, kernel and download streams overlapped, ordered per tensor by events"},
         "gpu_launches": 2 * len(cases) * args.steps,
         "roofline": {"bound": "tensor", "kernel": "conv_tc_kernel", "achieved": kernel_tops, "peak": int8_peak,
                      "unit": UNIT, "frac": kernel_tops / int8_peak, "traffic": kernel_traffic(),
