@@ -49,6 +49,8 @@ constexpr int kMaxStages = 8;
 constexpr int kNumBarriers = 2 * kMaxStages + 2 * kMaxAcc + 2 * kEpiGroups * kMaxObuf + 1;
 constexpr int kResidentBMax = 80 * 1024;   // weights of a whole layer stay in shared memory up to this size
 constexpr int kMaxCls = 16;
+constexpr int kRunBytes = 2048;      // row-window layers: bytes of a frame row one copy brings in (256 elements of 8 bytes)
+constexpr int kRunCols = 120;        // ... and the output columns of a tile: 16 * 119 + rb <= 2048 for rb <= 128
 constexpr int kSmemBudget = 227 * 1024 - 1024;  // leave room for the 1 KB alignment slack
 
 // Division of a 31-bit unsigned number by a constant known on the host, as one high multiply and one
@@ -335,10 +337,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int nrow = n_tile * a.BN;
             int tap_x = 0, tap_y = 0, kcol = 0, kc = 0;   // filter tap of the next K block, its first weight column, channel offset
             // row-window layers: the tile is a run of output columns of one output row; filter row tap_y
-            // reads frame row h0 * cstride + tap_y from the byte where the window of column w0 starts
-            const uint8_t* const frame_at =
-                a.cstride > 0 ? a.frame + (static_cast<int64_t>(b0) * a.frame_rows + h0 * a.cstride) * a.frame_row + 16 * w0
-                              : nullptr;
+            // reads frame row h0 * cstride + tap_y from the byte where the window of column w0 starts (16 w0)
+            const int frame_x = 2 * w0, frame_y = b0 * a.frame_rows + h0 * a.cstride;   // 8-byte element, frame row
             for (int st = 0; st < nst; ++st) {
                 if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget, 64u)) ||
                     *abort_flag != 0) {
@@ -353,7 +353,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         const uint32_t dst_a = base + L.a_off + stage * L.a_stage + j * L.a_blk;
                         if (a.is4d)
                             if (a.cstride > 0)
-                                bulk_load(dst_a, frame_at + tap_y * a.frame_row, static_cast<uint32_t>(a.seg_bytes), full);
+                            {   // one copy per ring stage: the runs of its spb consecutive filter rows, 2 KB apart
+                                if (j == 0) tma_load_2d(dst_a, &map_a, full, frame_x, frame_y + tap_y);
+                            }
                             else
                                 tma_load_4d(dst_a, &map_a, full, kc, w0 + tap_x - a.pad, h0 + tap_y - a.pad, b0);
                         else
@@ -983,6 +985,7 @@ struct qtz_tc_state {
     bool rowwin = false;       // row-window layer: padded frame read through a sliding operand descriptor (see pad_copy_kernel)
     int hp = 0, wp = 0;        // its frame extent
     int fp = 16, rb = 128;     // bytes per frame pixel, bytes of one filter-row run
+    size_t frame_bytes = 0;    // the frame with its slack
     int cs = 0;                // im2col: bytes per tap in the window matrix (channels rounded up to 4)
     CUtensorMap map_b{};
     int8_t* w_packed = nullptr;
@@ -1029,6 +1032,20 @@ bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims
                 const uint32_t* box, int swizzle_bytes)
 {
     return qtz_encode_u8_map(m, base, rank, dims, strides_bytes, box, swizzle_bytes);
+}
+
+// The padded frame as a matrix of 8-byte elements, one row per frame row; a box is 2048 bytes of each of
+// `rows` consecutive frame rows.
+bool encode_frame_map(CUtensorMap* m, const void* base, int64_t row_bytes, int64_t frame_rows, int rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t gd[2] = {static_cast<cuuint64_t>(row_bytes / 8), static_cast<cuuint64_t>(frame_rows)};
+    cuuint64_t gs[1] = {static_cast<cuuint64_t>(row_bytes)};
+    cuuint32_t bx[2] = {static_cast<cuuint32_t>(kRunBytes / 8), static_cast<cuuint32_t>(rows)};
+    cuuint32_t es[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(base), gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 bool is_pointwise(const qtz_conv_desc& d) { return d.kh == 1 && d.kw == 1 && d.pad == 0; }
@@ -1183,8 +1200,8 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
         if (rw) {
             // a tile is a run of 128 output columns of one output row (columns beyond the image are
             // computed from whatever follows in the frame and clipped by the store)
-            a.tw = kTileM; a.th = 1; a.tb = 1;
-            best_tiles = static_cast<int64_t>((a.W + kTileM - 1) / kTileM) * a.H * a.B;
+            a.tw = kRunCols; a.th = 1; a.tb = 1;
+            best_tiles = static_cast<int64_t>((a.W + kRunCols - 1) / kRunCols) * a.H * a.B;
         } else {
             for (int tw = 1; tw <= std::min(a.W, kTileM); ++tw)
                 for (int th = 1; th <= std::min(a.H, kTileM / tw); ++th) {
@@ -1255,11 +1272,16 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
         // the last tiles of a row read past its end (into the next row, or into this slack after the last one)
         a.frame_row = static_cast<int64_t>(t->wp) * t->fp;
         a.frame_rows = t->hp;
-        a.seg_bytes = 16 * (kTileM - 1) + t->rb;
-        a.a_blk = (a.seg_bytes + 127) / 128 * 128;
+        // a copy brings 2048 bytes of each filter row (the row's end and whatever lies past the image arrive as
+        // zeros); the MMA reads 16 * 127 + rb bytes per row, i.e. up to 112 bytes into the next row's slot, which only
+        // accumulator rows beyond the 120 columns of a tile ever see
+        a.seg_bytes = kRunBytes;
+        a.a_blk = kRunBytes;
         const size_t slack = static_cast<size_t>(a.tiles_w) * kTileM * 16 + 256;
-        QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->x_gather), static_cast<size_t>(d.batch) * t->hp * a.frame_row + slack));
-        QTZ_CUDA(h, cudaMemsetAsync(p->x_gather, 0, static_cast<size_t>(d.batch) * t->hp * a.frame_row + slack, st));
+        t->frame_bytes = static_cast<size_t>(d.batch) * t->hp * a.frame_row + slack;
+        if (t->frame_bytes / 8 > 0x7fffffffull) return QTZ_ERR_UNSUPPORTED;      // element indices are 32-bit
+        QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->x_gather), t->frame_bytes));
+        QTZ_CUDA(h, cudaMemsetAsync(p->x_gather, 0, t->frame_bytes, st));
     }
 
     // the weight map never changes
@@ -1340,7 +1362,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     CUtensorMap map_a, map_y;
     const uint64_t pitch = static_cast<uint64_t>(d.c_pitch_in);
     if (t->rowwin) {
-        map_a = t->map_b;   // unused: the producer copies runs of the frame with plain bulk copies
+        map_a = t->map_b;   // encoded below, once the number of filter rows per ring stage is known
         a.frame = xin;
     } else if (pw) {
         const uint64_t dims[2] = {static_cast<uint64_t>(d.c), static_cast<uint64_t>(t->in_pixels)};
@@ -1432,6 +1454,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.fold = 0;
     if (!a.raw && a.ncls == 1 && a.zw == 0 && p->rshift_max <= 53)
         a.fold = p->rshift_min >= 32 ? 1 : (p->narrow_ok ? 2 : 0);
+    if (t->rowwin && !encode_frame_map(&map_a, xin, a.frame_row, static_cast<int64_t>(d.batch) * t->hp, a.spb)) return QTZ_ERR_CUDA;
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
     conv_tc_kernel<<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, a);
     QTZ_LAUNCH_CHECK(h, "conv_tc_kernel");
