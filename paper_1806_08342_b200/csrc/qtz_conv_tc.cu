@@ -16,8 +16,8 @@
 //   warps 18,19 one store thread per group: TMA store of every filled box (which also clips ragged
 //               tile edges), box handed back once the store has read it
 // Image stems (few channels, wide filters) run as "row-window" layers: a frame of the input padded
-// with z_x is staged one contiguous run per filter row by plain bulk copies, and the MMA reads the
-// overlapping windows of 128 neighbouring output columns straight out of that run (pad_copy_kernel).
+// with z_x is staged one contiguous run per filter row (one tensor copy per tile brings them all), and the MMA
+// reads the overlapping windows of 120 neighbouring output columns straight out of those runs (pad_copy_kernel).
 // Zero filling stands for padding, so the -z_x sum(w) term must skip the padded taps as well:
 // the weight sums are tabulated per border class (which filter rows / columns are cut) and each
 // epilogue thread, owning one output pixel, picks its class.
@@ -86,9 +86,8 @@ struct TcArgs {
     uint32_t num_tiles;
     int32_t W, H, B;                        // output extent (2-D case: W = number of pixels)
     int32_t taps, kw, pad, cstride;          // cstride > 0: row-window layer with that convolution stride (else 0)
-    const uint8_t* frame;                    // row-window layers: the padded frame, its row pitch and rows per image,
-    int64_t frame_row;                       // and the bytes one tile takes from a frame row
-    int32_t frame_rows, seg_bytes;
+    int64_t frame_row;                       // row-window layers: row pitch of the padded frame, its rows per image,
+    int32_t frame_rows, seg_bytes;           // and the bytes of a frame row one tile takes
     int32_t a_blk;                           // bytes of one activation K block in the ring (0: 128 rows of BK bytes)
     int32_t kb_per_tap, c_pad;
     int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
@@ -832,9 +831,9 @@ stride_gather_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, i
 // smallest that holds the channels and makes the step between output columns, stride * fp, a
 // multiple of 16 bytes -- here exactly 16); rb / fp consecutive pixels of a frame row (rb = 32, 64
 // or 128 bytes) are then one filter row of an output pixel's window plus zero-weight positions, and
-// the window of the next output column starts 16 bytes later.  A tile (128 output columns of one
-// output row) therefore needs, per filter row, one contiguous run of 16 * 127 + rb frame bytes in
-// shared memory, and the tensor cores read their K-major operand rows straight out of that run
+// the window of the next output column starts 16 bytes later.  A tile (120 output columns of one
+// output row) therefore needs, per filter row, one contiguous run of 16 * 119 + rb <= 2048 frame bytes
+// in shared memory, and the tensor cores read their K-major operand rows straight out of that run
 // through an unswizzled descriptor with a 16-byte row pitch (make_sliding_desc): no window matrix is
 // ever materialised.  No border classes: padding is data.  One thread writes 16 bytes of the frame.
 __global__ void __launch_bounds__(kPrepThreads)
@@ -1363,7 +1362,6 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     const uint64_t pitch = static_cast<uint64_t>(d.c_pitch_in);
     if (t->rowwin) {
         map_a = t->map_b;   // encoded below, once the number of filter rows per ring stage is known
-        a.frame = xin;
     } else if (pw) {
         const uint64_t dims[2] = {static_cast<uint64_t>(d.c), static_cast<uint64_t>(t->in_pixels)};
         const uint64_t strides[1] = {pitch};

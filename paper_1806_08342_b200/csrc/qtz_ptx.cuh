@@ -82,15 +82,6 @@ __device__ __forceinline__ void prefetch_tensormap(const void* tmap)
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
 
-// Plain (untiled) bulk copy of `bytes` contiguous bytes from global to shared memory; both addresses
-// 16-byte aligned, the size a multiple of 16.  Completes on the mbarrier like a tensor copy.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, uint32_t bar, int x, int y)
 {
     asm volatile(
