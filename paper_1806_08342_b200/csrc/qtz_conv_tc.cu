@@ -1173,7 +1173,9 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     // (one tile: 32-column granularity, the TMA store clips what lies beyond the real channels;
     //  several tiles: whole staging boxes, since a box must not spill into the next tile's columns)
     a.BN = a.n_tiles == 1 ? (d.n + 31) / 32 * 32 : ((d.n + a.n_tiles - 1) / a.n_tiles + 63) / 64 * 64;
-    a.out_box = (a.BN % 128 == 0) ? 128 : 64;
+    // (a single column tile wider than 128 also takes 128-byte boxes: the store clips the last one at N, and every
+    //  box row is one request to the copy engine whatever its length)
+    a.out_box = (a.BN % 128 == 0 || (a.n_tiles == 1 && a.BN > 128)) ? 128 : 64;
     // every accumulator a tile ahead lets the MMA warp start a tile before an epilogue group is back
     a.n_acc = std::min(kMaxAcc, kTmemCols / a.BN);
     a.acc_stride = a.BN;
