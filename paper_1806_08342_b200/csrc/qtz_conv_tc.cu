@@ -1170,6 +1170,11 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.kb_per_tap = a.c_pad / a.BK;
     // N tiling: as few tiles as possible, each a multiple of 32 columns
     a.n_tiles = (d.n + 255) / 256;
+    {   // a layer with few pixel tiles (a classifier: one or two) spreads over the SMs by its columns instead
+        const int64_t m_tiles = (t->in_pixels + kTileM - 1) / kTileM;
+        if (pw && d.n > 64 && m_tiles * a.n_tiles * 2 <= h->num_sms)
+            a.n_tiles = static_cast<int32_t>(std::max<int64_t>(a.n_tiles, std::min<int64_t>((d.n + 63) / 64, h->num_sms / m_tiles)));
+    }
     // (one tile: 32-column granularity, the TMA store clips what lies beyond the real channels;
     //  several tiles: whole staging boxes, since a box must not spill into the next tile's columns)
     a.BN = a.n_tiles == 1 ? (d.n + 31) / 32 * 32 : ((d.n + a.n_tiles - 1) / a.n_tiles + 63) / 64 * 64;
