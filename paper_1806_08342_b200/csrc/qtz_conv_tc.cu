@@ -86,6 +86,11 @@ struct TcArgs {
     uint32_t num_tiles;
     int32_t W, H, B;                        // output extent (2-D case: W = number of pixels)
     int32_t taps, kw, pad, cstride;          // cstride > 0: row-window layer with that convolution stride (else 0)
+    // Thread copies (lsu != 0, row-window layers): the lanes of the producer warp bring the frame runs of a tile in
+    // with 16-byte asynchronous copies instead of the copy engine, which is the full stage of these layers.
+    // src = the frame; full_count: arrivals a ring stage's "full" barrier expects.
+    const uint8_t* src;
+    int32_t lsu, full_count;
     int64_t frame_row;                       // row-window layers: row pitch of the padded frame, its rows per image,
     int32_t frame_rows, seg_bytes;           // and the bytes of a frame row one tile takes
     int32_t a_blk;                           // bytes of one activation K block in the ring (0: 128 rows of BK bytes)
@@ -275,7 +280,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < a.stages; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_full + 8 * s, a.full_count);
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int i = 0; i < kMaxAcc; ++i) {
@@ -328,7 +333,71 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             __syncwarp();
         }
-        for (uint32_t tile = blockIdx.x; !failed && tile < a.num_tiles; tile += gridDim.x) {
+        // ---- thread copies: every lane copies 16-byte pieces of the stage's activations; a stage is signalled
+        // `lag` stages late, once this warp's copies for it have landed and been fenced for the tensor cores
+        uint32_t issued = 0, signalled = 0, sig_stage = 0;
+        // stages a signal trails its copies by (what may be in flight); two stages short of the ring so that the MMA
+        // warp always has signalled stages ahead of it while the producer waits for a free one
+        const uint32_t lag = max(1u, min(S - 3u, 6u));
+        for (uint32_t tile = blockIdx.x; a.lsu != 0 && !failed && tile < a.num_tiles; tile += gridDim.x) {
+            int n_tile, w0, h0, b0;
+            uint32_t m_tile;
+            decode_tile(a, tile, m_tile, n_tile);
+            tile_origin(a, m_tile, w0, h0, b0);
+            const int nrow = n_tile * a.BN;
+            for (int st = 0; st < nst; ++st) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget, 64u)) ||
+                    *abort_flag != 0) {
+                    failed = true;
+                    break;
+                }
+                const uint32_t full = bar_full + 8 * stage;
+                if (!wres && elect_one()) {              // the weights still come through the copy engine
+                    mbar_arrive_expect_tx(full, static_cast<uint32_t>(a.spb * a.BN * a.BK));
+                    for (int j = 0; j < a.spb; ++j)
+                        tma_load_2d(base + L.b_off + stage * L.b_stage + j * L.b_blk, &map_b, full, (st * a.spb + j) * a.c_pad, nrow);
+                }
+                const uint32_t dst_a = base + L.a_off + stage * L.a_stage;
+                {                                        // spb filter rows: 2 KB of each frame row, as it lies
+                    const uint8_t* run = a.src + (static_cast<int64_t>(b0) * a.frame_rows + h0 * a.cstride + st * a.spb) * a.frame_row +
+                                         16 * w0 + 16 * lane;
+                    for (int j = 0; j < a.spb; ++j, run += a.frame_row)
+#pragma unroll
+                        for (int i = 0; i < kRunBytes / 512; ++i) cp_async_16(dst_a + j * kRunBytes + 16 * lane + 512 * i, run + 512 * i);
+                }
+                cp_async_commit();
+                if (++issued > lag) {
+                    switch (lag) {                       // all but the `lag` most recent stages of this lane have landed
+                    case 1: cp_async_wait<1>(); break;
+                    case 2: cp_async_wait<2>(); break;
+                    case 3: cp_async_wait<3>(); break;
+                    case 4: cp_async_wait<4>(); break;
+                    case 5: cp_async_wait<5>(); break;
+                    default: cp_async_wait<6>(); break;
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (elect_one()) mbar_arrive(bar_full + 8 * sig_stage);
+                    ++signalled;
+                    if (++sig_stage == S) sig_stage = 0;
+                }
+                if (++stage == S) {
+                    stage = 0;
+                    phase ^= 1;
+                }
+            }
+        }
+        if (a.lsu != 0) {                                // the last stages, and nothing in flight when the CTA leaves
+            cp_async_wait<0>();
+            fence_proxy_async_smem();
+            __syncwarp();
+            for (; signalled < issued; ++signalled) {
+                if (elect_one()) mbar_arrive(bar_full + 8 * sig_stage);
+                if (++sig_stage == S) sig_stage = 0;
+            }
+            __syncwarp();
+        }
+        for (uint32_t tile = blockIdx.x; a.lsu == 0 && !failed && tile < a.num_tiles; tile += gridDim.x) {
             int n_tile, w0, h0, b0;
             uint32_t m_tile;
             decode_tile(a, tile, m_tile, n_tile);
@@ -1460,6 +1529,11 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     if (!a.raw && a.ncls == 1 && a.zw == 0 && p->rshift_max <= 53)
         a.fold = p->rshift_min >= 32 ? 1 : (p->narrow_ok ? 2 : 0);
     if (t->rowwin && !encode_frame_map(&map_a, xin, a.frame_row, static_cast<int64_t>(d.batch) * t->hp, a.spb)) return QTZ_ERR_CUDA;
+    // thread copies for the frame runs of row-window layers (see TcArgs::lsu).  (For pointwise tiles with short
+    // rows one warp's 16-byte copies were slower than the copy engine: about 140 cycles per warp-wide copy.)
+    a.lsu = (a.stages >= 3 && t->rowwin) ? 1 : 0;
+    a.src = xin;
+    a.full_count = a.lsu ? (a.bres > 0 ? 1 : 2) : 1;
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
     conv_tc_kernel<<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, a);
     QTZ_LAUNCH_CHECK(h, "conv_tc_kernel");

@@ -76,6 +76,16 @@ __device__ __forceinline__ bool elect_one()
     return pred != 0;
 }
 
+// ---- asynchronous copies issued by threads (16 bytes each, L2 only) -------------------------------
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// Waits until all but the kPending most recent groups of this thread have landed.
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
+
 // ---- TMA --------------------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tensormap(const void* tmap)
 {
