@@ -45,7 +45,7 @@ def step_ops(sizes=None):
 # are the ones the counters were taken from.
 KERNEL_TRAFFIC = {"bytes_per_launch": 87.73e6,
                   "sources": ("paper_1806_08342_b200/csrc/qtz_conv_tc.cu", "paper_1806_08342_b200/csrc/qtz_ptx.cuh"),
-                  "sha256": "6a36d8ee8ea2161d82879563885b61261723e2b5c4663016a2b168473d521c4b"}
+                  "sha256": "8e28bfdd59344d5c68e17a42a0f51471666277c0cee2bdabaa4e2978b1faf211"}
 
 
 def kernel_traffic():

@@ -16,7 +16,7 @@
 //   warps 18,19 one store thread per group: TMA store of every filled box (which also clips ragged
 //               tile edges), box handed back once the store has read it
 // Image stems (few channels, wide filters) run as "row-window" layers: a frame of the input padded
-// with z_x is staged one contiguous run per filter row (one tensor copy per tile brings them all), and the MMA
+// with z_x is staged one contiguous run per filter row (copied by the producer warp's lanes), and the MMA
 // reads the overlapping windows of 120 neighbouring output columns straight out of those runs (pad_copy_kernel).
 // Zero filling stands for padding, so the -z_x sum(w) term must skip the padded taps as well:
 // the weight sums are tabulated per border class (which filter rows / columns are cut) and each
