@@ -71,6 +71,8 @@ STEM_SHAPES = [
     # b, h, w, c, n, k, stride, pad
     (2, 17, 15, 3, 32, 3, 2, 1),      # MobileNet stem shape (3 input channels, stride 2)
     (1, 23, 21, 3, 64, 7, 2, 3),      # ResNet stem shape
+    (1, 20, 250, 3, 256, 7, 2, 3),    # stems whose weights do not stay resident (they share ring stages with the frame
+    (1, 12, 14, 4, 272, 5, 2, 2),     # runs), several tiles per output row (125 columns), two column tiles
     (1, 9, 9, 5, 7, 3, 1, 1),         # odd channel counts, n not a multiple of 4
     (3, 6, 7, 20, 70, 1, 1, 0),       # pointwise, ragged n tile
     (1, 8, 8, 16, 16, 3, 1, 0),       # no padding
