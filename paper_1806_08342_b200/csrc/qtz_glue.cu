@@ -47,6 +47,46 @@ __device__ __forceinline__ uint32_t add4(uint32_t a, uint32_t b, const AddRule& 
     return pack_sat_u8(y1, y0, pack_sat_u8(y3, y2, 0u)) + lo4;
 }
 
+// The same for shifts 16 <= r <= 38 without 64-bit multiplies.  With m = mh 2^16 + ml (both halves below 2^16):
+//   a m_a + b m_b + addend = (a mah + b mbh + Ah) 2^16 + (a mal + b mbl + Al),  addend = Ah 2^16 + Al, 0 <= Al < 2^16,
+// every bracket fits 32 bits (a, b < 2^8; |addend| < 2^47), and since floor(floor(x / 2^16) / 2^(r-16)) =
+// floor(x / 2^r) the result is ((hi + Ah + (lo >> 16)) >> (r - 16)) exactly.  Each bracket is one dp2a on the
+// byte pair (a, b) against the 16-bit pair (m_a half, m_b half).
+struct AddSplit {
+    uint32_t mh, ml;     // (mah | mbh << 16), (mal | mbl << 16)
+    int32_t ah;          // addend >> 16 (arithmetic)
+    uint32_t al;         // addend & 0xffff
+    int32_t sh, span;    // r - 16, act_max - act_min
+};
+
+__device__ __forceinline__ uint32_t dp2a_lo(uint32_t m16x2, uint32_t bytes, uint32_t c)
+{
+    uint32_t d;
+    asm("dp2a.lo.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(m16x2), "r"(bytes), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t dp2a_hi(uint32_t m16x2, uint32_t bytes, uint32_t c)
+{
+    uint32_t d;
+    asm("dp2a.hi.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(m16x2), "r"(bytes), "r"(c));
+    return d;
+}
+
+__device__ __forceinline__ int32_t add_split1(uint32_t hi, uint32_t lo, const AddSplit& q)
+{
+    return __vimin_s32_relu((static_cast<int32_t>(hi) + q.ah + static_cast<int32_t>(lo >> 16)) >> q.sh, q.span);
+}
+
+__device__ __forceinline__ uint32_t add_split4(uint32_t a, uint32_t b, const AddSplit& q, uint32_t lo4)
+{
+    const uint32_t p01 = __byte_perm(a, b, 0x5140), p23 = __byte_perm(a, b, 0x7362);   // (a0,b0,a1,b1), (a2,b2,a3,b3)
+    const int32_t y0 = add_split1(dp2a_lo(q.mh, p01, 0u), dp2a_lo(q.ml, p01, q.al), q);
+    const int32_t y1 = add_split1(dp2a_hi(q.mh, p01, 0u), dp2a_hi(q.ml, p01, q.al), q);
+    const int32_t y2 = add_split1(dp2a_lo(q.mh, p23, 0u), dp2a_lo(q.ml, p23, q.al), q);
+    const int32_t y3 = add_split1(dp2a_hi(q.mh, p23, 0u), dp2a_hi(q.ml, p23, q.al), q);
+    return pack_sat_u8(y1, y0, pack_sat_u8(y3, y2, 0u)) + lo4;
+}
+
 // y = clamp(z_y + (((a - z_a) m_a + (b - z_b) m_b + 2^(r-1)) >> r)).  All constants fold into one
 // 64-bit addend: 2^(r-1) + (z_y - act_min) 2^r - z_a m_a - z_b m_b (|.| < 2^62 for r <= 53).
 template <int kShiftKind>
@@ -65,8 +105,22 @@ add_u8_kernel(const uint8_t* __restrict__ a, const uint8_t* __restrict__ b, int6
     const uint4 va = __ldcs(reinterpret_cast<const uint4*>(a) + g);
     const uint4 vb = __ldcs(reinterpret_cast<const uint4*>(b) + g);
     uint4 o;
-    o.x = add4<kShiftKind>(va.x, vb.x, r, addend, span, lo4); o.y = add4<kShiftKind>(va.y, vb.y, r, addend, span, lo4);
-    o.z = add4<kShiftKind>(va.z, vb.z, r, addend, span, lo4); o.w = add4<kShiftKind>(va.w, vb.w, r, addend, span, lo4);
+    if (kShiftKind == 3) {
+        AddSplit q;
+        q.mh = (static_cast<uint32_t>(r.a_mult) >> 16) | (static_cast<uint32_t>(r.b_mult) & 0xffff0000u);
+        q.ml = (static_cast<uint32_t>(r.a_mult) & 0xffffu) | (static_cast<uint32_t>(r.b_mult) << 16);
+        q.ah = static_cast<int32_t>(addend >> 16);
+        q.al = static_cast<uint32_t>(addend) & 0xffffu;
+        q.sh = r.rshift - 16;
+        q.span = span;
+        o.x = add_split4(va.x, vb.x, q, lo4); o.y = add_split4(va.y, vb.y, q, lo4);
+        o.z = add_split4(va.z, vb.z, q, lo4); o.w = add_split4(va.w, vb.w, q, lo4);
+        reinterpret_cast<uint4*>(y)[g] = o;
+        return;
+    }
+    o.x = add4<kShiftKind == 3 ? 0 : kShiftKind>(va.x, vb.x, r, addend, span, lo4); o.y = add4<kShiftKind == 3 ? 0 : kShiftKind>(va.y, vb.y, r, addend, span, lo4);
+    o.z = add4<kShiftKind == 3 ? 0 : kShiftKind>(va.z, vb.z, r, addend, span, lo4);
+    o.w = add4<kShiftKind == 3 ? 0 : kShiftKind>(va.w, vb.w, r, addend, span, lo4);
     reinterpret_cast<uint4*>(y)[g] = o;
 }
 
@@ -141,7 +195,9 @@ extern "C" qtz_status qtz_add_u8(qtz_handle h, const uint8_t* a_dev, int32_t a_z
     const AddRule r{a_zp, a_mult, b_zp, b_mult, rshift, y_zp, act_min, act_max};
     const unsigned blocks = static_cast<unsigned>(ceil_div(bytes >> 4, kThreads));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (rshift >= 32)
+    if (rshift >= 16 && rshift <= 38)
+        add_u8_kernel<3><<<blocks, kThreads, 0, st>>>(a_dev, b_dev, bytes, r, y_dev);
+    else if (rshift >= 32)
         add_u8_kernel<0><<<blocks, kThreads, 0, st>>>(a_dev, b_dev, bytes, r, y_dev);
     else if (rshift >= 10)
         add_u8_kernel<1><<<blocks, kThreads, 0, st>>>(a_dev, b_dev, bytes, r, y_dev);
