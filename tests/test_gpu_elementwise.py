@@ -173,6 +173,11 @@ def test_maxpool_and_global_avgpool(hq):
     want = oracle.maxpool_u8(x, 3, 2, 1, c=24)
     got = host(hq.maxpool_u8(dev(x), 24, 3, 2, 1))
     assert got.shape == want.shape and np.array_equal(got[..., :24], want[..., :24])
+    for shape, k, st, pad in [((2, 112, 112, 64), 3, 2, 1), ((1, 9, 12, 16), 3, 2, 0), ((2, 8, 7, 48), 3, 2, 2), ((1, 10, 10, 16), 2, 2, 0),
+                              ((1, 11, 9, 32), 3, 1, 1)]:
+        xx = pitched(synth.uniform_u8(shape, 12, shape[1]))
+        got = host(hq.maxpool_u8(dev(xx), shape[3], k, st, pad))
+        assert np.array_equal(got, oracle.maxpool_u8(xx, k, st, pad, c=shape[3]))
     x7 = pitched(synth.uniform_u8((5, 7, 7, 40), 12, 2))
     m, r = oracle.quantize_multiplier(0.02 / (49 * 0.015))
     want = oracle.global_avgpool_u8(x7, 4, m, r, 9, c=40)
