@@ -241,6 +241,33 @@ QTZ_API qtz_status qtz_activation_range(int32_t kind, float y_scale, int32_t y_z
 QTZ_API qtz_status qtz_add_params(float a_scale, float b_scale, float y_scale, int32_t* a_mult,
                           int32_t* b_mult, int32_t* rshift);
 
+/* ---- range rules between the layers of a network (host only; Sections 2.5, 3.1.2, 3.2.1) ---- */
+
+/* Range of a layer's output tensor from the min/max of its pre-activation values on calibration
+ * data (Section 2.5: activations take the min/max seen on a batch) and the activation fused into
+ * the layer (Section 3.2.1).  The quantized tensor is the one after the activation, and ReLU /
+ * ReLU6 are monotone, so each end of the range goes through the activation: kind 0 [lo,hi];
+ * 1 [max(lo,0), max(hi,0)]; 2 both ends also capped at 6.  Feed the result to
+ * qtz_params_from_range.  QTZ_ERR_NONFINITE for NaN/Inf, QTZ_ERR_INVALID_ARG for hi < lo.       */
+QTZ_API qtz_status qtz_range_after_activation(float lo, float hi, int32_t kind, float* lo_out, float* hi_out);
+/* Range of an element-wise sum of two quantized tensors (Section 3.2.1): the interval sum of the
+ * inputs' representable ranges (min_nudged + min_nudged, max_nudged + max_nudged, one fp32 add
+ * each) -- a bound that needs no pass over data and cannot saturate -- followed by the fused
+ * activation as in qtz_range_after_activation.                                                   */
+QTZ_API qtz_status qtz_add_output_range(const qtz_qparams* a_host, const qtz_qparams* b_host, int32_t kind,
+                                        float* lo_out, float* hi_out);
+/* Scale of Eq. 4's accumulator per output channel: acc_params[i].scale = x_scale * w_params[i].scale
+ * (one fp32 product), zero point 0 -- the parameters qtz_dequantize needs for QTZ_S32 input.     */
+QTZ_API qtz_status qtz_accumulator_scales(float x_scale, const qtz_qparams* w_params_host, int64_t n,
+                                          qtz_qparams* acc_params_host);
+/* Fixed-point form of Delta_x Delta_w[i] / Delta_y (the rescale Eq. 4 implies) for n output
+ * channels: the quotient is formed in fp64 and handed to qtz_quantize_multiplier.                 */
+QTZ_API qtz_status qtz_requant_multipliers(float x_scale, const qtz_qparams* w_params_host, int64_t n, float y_scale,
+                                           int32_t* mult_host, int32_t* rshift_host);
+/* Fixed-point form of Delta_x / (hw Delta_y) for qtz_global_avgpool_u8 (exactly 1 / hw when the
+ * two scales are equal).                                                                          */
+QTZ_API qtz_status qtz_avgpool_multiplier(int32_t hw, float x_scale, float y_scale, int32_t* mult, int32_t* rshift);
+
 /* ---- convolution (Eq. 4-6) -------------------------------------------------------------- */
 
 /* One-time preparation of a layer ("the weights are constant at inference", Section 2.1):

@@ -17,7 +17,7 @@ import subprocess
 import numpy as np
 
 _DIR = os.path.dirname(os.path.abspath(__file__))
-_SOURCES = ["qtz_oracle.c", "qtz_oracle_conv.c", "qtz_oracle_ops.c", "qtz_oracle_sim.c"]
+_SOURCES = ["qtz_oracle.c", "qtz_oracle_conv.c", "qtz_oracle_ops.c", "qtz_oracle_sim.c", "qtz_oracle_net.c"]
 _LIB_PATH = os.path.join(_DIR, "liboracle.so")
 _lib = None
 
@@ -334,3 +334,19 @@ def rescale_u8(x, z_x, mult, rshift, z_y, act_min=0, act_max=255, c=None, out=No
     _chk(lib().orc_rescale_u8(_p(x), I64(x.size // xp), I32(c), I32(xp), I32(z_x), I32(mult), I32(rshift),
                               I32(z_y), I32(act_min), I32(act_max), dst, I32(yp)))
     return out
+
+
+def range_after_activation(lo, hi, kind):
+    """Observed pre-activation range pushed through the fused activation (0 none, 1 ReLU, 2 ReLU6)."""
+    a, b = F32(), F32()
+    _chk(lib().orc_range_after_activation(F32(lo), F32(hi), I32(kind), ctypes.byref(a), ctypes.byref(b)))
+    return a.value, b.value
+
+
+def add_output_range(a_params, b_params, kind):
+    """Range of a + b from the inputs' nudged ranges, then the fused activation."""
+    pa = np.ascontiguousarray(np.atleast_1d(a_params), dtype=QPARAMS)
+    pb = np.ascontiguousarray(np.atleast_1d(b_params), dtype=QPARAMS)
+    lo, hi = F32(), F32()
+    _chk(lib().orc_add_output_range(_p(pa), _p(pb), I32(kind), ctypes.byref(lo), ctypes.byref(hi)))
+    return lo.value, hi.value

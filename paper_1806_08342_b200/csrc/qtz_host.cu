@@ -233,3 +233,65 @@ extern "C" qtz_status qtz_add_params(float a_scale, float b_scale, float y_scale
     *rshift = sh;
     return QTZ_OK;
 }
+
+// ---- range rules for the tensors between the layers of a network (Sections 2.5, 3.1.2, 3.2.1) ----
+
+extern "C" qtz_status qtz_range_after_activation(float lo, float hi, int32_t kind, float* lo_out, float* hi_out)
+{
+    if (!lo_out || !hi_out || kind < 0 || kind > 2) return QTZ_ERR_INVALID_ARG;
+    if (!std::isfinite(lo) || !std::isfinite(hi)) return QTZ_ERR_NONFINITE;
+    if (hi < lo) return QTZ_ERR_INVALID_ARG;
+    if (kind != 0) {                       // ReLU and ReLU6 are monotone: the range goes through them end by end
+        lo = std::fmax(lo, 0.0f);
+        hi = std::fmax(hi, 0.0f);
+    }
+    if (kind == 2) {
+        lo = std::fmin(lo, 6.0f);
+        hi = std::fmin(hi, 6.0f);
+    }
+    *lo_out = lo;
+    *hi_out = hi;
+    return QTZ_OK;
+}
+
+extern "C" qtz_status qtz_add_output_range(const qtz_qparams* a, const qtz_qparams* b, int32_t kind, float* lo_out,
+                                           float* hi_out)
+{
+    if (!a || !b) return QTZ_ERR_INVALID_ARG;
+    // interval sum of what the two inputs can represent, in fp32
+    return qtz_range_after_activation(a->min_nudged + b->min_nudged, a->max_nudged + b->max_nudged, kind, lo_out, hi_out);
+}
+
+extern "C" qtz_status qtz_accumulator_scales(float x_scale, const qtz_qparams* w_params_host, int64_t n,
+                                             qtz_qparams* acc_params_host)
+{
+    if (!w_params_host || !acc_params_host || n <= 0 || !(x_scale > 0.f)) return QTZ_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < n; ++i) {
+        acc_params_host[i].scale = x_scale * w_params_host[i].scale;     // one fp32 product
+        acc_params_host[i].zero_point = 0;
+        acc_params_host[i].min_nudged = 0.f;
+        acc_params_host[i].max_nudged = 0.f;
+    }
+    return QTZ_OK;
+}
+
+extern "C" qtz_status qtz_requant_multipliers(float x_scale, const qtz_qparams* w_params_host, int64_t n, float y_scale,
+                                              int32_t* mult_host, int32_t* rshift_host)
+{
+    if (!w_params_host || !mult_host || !rshift_host || n <= 0 || !(x_scale > 0.f) || !(y_scale > 0.f))
+        return QTZ_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < n; ++i) {
+        const double m = static_cast<double>(x_scale) * static_cast<double>(w_params_host[i].scale) / static_cast<double>(y_scale);
+        const qtz_status s = qtz_quantize_multiplier(m, mult_host + i, rshift_host + i);
+        if (s != QTZ_OK) return s;
+    }
+    return QTZ_OK;
+}
+
+extern "C" qtz_status qtz_avgpool_multiplier(int32_t hw, float x_scale, float y_scale, int32_t* mult, int32_t* rshift)
+{
+    if (hw <= 0 || !(x_scale > 0.f) || !(y_scale > 0.f)) return QTZ_ERR_INVALID_ARG;
+    // identical quantizers in and out leave exactly 1 / hw
+    const double m = x_scale == y_scale ? 1.0 / hw : static_cast<double>(x_scale) / (static_cast<double>(hw) * static_cast<double>(y_scale));
+    return qtz_quantize_multiplier(m, mult, rshift);
+}

@@ -68,11 +68,9 @@ class QuantizedNetwork:
         self.batch = batch
         x0 = np.zeros(images_u8.shape[:3] + (16,), np.uint8)
         x0[..., :3] = images_u8
-        rec = np.zeros(1, qtz.QPARAMS)
-        rec["scale"], rec["zero_point"], rec["min_nudged"], rec["max_nudged"] = np.float32(1.0 / 255.0), 0, 0.0, 1.0
         tensors = {"in": torch.from_numpy(x0).cuda()}
         chans = {"in": 3}
-        self.params = {"in": rec[0]}
+        self.params = {"in": qtz.params_from_range(0.0, 1.0)}   # image codes 0..255 stand for reals in [0,1]
         self.layers = []
         for index, op in enumerate(self.ops):
             kind = op["op"]
@@ -96,31 +94,20 @@ class QuantizedNetwork:
                     self.layers.append(L)
                     continue
                 acc = raw_plan(x[:calib], zx)
-                ap = np.zeros(cout, qtz.QPARAMS)
-                ap["scale"] = xs * wp["scale"]                                   # fp32 product, formed once
-                lo, hi = h.minmax(h.dequantize(acc, ap, axis=3))
+                lo, hi = h.minmax(h.dequantize(acc, qtz.accumulator_scales(xs, wp), axis=3))
                 raw_plan.close()
-                lo, hi = float(lo[0]), float(hi[0])
-                if op["act"] == 1:
-                    lo, hi = max(lo, 0.0), max(hi, 0.0)
-                elif op["act"] == 2:
-                    lo, hi = min(max(lo, 0.0), 6.0), min(max(hi, 0.0), 6.0)
-                yp = qtz.params_from_range(lo, hi)
-                mr = [qtz.quantize_multiplier(float(xs) * float(s) / float(yp["scale"])) for s in wp["scale"]]
+                yp = qtz.params_from_range(*qtz.range_after_activation(lo[0], hi[0], op["act"]))
+                mult, rshift = qtz.requant_multipliers(xs, wp, yp["scale"])
                 amin, amax = qtz.activation_range(op["act"], yp["scale"], int(yp["zero_point"]))
                 desc = qtz.conv_desc(batch, hh, ww, cin, cout, k, k, st, pad, wkind, qtz.OUT_U8, c_pitch_in=pitch)
-                L.plan = h.conv_create(desc, w_q, bias_q, None, [m for m, _ in mr], [r for _, r in mr], depthwise=dw)
+                L.plan = h.conv_create(desc, w_q, bias_q, None, mult, rshift, depthwise=dw)
                 L.args = (zx, int(yp["zero_point"]), amin, amax)
                 tensors[op["dst"]] = L.plan(x, *L.args)
                 chans[op["dst"]] = cout
                 self.params[op["dst"]] = yp
             elif kind == "add":
                 a, b = self.params[op["a"]], self.params[op["b"]]
-                lo = float(np.float32(a["min_nudged"]) + np.float32(b["min_nudged"]))
-                hi = float(np.float32(a["max_nudged"]) + np.float32(b["max_nudged"]))
-                if op["act"] == 1:
-                    lo, hi = max(lo, 0.0), max(hi, 0.0)
-                yp = qtz.params_from_range(lo, hi)
+                yp = qtz.params_from_range(*qtz.add_output_range(a, b, op["act"]))
                 ma, mb, r = qtz.add_params(a["scale"], b["scale"], yp["scale"])
                 amin, amax = qtz.activation_range(op["act"], yp["scale"], int(yp["zero_point"]))
                 L.args = (int(a["zero_point"]), ma, int(b["zero_point"]), mb, r, int(yp["zero_point"]), amin, amax,
@@ -137,7 +124,7 @@ class QuantizedNetwork:
                 self.params[op["dst"]] = self.params[op["src"]]
             elif kind == "avgpool":
                 x, xp = tensors[op["src"]], self.params[op["src"]]
-                m, r = qtz.quantize_multiplier(1.0 / (x.shape[1] * x.shape[2]))
+                m, r = qtz.avgpool_multiplier(x.shape[1] * x.shape[2], xp["scale"], xp["scale"])
                 z = int(xp["zero_point"])
                 L.args = (z, z, m, r, chans[op["src"]])
                 tensors[op["dst"]] = h.global_avgpool_u8(x, *L.args)

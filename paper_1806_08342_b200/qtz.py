@@ -60,6 +60,11 @@ SIGNATURES = {
     "qtz_quantize_multiplier": (c_int32, [c_double, POINTER(c_int32), POINTER(c_int32)]),
     "qtz_activation_range": (c_int32, [c_int32, c_float, c_int32, POINTER(c_int32), POINTER(c_int32)]),
     "qtz_add_params": (c_int32, [c_float, c_float, c_float, POINTER(c_int32), POINTER(c_int32), POINTER(c_int32)]),
+    "qtz_range_after_activation": (c_int32, [c_float, c_float, c_int32, POINTER(c_float), POINTER(c_float)]),
+    "qtz_add_output_range": (c_int32, [c_void_p, c_void_p, c_int32, POINTER(c_float), POINTER(c_float)]),
+    "qtz_accumulator_scales": (c_int32, [c_float, c_void_p, c_int64, c_void_p]),
+    "qtz_requant_multipliers": (c_int32, [c_float, c_void_p, c_int64, c_float, c_void_p, c_void_p]),
+    "qtz_avgpool_multiplier": (c_int32, [c_int32, c_float, c_float, POINTER(c_int32), POINTER(c_int32)]),
     "qtz_conv_create": (c_int32, [c_void_p, POINTER(ConvDesc), c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
                                   c_void_p, POINTER(c_void_p), c_void_p]),
     "qtz_conv_destroy": (c_int32, [c_void_p]),
@@ -143,6 +148,50 @@ def add_params(a_scale, b_scale, y_scale):
     if rc:
         raise QtzError(rc, "qtz_add_params")
     return ma.value, mb.value, r.value
+
+
+def range_after_activation(lo, hi, kind):
+    a, b = c_float(), c_float()
+    rc = load_library().qtz_range_after_activation(float(lo), float(hi), int(kind), byref(a), byref(b))
+    if rc:
+        raise QtzError(rc, "qtz_range_after_activation")
+    return a.value, b.value
+
+
+def add_output_range(a_params, b_params, kind):
+    pa = np.ascontiguousarray(np.atleast_1d(a_params), dtype=QPARAMS)
+    pb = np.ascontiguousarray(np.atleast_1d(b_params), dtype=QPARAMS)
+    lo, hi = c_float(), c_float()
+    rc = load_library().qtz_add_output_range(_np(pa), _np(pb), int(kind), byref(lo), byref(hi))
+    if rc:
+        raise QtzError(rc, "qtz_add_output_range")
+    return lo.value, hi.value
+
+
+def accumulator_scales(x_scale, w_params):
+    wp = np.ascontiguousarray(np.atleast_1d(w_params), dtype=QPARAMS)
+    out = np.zeros(wp.shape[0], QPARAMS)
+    rc = load_library().qtz_accumulator_scales(float(x_scale), _np(wp), wp.shape[0], _np(out))
+    if rc:
+        raise QtzError(rc, "qtz_accumulator_scales")
+    return out
+
+
+def requant_multipliers(x_scale, w_params, y_scale):
+    wp = np.ascontiguousarray(np.atleast_1d(w_params), dtype=QPARAMS)
+    mult, rshift = np.zeros(wp.shape[0], np.int32), np.zeros(wp.shape[0], np.int32)
+    rc = load_library().qtz_requant_multipliers(float(x_scale), _np(wp), wp.shape[0], float(y_scale), _np(mult), _np(rshift))
+    if rc:
+        raise QtzError(rc, "qtz_requant_multipliers")
+    return mult, rshift
+
+
+def avgpool_multiplier(hw, x_scale, y_scale):
+    m, r = c_int32(), c_int32()
+    rc = load_library().qtz_avgpool_multiplier(int(hw), float(x_scale), float(y_scale), byref(m), byref(r))
+    if rc:
+        raise QtzError(rc, "qtz_avgpool_multiplier")
+    return m.value, r.value
 
 
 def ema_update(state_lo, state_hi, batch_lo, batch_hi, decay, initialised):

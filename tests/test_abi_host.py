@@ -110,3 +110,37 @@ def test_ema_update_matches_oracle_bit_for_bit(qtz):
         a = qtz.params_from_range(np.float32(lo_a[i]), np.float32(hi_a[i]))
         b = oracle.affine_params(np.float32(lo_b[i]), np.float32(hi_b[i]))
         assert a["zero_point"] == b["zero_point"] and a["scale"] == b["scale"]
+
+
+def test_range_rules_between_layers_match_oracle(qtz):
+    g = np.random.default_rng(21)
+    for _ in range(2000):
+        lo = float(np.float32(g.normal() * 10 ** g.uniform(-3, 2)))
+        hi = float(np.float32(lo + abs(g.normal()) * 10 ** g.uniform(-3, 2)))
+        for kind in (0, 1, 2):
+            assert qtz.range_after_activation(lo, hi, kind) == oracle.range_after_activation(lo, hi, kind)
+        pa, pb = oracle.affine_params(lo, hi, 8), oracle.affine_params(-abs(hi), abs(lo) + 1.0, 8)
+        for kind in (0, 1, 2):
+            assert qtz.add_output_range(pa, pb, kind) == oracle.add_output_range(pa, pb, kind)
+    with pytest.raises(qtz.QtzError) as e:
+        qtz.range_after_activation(1.0, 0.0, 0)
+    assert e.value.code == -1
+    with pytest.raises(qtz.QtzError) as e:
+        qtz.range_after_activation(float("inf"), 0.0, 0)
+    assert e.value.code == -5
+
+
+def test_accumulator_scales_and_multipliers_match_oracle(qtz):
+    g = np.random.default_rng(22)
+    wp = np.zeros(300, qtz.QPARAMS)
+    wp["scale"] = (10 ** g.uniform(-5, -1, 300)).astype(np.float32)
+    for xs, ys in [(np.float32(1 / 255), np.float32(0.0235)), (np.float32(0.047), np.float32(0.013))]:
+        acc = qtz.accumulator_scales(xs, wp)
+        assert np.array_equal(acc["scale"], xs * wp["scale"]) and not acc["zero_point"].any()
+        mult, rshift = qtz.requant_multipliers(xs, wp, ys)
+        want = [oracle.quantize_multiplier(float(xs) * float(s) / float(ys)) for s in wp["scale"]]
+        assert [(int(m), int(r)) for m, r in zip(mult, rshift)] == want
+    for hw in (1, 49, 196, 3136):
+        assert qtz.avgpool_multiplier(hw, 0.02, 0.02) == oracle.quantize_multiplier(1.0 / hw)
+    assert qtz.avgpool_multiplier(49, np.float32(0.02), np.float32(0.05)) == \
+        oracle.quantize_multiplier(float(np.float32(0.02)) / (49.0 * float(np.float32(0.05))))
