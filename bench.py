@@ -39,28 +39,38 @@ def step_ops(sizes=None):
     return float(sum(2.0 * s * s * s for s in (SIZES if sizes is None else sizes)))
 
 
-# DRAM traffic of the dominant kernel, from one ncu capture of a timed step of the full sweep
-# (dram__bytes_read.sum + dram__bytes_write.sum over the five conv_tc_kernel launches, divided by five;
-# the summary is profiles/conv_tc_kernel_gemm_8192.md).  It is reported only while the kernel's sources
-# are the ones the counters were taken from.
-KERNEL_TRAFFIC = {"bytes_per_launch": 87.73e6,
-                  "sources": ("paper_1806_08342_b200/csrc/qtz_conv_tc.cu", "paper_1806_08342_b200/csrc/qtz_ptx.cuh"),
-                  "sha256": "8e28bfdd59344d5c68e17a42a0f51471666277c0cee2bdabaa4e2978b1faf211"}
+# DRAM traffic of the dominant kernel: read from the text summary of one ncu capture of the five
+# conv_tc_kernel launches of a step (dram__bytes_read.sum + dram__bytes_write.sum, divided by five), which
+# also records the SHA-256 of the kernel's sources at the time.  Reported only while those sources are
+# unchanged; null otherwise.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "conv_tc_kernel_gemm_sweep_traffic.txt")
+TRAFFIC_SOURCES = ("paper_1806_08342_b200/csrc/qtz_conv_tc.cu", "paper_1806_08342_b200/csrc/qtz_ptx.cuh")
+
+
+def kernel_sources_sha256():
+    import hashlib
+    h = hashlib.sha256()
+    for f in TRAFFIC_SOURCES:
+        with open(os.path.join(ROOT, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
 
 
 def kernel_traffic():
-    import hashlib
-    h = hashlib.sha256()
     try:
-        for f in KERNEL_TRAFFIC["sources"]:
-            with open(os.path.join(ROOT, f), "rb") as fh:
-                h.update(fh.read())
-    except OSError:
+        rec = dict(line.split(":", 1) for line in open(TRAFFIC_FILE) if ":" in line and not line.startswith("#"))
+        if rec["kernel_sources_sha256"].strip() != kernel_sources_sha256() or len(SIZES) != 5:
+            return None
+        return float(rec["dram_bytes_per_launch"])
+    except (OSError, KeyError, ValueError):
         return None
-    return KERNEL_TRAFFIC["bytes_per_launch"] if h.hexdigest() == KERNEL_TRAFFIC["sha256"] and len(SIZES) == 5 else None
 
 
-DW_CLOCK_GHZ = 1.94   # SM clock ncu reports while the depthwise kernel runs (no tensor work, no power cap)
+# Integer-issue ceiling of the depthwise kernel, in outputs per clock and SM: per output three dp4a (64 lanes
+# per clock and SM) and one 32x32->64 multiply-add (16 lanes per clock and SM) on the same pipe:
+# 1 / (3/64 + 1/16).  A loop of exactly these instructions measured 9.6.
+DW_ALU_OUT_PER_CLK_SM = 1.0 / (3.0 / 64.0 + 1.0 / 16.0)
+
 
 
 def load_peaks():
@@ -150,9 +160,17 @@ def cpu_baseline(target_seconds=15.0):
     frac = min(1.0, budget_ops / step_ops())
     rows = {s: max(1, int(round(s * frac))) for s in SIZES}
     ops, secs = oracle_sample(rows)
-    return {"value": ops / secs / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+    cores = oracle.num_threads()
+    # the same program on one thread, on a sample a sixth as long
+    oracle.set_num_threads(1)
+    rows1 = {s: max(1, int(round(s * frac / (6.0 * cores)))) for s in SIZES}
+    ops1, secs1 = oracle_sample(rows1)
+    oracle.set_num_threads(cores)
+    return {"value": ops / secs / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": "first rows of A per size " + json.dumps({str(k): v for k, v in rows.items()}) +
-                      f" against full B ({ops / 1e9:.1f} GOP in {secs:.1f} s)"}
+                      f" against full B ({ops / 1e9:.1f} GOP in {secs:.1f} s)",
+            "one_thread": {"value": ops1 / secs1 / 1e12, "unit": UNIT,
+                           "sample": f"{ops1 / 1e9:.1f} GOP in {secs1:.1f} s, rows " + json.dumps({str(k): v for k, v in rows1.items()})}}
 
 
 def run_reference(args, rank):
@@ -218,6 +236,7 @@ class GemmCase:
 def time_hbm_kernels(hq, qtz, torch, peaks):
     """Achieved GB/s of the element-wise and depthwise kernels (algorithmic bytes / event time)."""
     res = {}
+    hq_sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
     n = 1 << 28                                                    # 1 GiB of fp32: far larger than L2
     x = torch.empty(n, dtype=torch.float32, device="cuda").uniform_(-1.0, 6.0)
     p = hq.calibrate_minmax(x)
@@ -245,10 +264,8 @@ def time_hbm_kernels(hq, qtz, torch, peaks):
     del x, q, y
     # MobileNet-v1 depthwise layers at batch 128: (H, C, stride, zero points and clamp).  "ranged": z_x = 3,
     # z_y = 10, clamp [10,255] (border cells refilled with z_x, explicit clamp); "relu6": the case between two
-    # ReLU6 tensors, z_x = z_y = 0 and the whole byte as the range.  The kernel is bound by integer issue, not by
-    # HBM: per output 3 dp4a (2 issue cycles each per warp) and one 32x32->64 multiply (4 cycles), i.e. 10 cycles
-    # per warp of 32 outputs on each of the 4 schedulers of an SM -- the ALU peak the fraction refers to.
-    alu_peak = 148 * 4 * 32 / 10.0 * DW_CLOCK_GHZ * 1e9                  # outputs per second
+    # ReLU6 tensors, z_x = z_y = 0 and the whole byte as the range.  At stride 1 the kernel is bound by integer
+    # issue, not by HBM: frac_of_alu_peak refers to DW_ALU_OUT_PER_CLK_SM at the SM clock sampled under load.
     for hh, c, stride, name, z in [(112, 64, 2, "ranged", (3, 10, 10, 255)), (56, 128, 1, "ranged", (3, 10, 10, 255)),
                                    (56, 128, 1, "relu6", (0, 0, 0, 255)), (14, 512, 1, "ranged", (3, 10, 10, 255))]:
         xin = torch.randint(0, 256, (128, hh, hh, c), dtype=torch.uint8, device="cuda")
@@ -258,9 +275,21 @@ def time_hbm_kernels(hq, qtz, torch, peaks):
                               np.full(c, m, np.int32), np.full(c, r, np.int32), depthwise=True)
         y = plan.empty_output("cuda")
         secs = timed(lambda: plan(xin, *z, out=y), reps=10)
+        # the SM clock while this kernel runs, sampled over a longer loop of the same launch
+        sampler = ClockSampler(torch.cuda.current_device())
+        sampler.start()
+        t_end = time.time() + 0.7
+        while time.time() < t_end:
+            for _ in range(50):
+                plan(xin, *z, out=y)
+            torch.cuda.synchronize()
+        clk = sampler.stop()
+        mhz = clk["sm_mhz"] or clk["sm_max_mhz"] or 1965.0
+        alu_peak = hq_sms * DW_ALU_OUT_PER_CLK_SM * mhz * 1e6            # outputs per second
         key = f"depthwise3x3 128x{hh}x{hh}x{c} s{stride} {name}"
         entry(key, secs, float(xin.numel() + y.numel()))
         res[key]["frac_of_alu_peak"] = round(y.numel() / secs / alu_peak, 3)
+        res[key]["sm_mhz"] = mhz
         plan.close()
     a = torch.randint(0, 256, (1 << 28,), dtype=torch.uint8, device="cuda").view(-1, 64)
     b = torch.randint(0, 256, (1 << 28,), dtype=torch.uint8, device="cuda").view(-1, 64)
@@ -304,7 +333,43 @@ def time_layer(hq, qtz, torch, spec, reps=20):
 NETWORK_CONFIGS = [("mobilenet_v1", 128, 8), ("resnet50", 256, 8), ("mobilenet_v2_14", 256, 4)]
 
 
-def time_networks(hq, qtz, torch, reps=10, detail=False):
+def roofline_sum_ms(ops, batch, wbits, peaks, resolution=224):
+    """Lower bound of one forward pass with one kernel per layer and no fusion between layers: per layer the
+    larger of its tensor time (dense layers; 2 ops per multiply-accumulate against the int8 peak, taken as the
+    measured bf16 burst x 2) and its HBM time (input + output + weights once, against the measured copy rate)."""
+    shape = {"in": (resolution, resolution, 3)}
+    hbm, tensor = peaks["hbm_gbs"] * 1e9, 2.0 * peaks["bf16_burst"] * 1e12
+    total = 0.0
+    for op in ops:
+        kind = op["op"]
+        if kind in ("conv", "fc"):
+            h, w, c = shape[op["src"]] if kind == "conv" else (1, 1, op["cin"])
+            k, st, pad = (op["k"], op["stride"], op["pad"]) if kind == "conv" else (1, 1, 0)
+            oh, ow = (h + 2 * pad - k) // st + 1, (w + 2 * pad - k) // st + 1
+            dw = kind == "conv" and op["depthwise"]
+            n = op["cout"]
+            macs = batch * oh * ow * n * k * k * (1 if dw else op["cin"])
+            wbytes = k * k * op["cin"] * (1 if dw else n) * wbits / 8.0
+            nbytes = batch * h * w * c + batch * oh * ow * n * (4 if kind == "fc" else 1) + wbytes
+            total += max(nbytes / hbm, 0.0 if dw else 2.0 * macs / tensor)
+            shape[op["dst"]] = (oh, ow, n)
+        elif kind == "add":
+            h, w, c = shape[op["a"]]
+            total += 3.0 * batch * h * w * c / hbm
+            shape[op["dst"]] = (h, w, c)
+        elif kind == "maxpool":
+            h, w, c = shape[op["src"]]
+            oh, ow = (h + 2 * op["pad"] - op["k"]) // op["stride"] + 1, (w + 2 * op["pad"] - op["k"]) // op["stride"] + 1
+            total += batch * (h * w + oh * ow) * c / hbm
+            shape[op["dst"]] = (oh, ow, c)
+        else:
+            h, w, c = shape[op["src"]]
+            total += batch * (h * w + 1) * c / hbm
+            shape[op["dst"]] = (1, 1, c)
+    return total * 1e3
+
+
+def time_networks(hq, qtz, torch, peaks, reps=10, detail=False):
     """Images/s of whole-network integer inference at the batch sizes of the network workloads
     (calibration and plan creation outside the timed region; activations stay in HBM)."""
     from paper_1806_08342_b200 import network
@@ -344,8 +409,11 @@ def time_networks(hq, qtz, torch, reps=10, detail=False):
             graph_ms = None
             res.setdefault("graph_errors", []).append(f"{name}: {type(exc).__name__}: {exc}"[:200])
         best = min(eager_ms, graph_ms) if graph_ms else eager_ms
+        bound = roofline_sum_ms(ops, batch, wbits, peaks)
         entry = {"batch": batch, "weight_bits": wbits, "ms_eager": round(eager_ms, 4),
-                 "ms_graph": None if graph_ms is None else round(graph_ms, 4), "images_per_s": round(batch / best * 1e3, 1)}
+                 "ms_graph": None if graph_ms is None else round(graph_ms, 4), "images_per_s": round(batch / best * 1e3, 1),
+                 "roofline_sum_ms": round(bound, 4), "frac_of_roofline_sum": round(bound / best, 3),
+                 "launches": net.num_launch_calls()}
         if detail:
             evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(net.layers) + 1)]
             t = net.tensors
@@ -374,6 +442,43 @@ def time_networks(hq, qtz, torch, reps=10, detail=False):
         del net
         torch.cuda.empty_cache()
     return res
+
+
+def probe_int8(hq, torch, device_index, sustained_seconds=4.0):
+    """tcgen05.mma kind::i8 alone (operands resident in shared memory, nothing loaded in the loop): a burst figure
+    (ten launches of about 1 ms) and one held for `sustained_seconds` with the SM clock sampled meanwhile."""
+    hq.probe_int8_peak(8192, 2)                                       # warm-up, module load
+    burst = max(hq.probe_int8_peak(16384, 10)[0] for _ in range(3))
+    sampler = ClockSampler(device_index)
+    sampler.start()
+    t0, ops_t, ms_t = time.time(), 0.0, 0.0
+    while time.time() - t0 < sustained_seconds:
+        tops, ms = hq.probe_int8_peak(16384, 100)
+        ops_t += tops * ms
+        ms_t += ms
+    clocks = sampler.stop()
+    return {"burst_tops": round(burst, 1), "sustained_tops": round(ops_t / ms_t, 1), "sustained_seconds": round(ms_t * 1e-3, 2),
+            "clocks_sustained": clocks, "how": "128x256x32 u8*s8->s32 MMAs back to back on shared-memory resident operands, one CTA per SM"}
+
+
+def sustained_gemm(case, torch, device_index, seconds=2.5):
+    """The largest size of the sweep back to back for `seconds`, with the SM clock sampled meanwhile."""
+    sampler = ClockSampler(device_index)
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        case.run()
+    torch.cuda.synchronize()
+    sampler.start()
+    t0, n, ms = time.time(), 0, 0.0
+    while time.time() - t0 < seconds:
+        s.record()
+        for _ in range(200):
+            case.run()
+        e.record(); torch.cuda.synchronize()
+        ms += s.elapsed_time(e); n += 200
+    clocks = sampler.stop()
+    return {"size": case.size, "launches": n, "seconds": round(ms * 1e-3, 2), "TOP/s": round(case.ops * n / (ms * 1e-3) / 1e12, 1),
+            "clocks": clocks, "includes": "pixel_sum_kernel pre-pass + conv_tc_kernel per launch"}
 
 
 def max_over_ranks(values, dist, device):
@@ -406,6 +511,9 @@ def run_ours(args, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     peaks = load_peaks()
     hq = qtz.Handle(local_rank)
+    if args.probe_int8:
+        print(json.dumps({"int8_probe": probe_int8(hq, torch, local_rank)}), flush=True)
+        return
     if args.hbm_only:
         print(json.dumps({"hbm_kernels": time_hbm_kernels(hq, qtz, torch, peaks)}), flush=True)
         return
@@ -413,7 +521,7 @@ def run_ours(args, rank, world, local_rank):
         print(json.dumps({"layers": [time_layer(hq, qtz, torch, sp) for sp in args.layer.split(";")]}), flush=True)
         return
     if args.networks_only:
-        print(json.dumps({"networks": time_networks(hq, qtz, torch, detail=True)}), flush=True)
+        print(json.dumps({"networks": time_networks(hq, qtz, torch, peaks, detail=True)}), flush=True)
         return
     cases = [GemmCase(hq, qtz, torch, s) for s in SIZES]
     torch.cuda.synchronize()
@@ -537,8 +645,15 @@ def run_ours(args, rank, world, local_rank):
         "sweep": sweep,
     }
     if world == 1 and not args.no_extras:
+        probe = probe_int8(hq, torch, local_rank, sustained_seconds=3.0)
+        out["roofline"]["int8_peak_measured"] = probe
+        out["roofline"]["frac_of_int8_measured_burst"] = kernel_tops / probe["burst_tops"]
+        sus = sustained_gemm(cases[-1], torch, local_rank)
+        sus["frac_of_sustained_peak"] = round(sus["TOP/s"] / (2.0 * peaks["bf16_sustained"]), 3)
+        sus["frac_of_int8_measured_sustained"] = round(sus["TOP/s"] / probe["sustained_tops"], 3)
+        out["sustained"] = sus
         out["hbm_kernels"] = time_hbm_kernels(hq, qtz, torch, peaks)
-        out["networks"] = time_networks(hq, qtz, torch)
+        out["networks"] = time_networks(hq, qtz, torch, peaks)
         out["cpu_baseline"] = cpu_baseline()
     print(json.dumps(out), flush=True)
     if dist is not None:
@@ -552,6 +667,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the HBM-kernel table and the CPU baseline")
+    ap.add_argument("--probe-int8", action="store_true",
+                    help="run only the tensor-core probe (tcgen05.mma kind::i8, burst and 4-s sustained); prints it as JSON")
     ap.add_argument("--hbm-only", action="store_true",
                     help="run only the element-wise / depthwise kernel table (profiling runs); prints it as JSON")
     ap.add_argument("--layer", default="", help='time single conv layers: "batch,h,w,c,n,k,stride[,dw];..." (profiling runs)')

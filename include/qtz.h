@@ -43,7 +43,7 @@ extern "C" {
 typedef int32_t qtz_status;
 #define QTZ_OK 0
 #define QTZ_ERR_INVALID_ARG (-1)    /* null pointer, non-positive size, bad enum            */
-#define QTZ_ERR_MISALIGNED (-2)     /* pointer or pitch not a multiple of 16 bytes          */
+#define QTZ_ERR_MISALIGNED (-2)     /* pointer or pitch misaligned (16 bytes unless a call says otherwise) */
 #define QTZ_ERR_UNSUPPORTED (-3)    /* well-formed request outside what is implemented      */
 #define QTZ_ERR_OVERFLOW (-4)       /* reduction length too large for int32 accumulation    */
 #define QTZ_ERR_NONFINITE (-5)      /* NaN or Inf met while calibrating                     */
@@ -98,6 +98,23 @@ QTZ_API const char* qtz_last_error(qtz_handle h);
  * QTZ_ERR_DEVICE_TIMEOUT with *site_id telling which wait.  Synchronises `stream`.        */
 QTZ_API qtz_status qtz_last_device_status(qtz_handle h, int32_t* site_id, void* stream);
 
+/* Cycle budget of every bounded device-side wait of later launches through this handle (default
+ * 2e9, about one second of SM clocks; at least 1000).  When a wait runs out the kernel records
+ * QTZ_ERR_DEVICE_TIMEOUT and returns; qtz_last_device_status reports it.                        */
+QTZ_API qtz_status qtz_set_wait_budget(qtz_handle h, int64_t cycles);
+/* Self-test of that mechanism: launches one small CTA that waits, for at most budget_cycles
+ * (1 .. 1e8), on a barrier nothing ever signals.  The wait gives up by itself and the kernel
+ * returns normally; afterwards qtz_last_device_status reports QTZ_ERR_DEVICE_TIMEOUT with site
+ * id 8.  Asynchronous on `stream`.  Nothing faults, traps or hangs.                             */
+QTZ_API qtz_status qtz_selftest_wait_timeout(qtz_handle h, int64_t budget_cycles, void* stream);
+/* Measures the tensor cores alone for the contraction of Eq. 5 (first term): one CTA per SM issues
+ * mmas_per_cta (>= 32, rounded down to a multiple of 32) tcgen05.mma kind::i8 instructions of
+ * 128 x 256 x 32 (u8 x s8 -> s32) on operands that stay in shared memory, `launches` times back
+ * to back.  Writes the achieved TOP/s (2 ops per multiply-accumulate) and, if ms_out is not NULL,
+ * the elapsed milliseconds of the timed launches (CUDA events on `stream`).  BLOCKS.             */
+QTZ_API qtz_status qtz_probe_int8_peak(qtz_handle h, int32_t mmas_per_cta, int32_t launches, double* tops_out,
+                                       float* ms_out, void* stream);
+
 /* ---- quantizer parameters (Sections 2.1, 2.2, 2.5, 2.6) ------------------------------- */
 
 /* Range estimation by min/max (Section 2.5) followed by parameter derivation.
@@ -138,7 +155,12 @@ QTZ_API qtz_status qtz_minmax(qtz_handle h, const float* x_dev, int64_t outer, i
  *     two calls whose kernels may overlap on the GPU -- different streams -- race on it: issue
  *     them in order on one stream, or synchronise in between;
  *   - the first call on each device looks the array's device address up
- *     (cudaGetSymbolAddress); make that first call before starting any stream capture.
+ *     (cudaGetSymbolAddress) and makes the CUDA runtime load this library's kernels and the
+ *     array onto that device, which takes a little device memory once: make one small warm-up
+ *     call per device early -- before a memory pool claims the rest of the GPU, and before
+ *     starting any stream capture.  If that first call fails for lack of memory it returns
+ *     QTZ_ERR_CUDA (there is no handle to ask for the error text).
+ * x_dev and out_dev must be 4-byte aligned (QTZ_ERR_MISALIGNED otherwise; no 16-byte rule here).
  * The call performs no cudaMalloc / cudaFree and uses no allocating library routine.         */
 QTZ_API qtz_status qtz_minmax_static(const float* x_dev, int64_t count, float* out_dev, void* stream);
 QTZ_API int64_t qtz_minmax_static_max_count(void);

@@ -53,8 +53,12 @@ def lib():
 
 def num_threads() -> int:
     """Threads the OpenMP loops of the oracle use."""
-    env = os.environ.get("OMP_NUM_THREADS")
-    return int(env) if env else (os.cpu_count() or 1)
+    return int(lib().orc_set_threads(0))
+
+
+def set_num_threads(n: int) -> int:
+    """Sets the number of OpenMP threads (timing runs); returns the value now in force."""
+    return int(lib().orc_set_threads(int(n)))
 
 
 def _p(a):

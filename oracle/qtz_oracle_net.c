@@ -8,6 +8,9 @@
  */
 #include <math.h>
 #include <stdint.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
 
 #include "orc_common.h"
 
@@ -50,4 +53,17 @@ int orc_add_output_range(const orc_qparams_net* a, const orc_qparams_net* b, int
     const float lo = a->min_nudged + b->min_nudged;
     const float hi = a->max_nudged + b->max_nudged;
     return orc_range_after_activation(lo, hi, kind, lo_out, hi_out);
+}
+
+/* Number of threads the oracle's OpenMP loops use from now on (timing runs report a   */
+/* one-thread figure beside the all-cores one).  Returns the value in force.            */
+int orc_set_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+    return omp_get_max_threads();
+#else
+    (void)n;
+    return 1;
+#endif
 }

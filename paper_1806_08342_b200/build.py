@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libqtz.so")
 SOURCES = ["qtz_host.cu", "qtz_elementwise.cu", "qtz_glue.cu", "qtz_conv_direct.cu", "qtz_depthwise.cu", "qtz_conv_tc.cu",
-           "qtz_plan.cu", "qtz_static.cu", "qtz_sim.cu"]
+           "qtz_plan.cu", "qtz_static.cu", "qtz_sim.cu", "qtz_probe.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--fmad=false",
               "-cudart", "static"]

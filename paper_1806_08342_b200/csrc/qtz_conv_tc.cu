@@ -1379,14 +1379,11 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.fast_requant = (!a.raw && p->rshift_min >= 33 && p->rshift_max <= 53) ? 1 : 0;
     a.fold = 0;                             // decided per launch (it depends on the zero points)
     a.status = h->status_dev;
-    a.wait_budget = 2000000000LL;  // about one second of SM clocks
+    a.wait_budget = h->wait_budget;
     t->grid = static_cast<int>(std::min<int64_t>(a.num_tiles, h->num_sms));
 
-    static bool attr_set = false;
-    if (!attr_set) {
-        QTZ_CUDA(h, cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr_set = true;
-    }
+    // per device, so set for the device of this plan every time (the call is cheap)
+    QTZ_CUDA(h, cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     return QTZ_OK;
 }
 
@@ -1397,6 +1394,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     qtz_tc_state* t = p->tc;
     const qtz_conv_desc& d = t->eff;
     TcArgs a = t->args;
+    a.wait_budget = h->wait_budget;
     const bool pw = is_pointwise(d);
 
     const uint8_t* xin = x;

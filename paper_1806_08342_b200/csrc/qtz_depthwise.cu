@@ -568,21 +568,18 @@ qtz_status qtz_depthwise_prepare(qtz_plan* p)
     *s = pick;
     a.taps = p->dw_taps; a.wsum = p->dw_wsum; a.bias = p->bias; a.mult = p->mult; a.rshift = p->rshift;
     a.status = p->h->status_dev;
-    a.wait_budget = 2000000000LL;
+    a.wait_budget = p->h->wait_budget;
     a.zw = p->w_zp_signed;
-    static bool attr_set = false;
-    if (!attr_set) {
-        for (int stride = 1; stride <= 2; ++stride)
-            for (int asym = 0; asym < 2; ++asym)
-                for (int mode = 0; mode < kNumModes; ++mode)
-                    for (int clamp = 0; clamp < 2; ++clamp) {
-                        const cudaError_t e = cudaFuncSetAttribute(pick_kernel(stride, asym != 0, mode, clamp != 0),
-                                                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                                   kDwSmemPerSm / 2);
-                        if (e != cudaSuccess) return qtz_cuda_fail(p->h, e, "cudaFuncSetAttribute(depthwise3x3_kernel)");
-                    }
-        attr_set = true;
-    }
+    // the attribute is per device: set it for this plan's device every time (cheap, and safe from any host thread)
+    for (int stride = 1; stride <= 2; ++stride)
+        for (int asym = 0; asym < 2; ++asym)
+            for (int mode = 0; mode < kNumModes; ++mode)
+                for (int clamp = 0; clamp < 2; ++clamp) {
+                    const cudaError_t e = cudaFuncSetAttribute(pick_kernel(stride, asym != 0, mode, clamp != 0),
+                                                               cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                               kDwSmemPerSm / 2);
+                    if (e != cudaSuccess) return qtz_cuda_fail(p->h, e, "cudaFuncSetAttribute(depthwise3x3_kernel)");
+                }
     return QTZ_OK;
 }
 
@@ -601,6 +598,7 @@ qtz_status qtz_depthwise_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, uin
     a.y = raw ? nullptr : y;
     a.y_raw = raw ? reinterpret_cast<int32_t*>(y) : nullptr;
     a.zx = x_zp; a.zy = y_zp; a.act_min = act_min; a.act_max = act_max;
+    a.wait_budget = p->h->wait_budget;
     CUtensorMap map;
     const uint64_t pitch = static_cast<uint64_t>(d.c_pitch_in);
     const uint64_t dims[4] = {static_cast<uint64_t>(d.c), static_cast<uint64_t>(d.w), static_cast<uint64_t>(d.h),

@@ -11,7 +11,7 @@ extern "C" const char* qtz_status_string(qtz_status s)
     switch (s) {
         case QTZ_OK: return "ok";
         case QTZ_ERR_INVALID_ARG: return "invalid argument";
-        case QTZ_ERR_MISALIGNED: return "pointer or pitch not 16-byte aligned";
+        case QTZ_ERR_MISALIGNED: return "pointer or pitch not aligned as the call requires";
         case QTZ_ERR_UNSUPPORTED: return "unsupported configuration";
         case QTZ_ERR_OVERFLOW: return "reduction too long for int32 accumulation";
         case QTZ_ERR_NONFINITE: return "non-finite value in calibration data";

@@ -24,6 +24,7 @@ struct qtz_ctx {
     int32_t* status_dev = nullptr;
     float* reduce_host = nullptr;  // pinned
     size_t reduce_host_bytes = 0;
+    long long wait_budget = 2000000000LL;   // cycle budget of every bounded device-side wait (about one second)
     std::string last_error;
 };
 
@@ -31,7 +32,8 @@ enum qtz_kernel_family { QTZ_K_DIRECT = 0, QTZ_K_TCGEN05 = 1, QTZ_K_DEPTHWISE = 
 
 // Device status sites (which bounded wait gave up).
 enum { QTZ_SITE_TMA_FULL = 1, QTZ_SITE_SMEM_EMPTY = 2, QTZ_SITE_TMEM_FULL = 3,
-       QTZ_SITE_TMEM_EMPTY = 4, QTZ_SITE_STORE = 5, QTZ_SITE_OUT_FULL = 6, QTZ_SITE_OUT_EMPTY = 7 };
+       QTZ_SITE_TMEM_EMPTY = 4, QTZ_SITE_STORE = 5, QTZ_SITE_OUT_FULL = 6, QTZ_SITE_OUT_EMPTY = 7,
+       QTZ_SITE_SELFTEST = 8, QTZ_SITE_PROBE = 9 };
 
 inline qtz_status qtz_cuda_fail(qtz_ctx* h, cudaError_t e, const char* what)
 {
@@ -51,6 +53,22 @@ inline qtz_status qtz_cuda_fail(qtz_ctx* h, cudaError_t e, const char* what)
         cudaError_t _e = cudaGetLastError();                           \
         if (_e != cudaSuccess) return qtz_cuda_fail((h), _e, name);    \
     } while (0)
+
+// Makes `device` current for the lifetime of the object and puts the caller's device back afterwards.
+struct qtz_device_guard {
+    int prev = -1;
+    bool switched = false;
+    explicit qtz_device_guard(int device)
+    {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != device) switched = cudaSetDevice(device) == cudaSuccess;
+    }
+    ~qtz_device_guard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+    qtz_device_guard(const qtz_device_guard&) = delete;
+    qtz_device_guard& operator=(const qtz_device_guard&) = delete;
+};
 
 static inline bool qtz_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -106,8 +106,9 @@ qtz_status validate_desc(const qtz_conv_desc& d, int depthwise)
 extern "C" qtz_status qtz_conv_destroy(qtz_conv_plan p)
 {
     if (!p) return QTZ_ERR_INVALID_ARG;
-    cudaSetDevice(p->device);
-    cudaDeviceSynchronize();
+    // cudaFree waits for the work that may still use a buffer before it releases it, so no
+    // device-wide synchronisation is needed here
+    qtz_device_guard guard(p->device);
     qtz_tc_release(p);
     qtz_depthwise_release(p);
     cudaFree(p->w_direct);
@@ -157,7 +158,7 @@ extern "C" qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, i
             if (mult_host[i] < 0 || rshift_host[i] < 1 || rshift_host[i] > 62) return QTZ_ERR_INVALID_ARG;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    QTZ_CUDA(h, cudaSetDevice(h->device));
+    qtz_device_guard guard(h->device);       // the caller's current device is restored on every return path
     qtz_plan* p = new (std::nothrow) qtz_plan();
     if (!p) return QTZ_ERR_INVALID_ARG;
     p->h = h;
@@ -270,6 +271,7 @@ extern "C" qtz_status qtz_conv2d_u8(qtz_conv_plan p, const uint8_t* x_dev, int32
     if (s != QTZ_OK) return s;
     if (p->depthwise) return QTZ_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    qtz_device_guard guard(p->device);
     if (p->family == QTZ_K_TCGEN05)
         return qtz_tc_launch(p, x_dev, x_zero_point, y_dev, y_zero_point, act_min, act_max, st);
     return qtz_direct_launch(p, x_dev, x_zero_point, y_dev, y_zero_point, act_min, act_max, st);
@@ -281,6 +283,7 @@ extern "C" qtz_status qtz_depthwise_u8(qtz_conv_plan p, const uint8_t* x_dev, in
     qtz_status s = check_run_args(p, x_dev, y_dev, x_zero_point, y_zero_point, act_min, act_max);
     if (s != QTZ_OK) return s;
     if (!p->depthwise) return QTZ_ERR_INVALID_ARG;
+    qtz_device_guard guard(p->device);
     return qtz_depthwise_launch(p, x_dev, x_zero_point, static_cast<uint8_t*>(y_dev), y_zero_point, act_min, act_max,
                                 static_cast<cudaStream_t>(stream));
 }

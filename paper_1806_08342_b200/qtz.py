@@ -45,6 +45,9 @@ SIGNATURES = {
     "qtz_status_string": (c_char_p, [c_int32]),
     "qtz_last_error": (c_char_p, [c_void_p]),
     "qtz_last_device_status": (c_int32, [c_void_p, POINTER(c_int32), c_void_p]),
+    "qtz_set_wait_budget": (c_int32, [c_void_p, c_int64]),
+    "qtz_selftest_wait_timeout": (c_int32, [c_void_p, c_int64, c_void_p]),
+    "qtz_probe_int8_peak": (c_int32, [c_void_p, c_int32, c_int32, POINTER(c_double), POINTER(c_float), c_void_p]),
     "qtz_calibrate_minmax": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int32, c_void_p,
                                        c_void_p]),
     "qtz_minmax": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p]),
@@ -264,6 +267,19 @@ class Handle:
         site = c_int32()
         rc = self.lib.qtz_last_device_status(self.h, byref(site), _stream())
         return rc, site.value
+
+    def set_wait_budget(self, cycles):
+        self._chk(self.lib.qtz_set_wait_budget(self.h, int(cycles)), "qtz_set_wait_budget")
+
+    def selftest_wait_timeout(self, budget_cycles):
+        self._chk(self.lib.qtz_selftest_wait_timeout(self.h, int(budget_cycles), _stream()), "qtz_selftest_wait_timeout")
+
+    def probe_int8_peak(self, mmas_per_cta=32768, launches=10):
+        """(TOP/s, ms) of tcgen05.mma kind::i8 issued back to back on shared-memory resident operands."""
+        tops, ms = c_double(), c_float()
+        self._chk(self.lib.qtz_probe_int8_peak(self.h, int(mmas_per_cta), int(launches), byref(tops), byref(ms), _stream()),
+                  "qtz_probe_int8_peak")
+        return tops.value, ms.value
 
     def calibrate_minmax(self, x, axis=None, bits=8, symmetric=False):
         _check_dev(x)

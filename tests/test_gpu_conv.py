@@ -239,16 +239,11 @@ def gemm_case(hq, m, n, k, seed=2, rows=None):
     return plan.kernel
 
 
-@pytest.mark.parametrize("size", [512, 1024])
+@pytest.mark.parametrize("size", [512, 1024, 2048, 4096, 8192])
 def test_gemm_workload_full_parity(hq, size):
+    # every row of every size: each 128-row pixel tile, each band of the tile rasterisation and each column
+    # tile is compared element by element (the oracle needs about half a minute for the three large sizes)
     gemm_case(hq, size, size, size)
-
-
-@pytest.mark.parametrize("size", [2048, 4096, 8192])
-def test_gemm_workload_sampled_rows(hq, size):
-    rows = np.unique(np.concatenate([np.arange(0, 130), synth.rng(5, size).integers(0, size, 64),
-                                     np.arange(size - 3, size)]))
-    gemm_case(hq, size, size, size, rows=rows)
 
 
 def test_gemm_ragged(hq):

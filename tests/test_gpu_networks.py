@@ -6,6 +6,10 @@ Small-batch cases compare all images at full 224x224 resolution; the full-batch 
 images, the launch configuration the benchmark uses) compare the calibration images plus sampled
 images, which the oracle computes one by one (images are independent once the quantizers are fixed).
 """
+import hashlib
+import json
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -69,5 +73,39 @@ def test_network_full_batch_sampled_images(hq, name, batch):
     got = net.build(images, 2)
     torch.cuda.synchronize()
     compare(net, got, want, rows)
+    rc, site = hq.device_status()
+    assert rc == 0, (rc, site)
+
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "network_hashes.json")
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_network_full_batch_every_image(hq, name):
+    """The whole batch the benchmark runs (128 / 256 images), every tensor of every layer: the SHA-256 of the
+    library's codes and quantizer record must equal the digest the oracle alone wrote
+    (tests/golden/make_network_hashes.py, which imports nothing of the CUDA library)."""
+    table = json.load(open(GOLDEN))
+    if name not in table:
+        pytest.skip(f"no oracle digests stored for {name}")
+    cfg = table[name]
+    ops = synth.NETWORKS[name]()
+    images = synth.network_input(cfg["batch"], 224, cfg["seed"])
+    net = network.QuantizedNetwork(hq, ops, cfg["seed"], cfg["weight_bits"])
+    got = net.build(images, cfg["calib"])
+    torch.cuda.synchronize()
+    assert set(cfg["tensors"]) == set(got)
+    wrong = []
+    for key, want in cfg["tensors"].items():
+        g = got[key].cpu().numpy()
+        h = hashlib.sha256()
+        if key == "logits":
+            h.update(np.ascontiguousarray(g).tobytes())
+        else:
+            h.update(np.ascontiguousarray(g[..., :net.chans[key]]).tobytes())
+            h.update(net.params[key].tobytes())
+        if h.hexdigest() != want:
+            wrong.append(key)
+    assert not wrong, f"{len(wrong)} of {len(cfg['tensors'])} tensors differ, first: {wrong[:3]}"
     rc, site = hq.device_status()
     assert rc == 0, (rc, site)

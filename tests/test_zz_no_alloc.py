@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_1806_08342_b200 import qtz, synth
 
 pytestmark = pytest.mark.gpu
@@ -31,7 +32,8 @@ def test_static_minmax_matches_allocating_entry_point_twice_in_a_row():
         g = got.cpu().numpy()
         assert g[0] == want_lo[0] and g[1] == want_hi[0]               # min/max are exact: same bits
         assert g[2:].view(np.uint32)[0] == 0
-        assert want_lo[0] == x.min().item() and want_hi[0] == x.max().item()
+        o_lo, o_hi = oracle.minmax(x.cpu().numpy())                     # and what the oracle's definition gives
+        assert g[0] == o_lo[0] and g[1] == o_hi[0]
     # misaligned start and a NaN: same verdicts as the allocating call
     got = qtz.minmax_static(first[3:1000], out=out).cpu().numpy()
     lo, hi = hq.minmax(first[3:1000])
@@ -54,3 +56,22 @@ def test_static_minmax_rejects_sizes_beyond_its_fixed_capacity():
     assert rc == -9 and b"capacity" in lib.qtz_status_string(rc)
     assert lib.qtz_minmax_static(None, 16, out.data_ptr(), None) == -1
     assert lib.qtz_minmax_static(x.data_ptr(), 0, out.data_ptr(), None) == -1
+
+
+def test_static_minmax_chunk_boundaries_and_no_allocation():
+    """One partial covers 65 536 values: sizes on either side of that boundary, a 16-byte aligned start with
+    a tail that is not a multiple of four, and the promise itself -- after the first call on the device (which
+    loads the kernels and looks the array's address up) a call leaves the amount of free device memory as it was."""
+    out = torch.empty(3, dtype=torch.float32, device="cuda")
+    base = synth.normal_f32((2 * 65536 + 64,), 43, 1, std=3.0)
+    dev_x = torch.from_numpy(base).cuda()
+    qtz.minmax_static(dev_x[:16], out=out)                              # the per-device set-up happens here
+    torch.cuda.synchronize()
+    for count in (1, 3, 65535, 65536, 65537, 2 * 65536 - 1, 2 * 65536 + 1, 65536 + 7):
+        free_before = torch.cuda.mem_get_info()[0]
+        g = qtz.minmax_static(dev_x[:count], out=out)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before, count       # nothing was allocated or freed
+        lo, hi = oracle.minmax(base[:count])
+        g = g.cpu().numpy()
+        assert g[0] == lo[0] and g[1] == hi[0] and g[2:].view(np.uint32)[0] == 0, count
