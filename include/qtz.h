@@ -165,6 +165,31 @@ QTZ_API qtz_status qtz_minmax(qtz_handle h, const float* x_dev, int64_t outer, i
 QTZ_API qtz_status qtz_minmax_static(const float* x_dev, int64_t count, float* out_dev, void* stream);
 QTZ_API int64_t qtz_minmax_static_max_count(void);
 
+/* Streaming range estimation for activations (Section 2.5: "a moving average of the minimum and
+ * maximum values across batches"; Section 3.1.2 calibrates on about 100 mini-batches).  The running
+ * state lives on the device, so a calibration loop enqueues one call per batch and tensor and never
+ * waits; one blocking read at the end turns the state into parameters.
+ *   state_dev   qtz_range_state_bytes(axis_len) bytes of device memory, 8-byte aligned, owned by the
+ *               caller; qtz_range_reset (or zero filling) starts a new average.
+ *   accumulate  min/max of this batch per index of the middle axis (the view of
+ *               qtz_calibrate_minmax), then state <- decay * state + (1 - decay) * batch in fp64
+ *               (0 <= decay < 1; the first batch initialises the state) -- the arithmetic of
+ *               qtz_ema_update, bit for bit.  A batch that holds NaN or Inf is skipped as a whole and
+ *               remembered.  Asynchronous on `stream`.
+ *   finish      BLOCKS once: copies the state to the host and writes, per axis index, the averaged
+ *               range rounded to fp32 (lo_host / hi_host, may be NULL) and the parameters derived from
+ *               it by the rules of qtz_params_from_range (params_host, may be NULL); *batches_host
+ *               (may be NULL) receives the number of batches folded in.  QTZ_ERR_NONFINITE if a batch
+ *               was skipped, QTZ_ERR_INVALID_ARG if nothing was accumulated.
+ * Calls that share a handle share its scratch: keep them on one stream.                          */
+QTZ_API int64_t qtz_range_state_bytes(int64_t axis_len);
+QTZ_API qtz_status qtz_range_reset(qtz_handle h, void* state_dev, int64_t axis_len, void* stream);
+QTZ_API qtz_status qtz_range_accumulate(qtz_handle h, const float* x_dev, int64_t outer, int64_t axis_len,
+                                        int64_t inner, double decay, void* state_dev, void* stream);
+QTZ_API qtz_status qtz_range_finish(qtz_handle h, const void* state_dev, int64_t axis_len, int32_t bits,
+                                    int32_t symmetric, float* lo_host, float* hi_host, qtz_qparams* params_host,
+                                    int32_t* batches_host, void* stream);
+
 /* Host-only: parameters from a known real range (same rules as above).                    */
 QTZ_API qtz_status qtz_params_from_range(float lo, float hi, int32_t bits, int32_t symmetric,
                                  qtz_qparams* out_host);

@@ -17,7 +17,7 @@ import subprocess
 import numpy as np
 
 _DIR = os.path.dirname(os.path.abspath(__file__))
-_SOURCES = ["qtz_oracle.c", "qtz_oracle_conv.c", "qtz_oracle_ops.c", "qtz_oracle_sim.c", "qtz_oracle_net.c"]
+_SOURCES = ["qtz_oracle.c", "qtz_oracle_conv.c", "qtz_oracle_ops.c", "qtz_oracle_sim.c", "qtz_oracle_net.c", "qtz_oracle_act4.c"]
 _LIB_PATH = os.path.join(_DIR, "liboracle.so")
 _lib = None
 
@@ -353,4 +353,29 @@ def add_output_range(a_params, b_params, kind):
     pb = np.ascontiguousarray(np.atleast_1d(b_params), dtype=QPARAMS)
     lo, hi = F32(), F32()
     _chk(lib().orc_add_output_range(_p(pa), _p(pb), I32(kind), ctypes.byref(lo), ctypes.byref(hi)))
+    return lo.value, hi.value
+
+
+def pack_u4(codes, packed_pitch=None):
+    """Unsigned 4-bit activation codes [..., k] (uint8, values 0..15) -> two per byte along k."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    k = codes.shape[-1]
+    pitch = (k + 1) // 2 if packed_pitch is None else packed_pitch
+    out = np.zeros(codes.shape[:-1] + (pitch,), np.uint8)
+    _chk(lib().orc_pack_u4(_p(codes), I64(codes.size // k), I64(k), I64(k), _p(out), I64(pitch)))
+    return out
+
+
+def unpack_u4(packed, k):
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    pitch = packed.shape[-1]
+    out = np.zeros(packed.shape[:-1] + (k,), np.uint8)
+    _chk(lib().orc_unpack_u4(_p(packed), I64(packed.size // pitch), I64(k), I64(pitch), _p(out), I64(k)))
+    return out
+
+
+def activation_range_bits(kind, y_scale, y_zero_point, bits):
+    lo, hi = I32(), I32()
+    _chk(lib().orc_activation_range_bits(int(kind), F32(y_scale), I32(y_zero_point), int(bits),
+                                         ctypes.byref(lo), ctypes.byref(hi)))
     return lo.value, hi.value

@@ -30,6 +30,7 @@
 #include <new>
 #include <vector>
 
+#include "qtz_device_util.cuh"
 #include "qtz_plan.cuh"
 #include "qtz_ptx.cuh"
 
@@ -788,15 +789,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ------------------------------------------------------------------------------------------
 constexpr int kPrepThreads = 256;
 
-__device__ __forceinline__ int32_t api_code_s8(const void* w, int wkind, int64_t row, int64_t k, int64_t k_total)
-{
-    if (wkind == QTZ_W_S8_PER_CHANNEL_SYM) return static_cast<const int8_t*>(w)[row * k_total + k];
-    if (wkind == QTZ_W_U8_PER_LAYER_ASYM) return static_cast<int32_t>(static_cast<const uint8_t*>(w)[row * k_total + k]) - 128;
-    const uint32_t byte = static_cast<const uint8_t*>(w)[row * ((k_total + 1) >> 1) + (k >> 1)];
-    const uint32_t nib = (k & 1) ? (byte >> 4) : (byte & 0xfu);
-    return static_cast<int32_t>(nib << 28) >> 28;
-}
-
 // OHWI codes -> int8 [n_pad][taps][c_pad], zero padded (K-major rows for the B operand).  The c
 // positions of a tap are c / cs runs of cs bytes, of which the first c_src come from the source
 // tensor (layers run over an im2col matrix pad every source tap from c_src to cs bytes; otherwise
@@ -814,7 +806,7 @@ prepack_tc_kernel(const void* __restrict__ w, int wkind, int n, int taps, int c,
     if (row < n && ch < c) {
         const int runs = c / cs, sub = ch / cs, cc = ch - sub * cs;
         if (cc < c_src)
-            v = static_cast<int8_t>(api_code_s8(w, wkind, row, (static_cast<int64_t>(tap) * runs + sub) * c_src + cc,
+            v = static_cast<int8_t>(qtz_dev::load_code_s8(w, wkind, row, (static_cast<int64_t>(tap) * runs + sub) * c_src + cc,
                                                 static_cast<int64_t>(taps) * runs * c_src));
     }
     out[i] = v;
@@ -952,7 +944,7 @@ prepack_rowwin_kernel(const void* __restrict__ w, int wkind, int n, int kh, int 
     const int px = byte / fp, ch = byte % fp;
     int8_t v = 0;
     if (row < n && px < kw && ch < c)
-        v = static_cast<int8_t>(api_code_s8(w, wkind, row, (static_cast<int64_t>(dy) * kw + px) * c + ch, static_cast<int64_t>(kh) * kw * c));
+        v = static_cast<int8_t>(qtz_dev::load_code_s8(w, wkind, row, (static_cast<int64_t>(dy) * kw + px) * c + ch, static_cast<int64_t>(kh) * kw * c));
     out[i] = v;
 }
 

@@ -6,6 +6,7 @@
 #include <cstring>
 #include <vector>
 
+#include "qtz_device_util.cuh"
 #include "qtz_internal.cuh"
 
 namespace {
@@ -15,48 +16,10 @@ constexpr int kThreads = 256;
 // ------------------------------------------------------------------------------------
 // min / max reduction
 // ------------------------------------------------------------------------------------
-struct Range {
-    float lo, hi;
-    unsigned bad;  // non-zero when a NaN or Inf was met
-};
-
-__device__ __forceinline__ void range_take(Range& r, float v)
-{
-    r.bad |= ((__float_as_uint(v) & 0x7f800000u) == 0x7f800000u);
-    r.lo = fminf(r.lo, v);
-    r.hi = fmaxf(r.hi, v);
-}
-
-__device__ __forceinline__ Range block_reduce(Range r)
-{
-    __shared__ float s_lo[kThreads / 32], s_hi[kThreads / 32];
-    __shared__ unsigned s_bad[kThreads / 32];
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        r.lo = fminf(r.lo, __shfl_xor_sync(0xffffffffu, r.lo, off));
-        r.hi = fmaxf(r.hi, __shfl_xor_sync(0xffffffffu, r.hi, off));
-        r.bad |= __shfl_xor_sync(0xffffffffu, r.bad, off);
-    }
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (lane == 0) {
-        s_lo[warp] = r.lo;
-        s_hi[warp] = r.hi;
-        s_bad[warp] = r.bad;
-    }
-    __syncthreads();
-    if (warp == 0) {
-        r.lo = lane < kThreads / 32 ? s_lo[lane] : FLT_MAX;
-        r.hi = lane < kThreads / 32 ? s_hi[lane] : -FLT_MAX;
-        r.bad = lane < kThreads / 32 ? s_bad[lane] : 0u;
-#pragma unroll
-        for (int off = 4; off > 0; off >>= 1) {
-            r.lo = fminf(r.lo, __shfl_xor_sync(0xffffffffu, r.lo, off));
-            r.hi = fmaxf(r.hi, __shfl_xor_sync(0xffffffffu, r.hi, off));
-            r.bad |= __shfl_xor_sync(0xffffffffu, r.bad, off);
-        }
-    }
-    return r;  // valid in thread 0
-}
+using qtz_dev::Range;
+using qtz_dev::range_take;
+using qtz_dev::block_reduce;
+static_assert(kThreads == qtz_dev::kReduceThreads, "block_reduce assumes this block size");
 
 // Per-layer reduction, first pass: every block streams a grid-strided share of the tensor
 // with 16-byte loads and leaves one (lo, hi, bad) triple in `partial`.
@@ -373,6 +336,106 @@ extern "C" qtz_status qtz_minmax(qtz_handle h, const float* x_dev, int64_t outer
         if (bad) return QTZ_ERR_NONFINITE;
         lo_host[a] = t[0];
         hi_host[a] = t[1];
+    }
+    return QTZ_OK;
+}
+
+// ---- streaming range estimation (Section 2.5: moving average of per-batch min and max) ----------
+namespace {
+
+// Device-resident state of qtz_range_accumulate: the averaged (lo, hi) per axis index in fp64 and a header.
+struct RangeHeader {
+    int32_t batches;      // batches folded in so far (0: the next batch initialises the state)
+    int32_t nonfinite;    // a batch held NaN or Inf: it was skipped and qtz_range_finish reports it
+    int32_t pad[2];
+};
+
+__host__ __device__ inline double* range_lo(void* state) { return reinterpret_cast<double*>(static_cast<char*>(state) + sizeof(RangeHeader)); }
+
+// One block: first agrees on whether this batch is usable at all (any non-finite value skips the whole
+// batch, as the host rule does), then state <- decay * state + (1 - decay) * batch, each product and the sum
+// rounded separately (no fused multiply-add), so that the host rule gives the same bits.
+__global__ void __launch_bounds__(kThreads)
+range_ema_kernel(const float* __restrict__ triples, int64_t axis_len, double keep, double take, void* state)
+{
+    RangeHeader* hdr = static_cast<RangeHeader*>(state);
+    double* lo = range_lo(state);
+    double* hi = lo + axis_len;
+    int bad = 0;
+    for (int64_t a = threadIdx.x; a < axis_len; a += kThreads) bad |= __float_as_uint(triples[3 * a + 2]) != 0u;
+    bad = __syncthreads_or(bad);
+    if (bad) {
+        if (threadIdx.x == 0) hdr->nonfinite = 1;
+        return;
+    }
+    const bool first = hdr->batches == 0;
+    for (int64_t a = threadIdx.x; a < axis_len; a += kThreads) {
+        const double blo = static_cast<double>(triples[3 * a]), bhi = static_cast<double>(triples[3 * a + 1]);
+        lo[a] = first ? blo : __dadd_rn(__dmul_rn(keep, lo[a]), __dmul_rn(take, blo));
+        hi[a] = first ? bhi : __dadd_rn(__dmul_rn(keep, hi[a]), __dmul_rn(take, bhi));
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) hdr->batches += 1;
+}
+
+}  // namespace
+
+extern "C" int64_t qtz_range_state_bytes(int64_t axis_len)
+{
+    if (axis_len <= 0 || axis_len > (1 << 30)) return 0;
+    return static_cast<int64_t>(sizeof(RangeHeader)) + 2 * static_cast<int64_t>(sizeof(double)) * axis_len;
+}
+
+extern "C" qtz_status qtz_range_reset(qtz_handle h, void* state_dev, int64_t axis_len, void* stream)
+{
+    if (!h || !state_dev || qtz_range_state_bytes(axis_len) == 0) return QTZ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(state_dev) & 7u) return QTZ_ERR_MISALIGNED;
+    QTZ_CUDA(h, cudaMemsetAsync(state_dev, 0, static_cast<size_t>(qtz_range_state_bytes(axis_len)), static_cast<cudaStream_t>(stream)));
+    return QTZ_OK;
+}
+
+extern "C" qtz_status qtz_range_accumulate(qtz_handle h, const float* x_dev, int64_t outer, int64_t axis_len, int64_t inner,
+                                           double decay, void* state_dev, void* stream)
+{
+    if (!h) return QTZ_ERR_INVALID_ARG;
+    qtz_status s = check_view(x_dev, state_dev, outer, axis_len, inner);
+    if (s != QTZ_OK) return s;
+    if (!(decay >= 0.0 && decay < 1.0) || qtz_range_state_bytes(axis_len) == 0) return QTZ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(x_dev) & 3u) || (reinterpret_cast<uintptr_t>(state_dev) & 7u)) return QTZ_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    s = launch_minmax(h, x_dev, outer, axis_len, inner, st);
+    if (s != QTZ_OK) return s;
+    range_ema_kernel<<<1, kThreads, 0, st>>>(h->reduce_dev, axis_len, decay, 1.0 - decay, state_dev);
+    QTZ_LAUNCH_CHECK(h, "range_ema_kernel");
+    return QTZ_OK;
+}
+
+extern "C" qtz_status qtz_range_finish(qtz_handle h, const void* state_dev, int64_t axis_len, int32_t bits, int32_t symmetric,
+                                       float* lo_host, float* hi_host, qtz_qparams* params_host, int32_t* batches_host,
+                                       void* stream)
+{
+    if (!h || !state_dev || qtz_range_state_bytes(axis_len) == 0) return QTZ_ERR_INVALID_ARG;
+    if (params_host && (bits < 2 || bits > 8)) return QTZ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t bytes = static_cast<size_t>(qtz_range_state_bytes(axis_len));
+    std::vector<char> host(bytes);
+    QTZ_CUDA(h, cudaMemcpyAsync(host.data(), state_dev, bytes, cudaMemcpyDeviceToHost, st));
+    QTZ_CUDA(h, cudaStreamSynchronize(st));
+    const RangeHeader* hdr = reinterpret_cast<const RangeHeader*>(host.data());
+    if (batches_host) *batches_host = hdr->batches;
+    if (hdr->nonfinite) return QTZ_ERR_NONFINITE;
+    if (hdr->batches == 0) return QTZ_ERR_INVALID_ARG;       // nothing was accumulated
+    const double* lo = range_lo(host.data());
+    const double* hi = lo + axis_len;
+    for (int64_t a = 0; a < axis_len; ++a) {
+        const float flo = static_cast<float>(lo[a]), fhi = static_cast<float>(hi[a]);
+        if (lo_host) lo_host[a] = flo;
+        if (hi_host) hi_host[a] = fhi;
+        if (params_host) {
+            const qtz_status s = symmetric ? qtz_host_symmetric_params(flo, fhi, bits, params_host + a)
+                                           : qtz_host_affine_params(flo, fhi, bits, params_host + a);
+            if (s != QTZ_OK) return s;
+        }
     }
     return QTZ_OK;
 }

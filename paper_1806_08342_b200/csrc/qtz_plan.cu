@@ -5,22 +5,14 @@
 #include <new>
 #include <vector>
 
+#include "qtz_device_util.cuh"
 #include "qtz_plan.cuh"
 
 namespace {
 
 constexpr int kThreads = 256;
 
-// Reads weight code k of output channel `row` from the API layout and moves it to int8:
-// int8 stays, uint8 is shifted by -128 (its zero point moves with it), 4-bit is sign-extended.
-__device__ __forceinline__ int32_t load_code_s8(const void* w, int wkind, int64_t row, int64_t k, int64_t k_total)
-{
-    if (wkind == QTZ_W_S8_PER_CHANNEL_SYM) return static_cast<const int8_t*>(w)[row * k_total + k];
-    if (wkind == QTZ_W_U8_PER_LAYER_ASYM) return static_cast<int32_t>(static_cast<const uint8_t*>(w)[row * k_total + k]) - 128;
-    const uint32_t byte = static_cast<const uint8_t*>(w)[row * ((k_total + 1) >> 1) + (k >> 1)];
-    const uint32_t nib = (k & 1) ? (byte >> 4) : (byte & 0xfu);
-    return static_cast<int32_t>(nib << 28) >> 28;
-}
+using qtz_dev::load_code_s8;
 
 __global__ void __launch_bounds__(kThreads)
 prepack_direct_kernel(const void* __restrict__ w, int wkind, int n, int k_total, int n_padded, int k_padded,

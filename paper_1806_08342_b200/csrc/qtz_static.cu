@@ -14,6 +14,7 @@
 #include <cfloat>
 #include <mutex>
 
+#include "qtz_device_util.cuh"
 #include "qtz_internal.cuh"
 
 namespace {
@@ -27,46 +28,11 @@ constexpr int kMaxDevices = 64;
 // the first pass overwrites exactly the entries the second pass reads.
 static __device__ __align__(256) float g_minmax_partials[3 * kMaxPartials];
 
-struct Range {
-    float lo, hi;
-    unsigned bad;
-};
+using qtz_dev::Range;
+static_assert(kThreads == qtz_dev::kReduceThreads, "block_reduce assumes this block size");
 
-__device__ __forceinline__ void take(Range& r, float v)
-{
-    r.bad |= ((__float_as_uint(v) & 0x7f800000u) == 0x7f800000u);
-    r.lo = fminf(r.lo, v);
-    r.hi = fmaxf(r.hi, v);
-}
-
-__device__ __forceinline__ Range reduce_block(Range r)
-{
-    __shared__ float s_lo[kThreads / 32], s_hi[kThreads / 32];
-    __shared__ unsigned s_bad[kThreads / 32];
-    for (int off = 16; off > 0; off >>= 1) {
-        r.lo = fminf(r.lo, __shfl_xor_sync(0xffffffffu, r.lo, off));
-        r.hi = fmaxf(r.hi, __shfl_xor_sync(0xffffffffu, r.hi, off));
-        r.bad |= __shfl_xor_sync(0xffffffffu, r.bad, off);
-    }
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (lane == 0) {
-        s_lo[warp] = r.lo;
-        s_hi[warp] = r.hi;
-        s_bad[warp] = r.bad;
-    }
-    __syncthreads();
-    if (warp == 0) {
-        r.lo = lane < kThreads / 32 ? s_lo[lane] : FLT_MAX;
-        r.hi = lane < kThreads / 32 ? s_hi[lane] : -FLT_MAX;
-        r.bad = lane < kThreads / 32 ? s_bad[lane] : 0u;
-        for (int off = 4; off > 0; off >>= 1) {
-            r.lo = fminf(r.lo, __shfl_xor_sync(0xffffffffu, r.lo, off));
-            r.hi = fmaxf(r.hi, __shfl_xor_sync(0xffffffffu, r.hi, off));
-            r.bad |= __shfl_xor_sync(0xffffffffu, r.bad, off);
-        }
-    }
-    return r;  // valid in thread 0
-}
+__device__ __forceinline__ void take(Range& r, float v) { qtz_dev::range_take(r, v); }
+__device__ __forceinline__ Range reduce_block(Range r) { return qtz_dev::block_reduce(r); }
 
 // First pass: block b reduces elements [b*kChunk, (b+1)*kChunk) and writes one triple.
 __global__ void __launch_bounds__(kThreads)

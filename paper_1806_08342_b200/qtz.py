@@ -53,6 +53,11 @@ SIGNATURES = {
     "qtz_minmax": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p]),
     "qtz_minmax_static": (c_int32, [c_void_p, c_int64, c_void_p, c_void_p]),
     "qtz_minmax_static_max_count": (c_int64, []),
+    "qtz_range_state_bytes": (c_int64, [c_int64]),
+    "qtz_range_reset": (c_int32, [c_void_p, c_void_p, c_int64, c_void_p]),
+    "qtz_range_accumulate": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_double, c_void_p, c_void_p]),
+    "qtz_range_finish": (c_int32, [c_void_p, c_void_p, c_int64, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
+                                   POINTER(c_int32), c_void_p]),
     "qtz_params_from_range": (c_int32, [c_float, c_float, c_int32, c_int32, c_void_p]),
     "qtz_quantize_tensor": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int32, c_int32,
                                       c_void_p, c_void_p]),
@@ -297,6 +302,31 @@ class Handle:
         lo, hi = np.zeros(a, np.float32), np.zeros(a, np.float32)
         self._chk(self.lib.qtz_minmax(self.h, _ptr(x), o, a, i, _np(lo), _np(hi), _stream()), "qtz_minmax")
         return lo, hi
+
+    def range_state(self, axis_len=1):
+        """A zeroed device buffer for range_accumulate (torch owns the memory)."""
+        n = self.lib.qtz_range_state_bytes(int(axis_len))
+        return torch.zeros(n // 8, dtype=torch.float64, device=f"cuda:{self.device}")
+
+    def range_reset(self, state, axis_len=1):
+        self._chk(self.lib.qtz_range_reset(self.h, _ptr(state), int(axis_len), _stream()), "qtz_range_reset")
+
+    def range_accumulate(self, x, state, decay, axis=None):
+        """Folds the min/max of batch `x` into the device-resident moving average; does not wait."""
+        _check_dev(x, state)
+        assert x.dtype == torch.float32
+        o, a, i = _view(x.shape, axis)
+        self._chk(self.lib.qtz_range_accumulate(self.h, _ptr(x), o, a, i, float(decay), _ptr(state), _stream()),
+                  "qtz_range_accumulate")
+
+    def range_finish(self, state, axis_len=1, bits=8, symmetric=False):
+        """One blocking read: (lo, hi, params, batches) of the averaged ranges."""
+        lo, hi = np.zeros(axis_len, np.float32), np.zeros(axis_len, np.float32)
+        params = np.zeros(axis_len, QPARAMS)
+        batches = c_int32()
+        self._chk(self.lib.qtz_range_finish(self.h, _ptr(state), int(axis_len), bits, int(symmetric), _np(lo), _np(hi),
+                                            _np(params), byref(batches), _stream()), "qtz_range_finish")
+        return lo, hi, params, batches.value
 
     def quantize_tensor(self, x, params, axis=None, out_dtype=U8, restrict_range=False, out=None):
         _check_dev(x, out)
