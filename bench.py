@@ -415,28 +415,19 @@ def time_networks(hq, qtz, torch, peaks, reps=10, detail=False):
                  "roofline_sum_ms": round(bound, 4), "frac_of_roofline_sum": round(bound / best, 3),
                  "launches": net.num_launch_calls()}
         if detail:
-            evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(net.layers) + 1)]
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(net.schedule) + 1)]
             t = net.tensors
             evs[0].record()
-            for i, L in enumerate(net.layers):
-                op = L.op
-                if op["op"] in ("conv", "fc"):
-                    L.plan(t[op["src"]], *L.args, out=t[op["dst"]])
-                elif op["op"] == "add":
-                    a = L.args
-                    hq.add_u8(t[op["a"]], a[0], a[1], t[op["b"]], a[2], a[3], a[4], a[5], a[6], a[7], a[8], out=t[op["dst"]])
-                elif op["op"] == "maxpool":
-                    hq.maxpool_u8(t[op["src"]], *L.args, out=t[op["dst"]])
-                else:
-                    hq.global_avgpool_u8(t[op["src"]], *L.args, out=t[op["dst"]])
+            for i, item in enumerate(net.schedule):
+                net.run_item(item)
                 evs[i + 1].record()
             torch.cuda.synchronize()
             rows = []
-            for i, L in enumerate(net.layers):
-                op = L.op
-                kern = L.plan.kernel if op["op"] in ("conv", "fc") else op["op"]
-                rows.append((round(evs[i].elapsed_time(evs[i + 1]) * 1e3, 1), op.get("dst"), kern,
-                             tuple(t[op["dst"]].shape)))
+            for i, item in enumerate(net.schedule):
+                L = item[2] if item[0] == "conv+add" else item[1]
+                kern = item[1].plan.detail if item[0] in ("conv", "fc", "conv+add") else item[0]
+                rows.append((round(evs[i].elapsed_time(evs[i + 1]) * 1e3, 1), L.op.get("dst"), kern,
+                             tuple(t[L.op["dst"]].shape)))
             entry["layers_us"] = rows
         res[name] = entry
         del net

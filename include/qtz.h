@@ -63,7 +63,7 @@ typedef struct {
     float max_nudged;   /* real value of the highest code, (L - z) * Delta  */
 } qtz_qparams;
 
-typedef enum { QTZ_U8 = 0, QTZ_S8 = 1, QTZ_S4_PACKED = 2, QTZ_S32 = 3 } qtz_dtype;
+typedef enum { QTZ_U8 = 0, QTZ_S8 = 1, QTZ_S4_PACKED = 2, QTZ_S32 = 3, QTZ_U4_PACKED = 4 } qtz_dtype;
 
 typedef enum {
     QTZ_W_S8_PER_CHANNEL_SYM = 0,       /* int8 codes, one scale per output channel, z_w = 0 */
@@ -199,10 +199,11 @@ QTZ_API qtz_status qtz_params_from_range(float lo, float hi, int32_t bits, int32
 /* x_int = round(x / Delta) + z, clamped to the code range (Eq. 1-2; Eq. 7-11 with z = 0).
  * The quotient is one IEEE fp32 division and round() is round-half-to-even.  Code ranges:
  *   QTZ_U8 [0,255] (restrict_range: [0,254]); QTZ_S8 [-128,127] (restrict_range, Eq. 10:
- *   [-127,127]); QTZ_S4_PACKED [-8,7] (restrict_range: [-7,7]).
+ *   [-127,127]); QTZ_S4_PACKED [-8,7] (restrict_range: [-7,7]); QTZ_U4_PACKED [0,15]
+ *   (restrict_range: [0,14]) -- 4-bit activations, Section 3.2.4.
  * NaN maps to the lowest code, +-Inf saturate.
  * params_host: axis_len entries, read before the call returns.
- * QTZ_S4_PACKED: two's-complement nibbles packed along the innermost run of the view
+ * QTZ_S4_PACKED / QTZ_U4_PACKED: nibbles (two's complement / unsigned) packed along the innermost run of the view
  * (`inner`, or `axis_len` when inner == 1): element 2i in the low nibble and 2i+1 in the
  * high nibble of byte i; each run occupies (len+1)/2 bytes, an odd tail's high nibble is 0. */
 QTZ_API qtz_status qtz_quantize_tensor(qtz_handle h, const float* x_dev, int64_t outer,
@@ -256,6 +257,24 @@ QTZ_API qtz_status qtz_ema_update(double* state_lo_host, double* state_hi_host, 
 QTZ_API qtz_status qtz_rescale_u8(qtz_handle h, const uint8_t* x_dev, int32_t x_zp, int32_t mult, int32_t rshift,
                                   uint8_t* y_dev, int32_t y_zp, int32_t act_min, int32_t act_max, int64_t pixels,
                                   int32_t c, int32_t x_pitch, int32_t y_pitch, void* stream);
+
+/* ---- activations at fewer than 8 bits (Section 3.2.4, Table 6: 4-bit activations) --------------- */
+
+/* A convolution takes its activations as one code per byte; 4-bit codes (0..15) go through it
+ * unchanged, with act_max <= 15 as the clamp of a 4-bit output.  For storage they pack two per
+ * byte: element 2i of a pixel's channels in the low nibble of byte i, element 2i+1 in the high
+ * nibble, an odd tail leaves the high nibble zero.
+ *   qtz_pack_u4    x [pixels][c] one code per byte, pitch x_pitch -> y [pixels][(c+1)/2], pitch y_pitch;
+ *                  only the low four bits of a code are kept.
+ *   qtz_unpack_u4  the reverse; bytes of y beyond c in a pixel are left untouched.
+ * No alignment rules (rows that are 4-byte aligned on both sides take a faster path).           */
+QTZ_API qtz_status qtz_pack_u4(qtz_handle h, const uint8_t* x_dev, int64_t pixels, int32_t c, int32_t x_pitch,
+                               uint8_t* y_dev, int32_t y_pitch, void* stream);
+QTZ_API qtz_status qtz_unpack_u4(qtz_handle h, const uint8_t* x_dev, int64_t pixels, int32_t c, int32_t x_pitch,
+                                 uint8_t* y_dev, int32_t y_pitch, void* stream);
+/* qtz_activation_range for an output of `bits` bits (2..8): the top code is 2^bits - 1.          */
+QTZ_API qtz_status qtz_activation_range_bits(int32_t kind, float y_scale, int32_t y_zero_point, int32_t bits,
+                                             int32_t* act_min, int32_t* act_max);
 
 /* ---- batch-norm folding (Eq. 20-21) ------------------------------------------------------ */
 
@@ -342,6 +361,12 @@ QTZ_API qtz_status qtz_conv_destroy(qtz_conv_plan p);
 QTZ_API qtz_status qtz_conv_set_profile_events(qtz_conv_plan p, void* start_event, void* stop_event);
 /* Name of the kernel family a plan dispatches to ("tcgen05", "direct", "depthwise").           */
 QTZ_API const char* qtz_conv_plan_kernel(qtz_conv_plan p);
+/* How the plan's most recent launch ran, as text: the family, the layer form and where the weights
+ * lived ("tcgen05 pointwise weights:int4-expanded-in-smem": packed 4-bit codes read from global
+ * memory and expanded to int8 in shared memory -- the on-the-fly decompression Section 7 asks
+ * hardware for; "weights:resident" / "weights:streamed": int8 codes).  Valid until the next launch
+ * or destroy; before the first launch it is the family name.                                      */
+QTZ_API const char* qtz_conv_plan_detail(qtz_conv_plan p);
 
 /* Quantized convolution, evaluated through the expansion of Eq. 5-6:
  *   acc = conv(w_Q, x_Q) - z_w sum(x_Q) - z_x sum(w_Q) + K_valid z_x z_w + bias_q
@@ -353,6 +378,26 @@ QTZ_API const char* qtz_conv_plan_kernel(qtz_conv_plan p);
 QTZ_API qtz_status qtz_conv2d_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point,
                          void* y_dev, int32_t y_zero_point, int32_t act_min, int32_t act_max,
                          void* stream);
+/* Convolution with the element-wise add that follows it fused into the epilogue (Section 3.2.1: "the
+ * addition and the activation fuse"; Section 7 recommends aggressive operator fusion).  Computes exactly
+ * what qtz_conv2d_u8 followed by qtz_add_u8 computes, without ever storing the intermediate tensor:
+ *   t = clamp(t_zero_point + ((acc mult[n] + 2^(rshift[n]-1)) >> rshift[n]), t_act_min, t_act_max)
+ *   y = clamp(z_y + (((t - t_zero_point) t_mult + (s - s_zero_point) s_mult + 2^(r-1)) >> r), act_min, act_max)
+ * where acc is the accumulator of qtz_conv2d_u8, (t_zero_point, t_act_min, t_act_max) the quantizer and
+ * clamp of the convolution's own output, s_dev the other addend (uint8, the geometry and pitch of the
+ * output; it may be y_dev itself), and (t_mult, s_mult, r = rshift) come from qtz_add_params.
+ * Both roundings of the two-step definition are kept, so results equal the unfused pair bit for bit.
+ * Errors: QTZ_ERR_UNSUPPORTED when the plan does not run on the tensor-core path or its output kind is
+ * not QTZ_OUT_U8 (run the two calls separately then), or when rshift > 53.                          */
+typedef struct {
+    int32_t t_zero_point, t_act_min, t_act_max; /* quantizer of the convolution's own output t        */
+    int32_t t_mult;                             /* multiplier of (t - t_zero_point) in the add        */
+    int32_t s_zero_point, s_mult;               /* zero point and multiplier of the other addend      */
+    int32_t rshift;                             /* right shift of the add                             */
+} qtz_residual;
+QTZ_API qtz_status qtz_conv2d_add_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point,
+                                     const qtz_residual* r_host, const uint8_t* s_dev, void* y_dev,
+                                     int32_t y_zero_point, int32_t act_min, int32_t act_max, void* stream);
 /* Depthwise form of the same (depth multiplier 1; Section 3.1.3 networks): the sum runs over
  * the kh x kw taps of one channel.  Plan must have been created with depthwise != 0.           */
 QTZ_API qtz_status qtz_depthwise_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point,

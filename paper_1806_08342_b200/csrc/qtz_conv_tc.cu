@@ -28,8 +28,10 @@
 #include <algorithm>
 #include <cstring>
 #include <new>
+#include <string>
 #include <vector>
 
+#include "qtz_add_math.cuh"
 #include "qtz_device_util.cuh"
 #include "qtz_plan.cuh"
 #include "qtz_ptx.cuh"
@@ -49,6 +51,7 @@ constexpr int kMaxObuf = 4;
 constexpr int kMaxStages = 8;
 constexpr int kNumBarriers = 2 * kMaxStages + 2 * kMaxAcc + 2 * kEpiGroups * kMaxObuf + 1;
 constexpr int kResidentBMax = 80 * 1024;   // weights of a whole layer stay in shared memory up to this size
+constexpr int kResidentB4Max = 128 * 1024; // ... and up to this size when they arrive as packed 4-bit codes
 constexpr int kMaxCls = 16;
 constexpr int kRunBytes = 2048;      // row-window layers: bytes of a frame row one copy brings in (256 elements of 8 bytes)
 constexpr int kRunCols = 120;        // ... and the output columns of a tile: 16 * 119 + rb <= 2048 for rb <= 128
@@ -99,6 +102,8 @@ struct TcArgs {
     int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
     int32_t obuf;                           // staging boxes per epilogue group (1..4)
     int32_t bres;                           // weight K blocks kept resident in shared memory (0: weights go through the ring)
+    const uint8_t* w4;                      // non-NULL: the resident weights arrive as packed 4-bit codes [n_pad][w4_row] (two per byte
+    int32_t w4_row;                         // along K) and the epilogue warps expand them to int8 in shared memory before the first tile
     int32_t spb;                            // K blocks per ring stage (one barrier handshake covers them all)
     int32_t n_acc, acc_stride;              // accumulators in TMEM and the columns between them
     int32_t gwarps;                         // warps per epilogue group: 4 (up to four groups) or 8 (up to two)
@@ -114,6 +119,14 @@ struct TcArgs {
     int32_t* y_raw;
     int32_t* status;
     long long wait_budget;
+    // Fused residual add (Section 3.2.1): the convolution's own output code t (quantizer zy / act_min / act_max
+    // above) is never stored; the shortcut tile s is brought into the output staging box by the store lane, and
+    // the epilogue replaces it in place by clamp(z_y + ((t - z_t) m_t + (s - z_s) m_s + 2^(r-1)) >> r).
+    int32_t res;                            // 0: plain convolution
+    int32_t res_kind;                       // arithmetic form of the add by its shift (see qtz_add_math.cuh)
+    qtz_add::AddRule res_rule;
+    qtz_add::AddSplit res_split;
+    int64_t res_addend;
 };
 
 struct SmemLayout {
@@ -258,7 +271,7 @@ __device__ __forceinline__ void tile_origin(const TcArgs& a, uint32_t m_tile, in
 
 __global__ void __launch_bounds__(kThreadsTc, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_y, const TcArgs a)
+               const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_s, const TcArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -292,12 +305,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             mbar_init(bar_ofull + 8 * i, a.gwarps);
             mbar_init(bar_oempty + 8 * i, 1);
         }
-        mbar_init(bar_wres, 1);
+        mbar_init(bar_wres, a.w4 ? kEpiWarps : 1);    // one arrival per expanding warp, or the producer's expect_tx
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_a);
         prefetch_tensormap(&map_b);
         prefetch_tensormap(&map_y);
+        if (a.res) prefetch_tensormap(&map_s);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
@@ -323,7 +337,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int nst = kblocks / a.spb;         // ring stages per tile
         uint32_t stage = 0, phase = 0;
         bool failed = false;
-        if (wres && blockIdx.x < a.num_tiles) {
+        if (wres && a.w4 == nullptr && blockIdx.x < a.num_tiles) {
             // the layer's weights are small: fetch all of their K blocks once, they stay for every tile
             if (elect_one()) {
                 mbar_arrive_expect_tx(bar_wres, static_cast<uint32_t>(a.bres) * L.b_blk);
@@ -537,42 +551,86 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t out_addr = base + L.out_off + grp * a.obuf * box_bytes;
             const uint32_t ofull = bar_ofull + 8 * kMaxObuf * grp, oempty = bar_oempty + 8 * kMaxObuf * grp;
             const bool lag = a.obuf >= 3;            // release a box one store late: its read is long over by then
-            uint32_t slot = 0, phase = 0, prev_slot = 0;
-            bool have_prev = false, ok = true;
-            for (uint32_t tile = blockIdx.x + grp * gridDim.x; ok && tile < a.num_tiles; tile += a.groups * gridDim.x) {
-                int n_tile;
-                uint32_t m_tile;
-                decode_tile(a, tile, m_tile, n_tile);
-                int w0, h0, b0;
-                tile_origin(a, m_tile, w0, h0, b0);
-                for (int nn = n_tile * a.BN, left = a.BN; left > 0 && nn < a.N; nn += a.out_box, left -= a.out_box) {
-                    if (!mbar_wait(ofull + 8 * slot, phase, a.wait_budget, 128u)) {
-                        report_timeout(a.status, QTZ_SITE_OUT_FULL);
-                        *abort_flag = 1;
-                        ok = false;
-                        break;
-                    }
-                    if (a.is4d)
-                        tma_store_4d(&map_y, out_addr + slot * box_bytes, nn, w0, h0, b0);
-                    else
-                        tma_store_2d(&map_y, out_addr + slot * box_bytes, nn, w0);
-                    tma_store_commit();
-                    if (lag) {
-                        if (have_prev) {
-                            tma_store_wait_read_n<1>();
-                            mbar_arrive(oempty + 8 * prev_slot);
-                        }
-                        prev_slot = slot;
-                        have_prev = true;
-                    } else {
-                        tma_store_wait_read();
-                        mbar_arrive(oempty + 8 * slot);
-                    }
-                    if (++slot == static_cast<uint32_t>(a.obuf)) {
-                        slot = 0;
-                        phase ^= 1;
-                    }
+            // the boxes of this group's tiles, in the order the epilogue fills them
+            struct BoxIter {
+                uint32_t tile;
+                int nn, left, w0, h0, b0;
+            };
+            auto enter_tile = [&](BoxIter& it) {
+                // (a column tile that lies wholly beyond the real channels has no box at all: skip it)
+                for (; it.tile < a.num_tiles; it.tile += a.groups * gridDim.x) {
+                    int n_tile;
+                    uint32_t m_tile;
+                    decode_tile(a, it.tile, m_tile, n_tile);
+                    it.nn = n_tile * a.BN;
+                    it.left = a.BN;
+                    if (it.nn >= a.N) continue;
+                    tile_origin(a, m_tile, it.w0, it.h0, it.b0);
+                    return;
                 }
+            };
+            auto advance = [&](BoxIter& it) {
+                it.nn += a.out_box;
+                it.left -= a.out_box;
+                if (!(it.left > 0 && it.nn < a.N)) {
+                    it.tile += a.groups * gridDim.x;
+                    enter_tile(it);
+                }
+            };
+            // with a fused residual add a box is handed to the epilogue by the arrival of its shortcut tile: the
+            // "empty" barrier of the box carries the bytes of that copy
+            auto fetch_shortcut = [&](uint32_t slot_, const BoxIter& it) {
+                mbar_arrive_expect_tx(oempty + 8 * slot_, static_cast<uint32_t>(a.rows * a.out_box));   // a box has a.rows rows
+                if (a.is4d)
+                    tma_load_4d(out_addr + slot_ * box_bytes, &map_s, oempty + 8 * slot_, it.nn, it.w0, it.h0, it.b0);
+                else
+                    tma_load_2d(out_addr + slot_ * box_bytes, &map_s, oempty + 8 * slot_, it.nn, it.w0);
+            };
+            BoxIter cur{blockIdx.x + grp * gridDim.x, 0, 0, 0, 0, 0};
+            enter_tile(cur);
+            BoxIter ahead = cur;
+            if (a.res)
+                for (uint32_t i = 0; i < static_cast<uint32_t>(a.obuf) && ahead.tile < a.num_tiles; ++i) {
+                    fetch_shortcut(i, ahead);
+                    advance(ahead);
+                }
+            auto release = [&](uint32_t slot_) {
+                if (!a.res) {
+                    mbar_arrive(oempty + 8 * slot_);
+                } else if (ahead.tile < a.num_tiles) {
+                    fetch_shortcut(slot_, ahead);
+                    advance(ahead);
+                }
+            };
+            uint32_t slot = 0, phase = 0, prev_slot = 0;
+            bool have_prev = false;
+            while (cur.tile < a.num_tiles) {
+                if (!mbar_wait(ofull + 8 * slot, phase, a.wait_budget, 128u)) {
+                    report_timeout(a.status, QTZ_SITE_OUT_FULL);
+                    *abort_flag = 1;
+                    break;
+                }
+                if (a.is4d)
+                    tma_store_4d(&map_y, out_addr + slot * box_bytes, cur.nn, cur.w0, cur.h0, cur.b0);
+                else
+                    tma_store_2d(&map_y, out_addr + slot * box_bytes, cur.nn, cur.w0);
+                tma_store_commit();
+                if (lag) {
+                    if (have_prev) {
+                        tma_store_wait_read_n<1>();
+                        release(prev_slot);
+                    }
+                    prev_slot = slot;
+                    have_prev = true;
+                } else {
+                    tma_store_wait_read();
+                    release(slot);
+                }
+                if (++slot == static_cast<uint32_t>(a.obuf)) {
+                    slot = 0;
+                    phase ^= 1;
+                }
+                advance(cur);
             }
             tma_store_wait_all();
         }
@@ -616,6 +674,39 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int dr_h = a.is4d ? (row / a.tw) % a.th : 0;
         const int dr_b = a.is4d ? row / (a.tw * a.th) : 0;
         int staged_n_tile = -1;
+        if (a.w4 != nullptr && a.bres > 0 && blockIdx.x < a.num_tiles) {
+            // 4-bit weights: the layer's codes stay packed in global memory (two per byte along K); all sixteen
+            // epilogue warps expand this CTA's column tile to int8 once, straight into the swizzled K blocks the
+            // tensor cores read.  A thread takes 16 packed bytes = 32 codes = two 16-byte chunks of one row.
+            int n_tile0;
+            uint32_t m_tile0;
+            decode_tile(a, blockIdx.x, m_tile0, n_tile0);       // (a CTA with several tiles has a single column tile)
+            const int parts = a.BK >> 5;                        // 32-code pieces per row of a K block
+            const int per_blk = a.BN * parts;
+            const uint8_t* const src = a.w4 + static_cast<int64_t>(n_tile0) * a.BN * a.w4_row;
+            for (int q = et; q < a.bres * per_blk; q += 32 * kEpiWarps) {
+                const int blk = q / per_blk, rem = q - blk * per_blk;
+                const int wrow = rem / parts, part = rem - wrow * parts;
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(src + static_cast<int64_t>(wrow) * a.w4_row + blk * (a.BK >> 1) + 16 * part));
+                const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+                uint32_t o[8];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    // byte j of a word holds code 2j (low nibble) and code 2j+1 (high nibble), two's complement
+                    uint32_t even = in[i] & 0x0f0f0f0fu, odd = (in[i] >> 4) & 0x0f0f0f0fu;
+                    even |= (even & 0x08080808u) * 0x1eu;       // sign bit of a nibble -> bits 4..7 of its byte
+                    odd |= (odd & 0x08080808u) * 0x1eu;
+                    o[2 * i] = __byte_perm(even, odd, 0x5140);
+                    o[2 * i + 1] = __byte_perm(even, odd, 0x7362);
+                }
+                uint8_t* const dstb = smem + L.b_off + blk * L.b_blk;
+                *reinterpret_cast<uint4*>(dstb + swz(wrow, 32 * part, a.BK)) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4*>(dstb + swz(wrow, 32 * part + 16, a.BK)) = make_uint4(o[4], o[5], o[6], o[7]);
+            }
+            fence_proxy_async_smem();                           // generic-proxy writes, read next by the tensor cores
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_wres);
+        }
         // A warp whose wait ran out stops working but keeps meeting the group at the table barriers,
         // so that nobody is left alone at one; everything else it would have signalled times out too.
         bool dead = false;
@@ -729,7 +820,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (nn >= a.N) break;                // boxes entirely beyond the real channels
                 uint8_t* const dst = out_s + slot * box_bytes;
                 // the store that last used this box has read it
-                if (!__all_sync(0xffffffffu, mbar_wait(oempty + 8 * slot, slot_phase ^ 1, a.wait_budget, 64u))) {
+                // (with a fused residual add this is also the arrival of the shortcut tile in the box: phase k of the
+                //  barrier ends when the k-th copy into the box has landed, so the parity to wait for is one earlier)
+                if (!__all_sync(0xffffffffu, mbar_wait(oempty + 8 * slot, a.res ? slot_phase : slot_phase ^ 1, a.wait_budget, 64u))) {
                     if (lane == 0) {
                         report_timeout(a.status, QTZ_SITE_OUT_EMPTY);
                         *abort_flag = 1;
@@ -757,8 +850,24 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         requant32<1, false>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
                     else
                         requant32<2, false>(v, mult_s + j0, sh_s + j0, add64_s + j0, corr_row + j0, addhi_s + j0, rowterm, span, off, lo4, packed);
-                    *reinterpret_cast<uint4*>(dst + swz(row, col, a.out_box)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                    *reinterpret_cast<uint4*>(dst + swz(row, col + 16, a.out_box)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                    uint4* const p0 = reinterpret_cast<uint4*>(dst + swz(row, col, a.out_box));
+                    uint4* const p1 = reinterpret_cast<uint4*>(dst + swz(row, col + 16, a.out_box));
+                    if (a.res) {
+                        // packed[] holds the convolution's own codes t; the box holds the shortcut s at the same places
+                        const uint4 s0 = *p0, s1 = *p1;
+                        const uint32_t sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                        const uint32_t lo4r = 0x01010101u * static_cast<uint32_t>(a.res_rule.act_min);
+                        const int32_t spanr = a.res_rule.act_max - a.res_rule.act_min;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            if (a.res_kind == 3) packed[q] = qtz_add::add_split4(packed[q], sv[q], a.res_split, lo4r);
+                            else if (a.res_kind == 0) packed[q] = qtz_add::add4<0>(packed[q], sv[q], a.res_rule, a.res_addend, spanr, lo4r);
+                            else if (a.res_kind == 1) packed[q] = qtz_add::add4<1>(packed[q], sv[q], a.res_rule, a.res_addend, spanr, lo4r);
+                            else packed[q] = qtz_add::add4<2>(packed[q], sv[q], a.res_rule, a.res_addend, spanr, lo4r);
+                        }
+                    }
+                    *p0 = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    *p1 = make_uint4(packed[4], packed[5], packed[6], packed[7]);
                 }
                 const bool drained = bx == boxes - 1 || nn + a.out_box >= a.N;
                 if (drained) tc_fence_before();
@@ -810,6 +919,15 @@ prepack_tc_kernel(const void* __restrict__ w, int wkind, int n, int taps, int c,
                                                 static_cast<int64_t>(taps) * runs * c_src));
     }
     out[i] = v;
+}
+
+// int8 codes in [-8, 7] -> two per byte along the row (even element in the low nibble).
+__global__ void __launch_bounds__(kPrepThreads)
+pack_nibbles_kernel(const int8_t* __restrict__ w, int64_t bytes_out, uint8_t* __restrict__ out)
+{
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
+    if (i >= bytes_out) return;
+    out[i] = static_cast<uint8_t>((static_cast<uint32_t>(w[2 * i]) & 0xfu) | (static_cast<uint32_t>(w[2 * i + 1]) << 4));
 }
 
 // Weight sums per border class.  Class = 4 * rowclass + colclass, each a 2-bit mask
@@ -1049,6 +1167,8 @@ struct qtz_tc_state {
     int cs = 0;                // im2col: bytes per tap in the window matrix (channels rounded up to 4)
     CUtensorMap map_b{};
     int8_t* w_packed = nullptr;
+    uint8_t* w_packed4 = nullptr;   // 4-bit layers: the same re-laid rows with two codes per byte (what the kernel reads when
+                                    // the layer's weights are expanded in shared memory)
     int32_t* xsum = nullptr;
     int64_t in_pixels = 0;     // pixels of the (possibly gathered) input
     int in_h = 0, in_w = 0;    // its spatial extent
@@ -1176,6 +1296,7 @@ void qtz_tc_release(qtz_plan* p)
 {
     if (!p->tc) return;
     cudaFree(p->tc->w_packed);
+    cudaFree(p->tc->w_packed4);
     cudaFree(p->tc->xsum);
     delete p->tc;
     p->tc = nullptr;
@@ -1239,6 +1360,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     // (one tile: 32-column granularity, the TMA store clips what lies beyond the real channels;
     //  several tiles: whole staging boxes, since a box must not spill into the next tile's columns)
     a.BN = a.n_tiles == 1 ? (d.n + 31) / 32 * 32 : ((d.n + a.n_tiles - 1) / a.n_tiles + 63) / 64 * 64;
+    a.n_tiles = (d.n + a.BN - 1) / a.BN;     // rounding the width up may have emptied the last tile
     // (a single column tile wider than 128 also takes 128-byte boxes: the store clips the last one at N, and every
     //  box row is one request to the copy engine whatever its length)
     a.out_box = (a.BN % 128 == 0 || (a.n_tiles == 1 && a.BN > 128)) ? 128 : 64;
@@ -1324,6 +1446,12 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
         prepack_tc_kernel<<<static_cast<unsigned>((wbytes + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
             w_q_dev, d.wkind, d.n, a.taps, d.c, t->n_pad, a.c_pad, t->w_packed, t->im2col ? t->cs : d.c, t->im2col ? p->d.c : d.c);
     QTZ_LAUNCH_CHECK(h, "prepack_tc_kernel");
+    if (d.wkind == QTZ_W_S4_PACKED_PER_CHANNEL_SYM) {
+        QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->w_packed4), static_cast<size_t>(wbytes / 2)));
+        pack_nibbles_kernel<<<static_cast<unsigned>((wbytes / 2 + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
+            t->w_packed, wbytes / 2, t->w_packed4);
+        QTZ_LAUNCH_CHECK(h, "pack_nibbles_kernel");
+    }
     QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->wsum), sizeof(int32_t) * a.ncls * d.n));
     if (rw)   // one class, the whole packed row as a single run
         class_sums_kernel<<<d.n, kPrepThreads, 0, st>>>(t->w_packed, d.n, 1, 1, a.taps * a.c_pad, 1, p->wsum);
@@ -1380,7 +1508,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
 }
 
 qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, int32_t y_zp, int32_t act_min,
-                         int32_t act_max, cudaStream_t st)
+                         int32_t act_max, cudaStream_t st, const qtz_residual* res, const uint8_t* s_dev)
 {
     qtz_ctx* h = p->h;
     qtz_tc_state* t = p->tc;
@@ -1424,7 +1552,8 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
         QTZ_LAUNCH_CHECK(h, "pixel_sum_kernel");
     }
 
-    CUtensorMap map_a, map_y;
+    if (res && a.raw) return QTZ_ERR_UNSUPPORTED;
+    CUtensorMap map_a, map_y, map_s;
     const uint64_t pitch = static_cast<uint64_t>(d.c_pitch_in);
     if (t->rowwin) {
         map_a = t->map_b;   // encoded below, once the number of filter rows per ring stage is known
@@ -1441,6 +1570,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
                                  static_cast<uint32_t>(a.tb)};
         if (!encode_map(&map_a, xin, 4, dims, strides, box, a.BK)) return QTZ_ERR_CUDA;
     }
+    map_s = t->map_b;      // placeholder unless a residual add is fused
     if (a.raw) {
         map_y = t->map_b;  // unused by the kernel in this mode
         a.y_raw = static_cast<int32_t*>(y);
@@ -1451,6 +1581,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
             const uint64_t strides[1] = {opitch};
             const uint32_t box[2] = {static_cast<uint32_t>(a.out_box), static_cast<uint32_t>(kTileM)};
             if (!encode_map(&map_y, y, 2, dims, strides, box, a.out_box)) return QTZ_ERR_CUDA;
+            if (res && !encode_map(&map_s, s_dev, 2, dims, strides, box, a.out_box)) return QTZ_ERR_CUDA;
         } else {
             const uint64_t dims[4] = {static_cast<uint64_t>(d.n), static_cast<uint64_t>(p->ow), static_cast<uint64_t>(p->oh),
                                       static_cast<uint64_t>(d.batch)};
@@ -1458,12 +1589,25 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
             const uint32_t box[4] = {static_cast<uint32_t>(a.out_box), static_cast<uint32_t>(a.tw), static_cast<uint32_t>(a.th),
                                      static_cast<uint32_t>(a.tb)};
             if (!encode_map(&map_y, y, 4, dims, strides, box, a.out_box)) return QTZ_ERR_CUDA;
+            if (res && !encode_map(&map_s, s_dev, 4, dims, strides, box, a.out_box)) return QTZ_ERR_CUDA;
         }
     }
     a.zx = x_zp;
     a.zy = y_zp;
     a.act_min = act_min;
     a.act_max = act_max;
+    a.res = 0;
+    if (res) {
+        // the requantisation of the epilogue produces t with its own quantizer; the add then produces y
+        a.res = 1;
+        a.zy = res->t_zero_point;
+        a.act_min = res->t_act_min;
+        a.act_max = res->t_act_max;
+        a.res_rule = qtz_add::AddRule{res->t_zero_point, res->t_mult, res->s_zero_point, res->s_mult, res->rshift, y_zp, act_min, act_max};
+        a.res_kind = (res->rshift >= 16 && res->rshift <= 38) ? 3 : (res->rshift >= 32 ? 0 : (res->rshift >= 10 ? 1 : 2));
+        a.res_split = qtz_add::make_split(a.res_rule);
+        a.res_addend = qtz_add::add_addend(a.res_rule);
+    }
     // with z_x = 0 the cross-term correction no longer depends on the border class: one class, small tables
     if (x_zp == 0) a.ncls = 1;
     // Shared memory is split between the operand ring, the epilogue groups and their staging boxes.
@@ -1478,7 +1622,13 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     };
     const int kblocks = a.taps * a.kb_per_tap;
     // weights of a single-column-tile layer stay resident when they are small: the ring then carries activations only
-    a.bres = (a.n_tiles == 1 && kblocks * a.BN * a.BK <= kResidentBMax) ? kblocks : 0;
+    // (4-bit layers expand their packed codes in shared memory, which needs them resident: they get a larger share,
+    //  and a layer with several column tiles qualifies when every CTA runs a single tile -- a classifier)
+    const bool one_tile_each = a.num_tiles <= static_cast<uint32_t>(t->grid);
+    if (t->w_packed4)
+        a.bres = ((a.n_tiles == 1 || one_tile_each) && kblocks * a.BN * a.BK <= kResidentB4Max) ? kblocks : 0;
+    else
+        a.bres = (a.n_tiles == 1 && kblocks * a.BN * a.BK <= kResidentBMax) ? kblocks : 0;
     // several K blocks share a ring stage (one barrier handshake for all of them) while the stage stays within 32 KB
     auto blocks_per_stage = [&]() {
         const int blk = (a.a_blk > 0 ? a.a_blk : kTileM * a.BK) + (a.bres > 0 ? 0 : a.BN * a.BK);
@@ -1490,7 +1640,9 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.spb = blocks_per_stage();
     int need = std::min(4, kblocks / a.spb + 1);
     static const int choice[7][2] = {{4, 3}, {4, 2}, {2, 3}, {2, 2}, {1, 2}, {2, 1}, {1, 1}};
-    for (int attempt = 0; attempt < 2; ++attempt) {
+    // attempts: resident weights with several K blocks per stage; resident weights with one K block per stage (a
+    // smaller ring beside a large resident tile); weights through the ring
+    for (int attempt = 0; attempt < 3; ++attempt) {
         a.groups = 1;
         a.obuf = 1;
         bool found = false;
@@ -1505,8 +1657,12 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
             }
         }
         if (found || a.bres == 0) break;
-        a.bres = 0;                                  // no room beside resident weights: send them through the ring
-        a.spb = blocks_per_stage();
+        if (attempt == 0 && a.spb > 1) {
+            a.spb = 1;
+        } else {
+            a.bres = 0;                              // no room beside resident weights: send them through the ring
+            a.spb = blocks_per_stage();
+        }
         need = std::min(4, kblocks / a.spb + 1);
     }
     a.gwarps = a.groups == 4 ? 4 : 8;
@@ -1524,8 +1680,13 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.lsu = (a.stages >= 3 && t->rowwin) ? 1 : 0;
     a.src = xin;
     a.full_count = a.lsu ? (a.bres > 0 ? 1 : 2) : 1;
+    a.w4 = (t->w_packed4 && a.bres > 0) ? t->w_packed4 : nullptr;
+    a.w4_row = (a.taps * a.c_pad) >> 1;
+    p->detail = std::string("tcgen05") + (t->rowwin ? " row-window" : (t->im2col ? " im2col" : (pw ? " pointwise" : " 3x3"))) +
+                (a.bres > 0 ? (a.w4 ? " weights:int4-expanded-in-smem" : " weights:resident") : " weights:streamed") +
+                (a.res ? " +residual-add" : "");
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
-    conv_tc_kernel<<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, a);
+    conv_tc_kernel<<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, map_s, a);
     QTZ_LAUNCH_CHECK(h, "conv_tc_kernel");
     if (p->ev_stop) QTZ_CUDA(h, cudaEventRecord(p->ev_stop, st));
     return QTZ_OK;

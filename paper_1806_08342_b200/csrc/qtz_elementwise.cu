@@ -231,7 +231,7 @@ dequantize_axis_kernel(const void* __restrict__ q, int32_t dtype, int64_t total,
         const int64_t run = i / run_len, e = i - run * run_len;
         const uint32_t byte = static_cast<const uint8_t*>(q)[run * ((run_len + 1) >> 1) + (e >> 1)];
         const uint32_t nib = (e & 1) ? (byte >> 4) : (byte & 0xfu);
-        code = static_cast<int32_t>(nib << 28) >> 28;
+        code = dtype == QTZ_U4_PACKED ? static_cast<int32_t>(nib) : static_cast<int32_t>(nib << 28) >> 28;
     }
     x[i] = __fmul_rn(static_cast<float>(code - r.zp), r.scale);
 }
@@ -487,7 +487,8 @@ extern "C" qtz_status qtz_quantize_tensor(qtz_handle h, const float* x_dev, int6
         rules[a] = QuantRule{p.scale, static_cast<float>(qmin - p.zero_point),
                              static_cast<float>(qmax - p.zero_point), p.zero_point};
     }
-    if (axis_len == 1 && out_dtype != QTZ_S4_PACKED && qtz_aligned16(x_dev) && qtz_aligned16(q_dev)) {
+    const bool packed4 = out_dtype == QTZ_S4_PACKED || out_dtype == QTZ_U4_PACKED;
+    if (axis_len == 1 && !packed4 && qtz_aligned16(x_dev) && qtz_aligned16(q_dev)) {
         const int64_t groups = (total >> 4) + 1;
         quantize_flat_kernel<<<static_cast<unsigned>(ceil_div(groups, kThreads)), kThreads, 0, st>>>(
             x_dev, total, rules[0], static_cast<uint8_t*>(q_dev));
@@ -499,7 +500,7 @@ extern "C" qtz_status qtz_quantize_tensor(qtz_handle h, const float* x_dev, int6
     if (s != QTZ_OK) return s;
     QTZ_CUDA(h, cudaMemcpyAsync(h->params_dev, rules.data(), bytes, cudaMemcpyHostToDevice, st));
     const QuantRule* rules_dev = static_cast<const QuantRule*>(h->params_dev);
-    if (out_dtype == QTZ_S4_PACKED) {
+    if (packed4) {
         const int64_t run_len = inner > 1 ? inner : axis_len;
         const int64_t runs = total / run_len;
         const int64_t work = runs * ((run_len + 1) >> 1);
@@ -523,7 +524,7 @@ extern "C" qtz_status qtz_dequantize(qtz_handle h, const void* q_dev, int32_t in
     if (!h || !params_host) return QTZ_ERR_INVALID_ARG;
     qtz_status s = check_view(q_dev, x_dev, outer, axis_len, inner);
     if (s != QTZ_OK) return s;
-    if (in_dtype < QTZ_U8 || in_dtype > QTZ_S32) return QTZ_ERR_INVALID_ARG;
+    if (in_dtype < QTZ_U8 || in_dtype > QTZ_U4_PACKED) return QTZ_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(x_dev) & 3u) return QTZ_ERR_MISALIGNED;
     if (in_dtype == QTZ_S32 && (reinterpret_cast<uintptr_t>(q_dev) & 3u)) return QTZ_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -3,89 +3,14 @@
 // thread moves 16 bytes per operand.
 #include <algorithm>
 
+#include "qtz_add_math.cuh"
 #include "qtz_internal.cuh"
 
 namespace {
 
 constexpr int kThreads = 256;
 
-struct AddRule {
-    int32_t a_zp, a_mult, b_zp, b_mult, rshift, y_zp, act_min, act_max;
-};
-
-// d = (c << 16) | (sat_u8(a) << 8) | sat_u8(b)
-__device__ __forceinline__ uint32_t pack_sat_u8(int32_t a, int32_t b, uint32_t c)
-{
-    uint32_t d;
-    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-
-// (a m_a + b m_b + addend) >> r for one byte lane, relative to act_min and clamped to
-// [0, act_max - act_min]; the zero points, the rounding constant and (z_y - act_min) 2^r are all
-// inside `addend`.  |a m| < 2^39, so the shifted value fits 32 bits whenever r >= 10; smaller
-// shifts take the 64-bit route.
-template <int kShiftKind>  // 0: r >= 32, 1: 10 <= r < 32, 2: r < 10
-__device__ __forceinline__ int32_t add1(uint32_t a, uint32_t b, const AddRule& r, int64_t addend, int32_t span)
-{
-    const int64_t v = static_cast<int64_t>(static_cast<uint64_t>(a) * static_cast<uint32_t>(r.a_mult)) +
-                      static_cast<int64_t>(static_cast<uint64_t>(b) * static_cast<uint32_t>(r.b_mult)) + addend;
-    if (kShiftKind == 0) return __vimin_s32_relu(static_cast<int32_t>(v >> 32) >> (r.rshift - 32), span);
-    if (kShiftKind == 1)
-        return __vimin_s32_relu(static_cast<int32_t>(__funnelshift_r(static_cast<uint32_t>(v), static_cast<uint32_t>(v >> 32), r.rshift)), span);
-    const int64_t s = v >> r.rshift;
-    return static_cast<int32_t>(min(max(s, static_cast<int64_t>(0)), static_cast<int64_t>(span)));
-}
-
-template <int kShiftKind>
-__device__ __forceinline__ uint32_t add4(uint32_t a, uint32_t b, const AddRule& r, int64_t addend, int32_t span, uint32_t lo4)
-{
-    const int32_t y0 = add1<kShiftKind>(a & 0xff, b & 0xff, r, addend, span);
-    const int32_t y1 = add1<kShiftKind>((a >> 8) & 0xff, (b >> 8) & 0xff, r, addend, span);
-    const int32_t y2 = add1<kShiftKind>((a >> 16) & 0xff, (b >> 16) & 0xff, r, addend, span);
-    const int32_t y3 = add1<kShiftKind>(a >> 24, b >> 24, r, addend, span);
-    return pack_sat_u8(y1, y0, pack_sat_u8(y3, y2, 0u)) + lo4;
-}
-
-// The same for shifts 16 <= r <= 38 without 64-bit multiplies.  With m = mh 2^16 + ml (both halves below 2^16):
-//   a m_a + b m_b + addend = (a mah + b mbh + Ah) 2^16 + (a mal + b mbl + Al),  addend = Ah 2^16 + Al, 0 <= Al < 2^16,
-// every bracket fits 32 bits (a, b < 2^8; |addend| < 2^47), and since floor(floor(x / 2^16) / 2^(r-16)) =
-// floor(x / 2^r) the result is ((hi + Ah + (lo >> 16)) >> (r - 16)) exactly.  Each bracket is one dp2a on the
-// byte pair (a, b) against the 16-bit pair (m_a half, m_b half).
-struct AddSplit {
-    uint32_t mh, ml;     // (mah | mbh << 16), (mal | mbl << 16)
-    int32_t ah;          // addend >> 16 (arithmetic)
-    uint32_t al;         // addend & 0xffff
-    int32_t sh, span;    // r - 16, act_max - act_min
-};
-
-__device__ __forceinline__ uint32_t dp2a_lo(uint32_t m16x2, uint32_t bytes, uint32_t c)
-{
-    uint32_t d;
-    asm("dp2a.lo.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(m16x2), "r"(bytes), "r"(c));
-    return d;
-}
-__device__ __forceinline__ uint32_t dp2a_hi(uint32_t m16x2, uint32_t bytes, uint32_t c)
-{
-    uint32_t d;
-    asm("dp2a.hi.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(m16x2), "r"(bytes), "r"(c));
-    return d;
-}
-
-__device__ __forceinline__ int32_t add_split1(uint32_t hi, uint32_t lo, const AddSplit& q)
-{
-    return __vimin_s32_relu((static_cast<int32_t>(hi) + q.ah + static_cast<int32_t>(lo >> 16)) >> q.sh, q.span);
-}
-
-__device__ __forceinline__ uint32_t add_split4(uint32_t a, uint32_t b, const AddSplit& q, uint32_t lo4)
-{
-    const uint32_t p01 = __byte_perm(a, b, 0x5140), p23 = __byte_perm(a, b, 0x7362);   // (a0,b0,a1,b1), (a2,b2,a3,b3)
-    const int32_t y0 = add_split1(dp2a_lo(q.mh, p01, 0u), dp2a_lo(q.ml, p01, q.al), q);
-    const int32_t y1 = add_split1(dp2a_hi(q.mh, p01, 0u), dp2a_hi(q.ml, p01, q.al), q);
-    const int32_t y2 = add_split1(dp2a_lo(q.mh, p23, 0u), dp2a_lo(q.ml, p23, q.al), q);
-    const int32_t y3 = add_split1(dp2a_hi(q.mh, p23, 0u), dp2a_hi(q.ml, p23, q.al), q);
-    return pack_sat_u8(y1, y0, pack_sat_u8(y3, y2, 0u)) + lo4;
-}
+using namespace qtz_add;
 
 // y = clamp(z_y + (((a - z_a) m_a + (b - z_b) m_b + 2^(r-1)) >> r)).  All constants fold into one
 // 64-bit addend: 2^(r-1) + (z_y - act_min) 2^r - z_a m_a - z_b m_b (|.| < 2^62 for r <= 53).
@@ -94,9 +19,7 @@ __global__ void __launch_bounds__(kThreads)
 add_u8_kernel(const uint8_t* __restrict__ a, const uint8_t* __restrict__ b, int64_t bytes, AddRule r,
               uint8_t* __restrict__ y)
 {
-    const int64_t addend = (static_cast<int64_t>(1) << (r.rshift - 1)) +
-                           static_cast<int64_t>(r.y_zp - r.act_min) * (static_cast<int64_t>(1) << r.rshift) -
-                           static_cast<int64_t>(r.a_zp) * r.a_mult - static_cast<int64_t>(r.b_zp) * r.b_mult;
+    const int64_t addend = add_addend(r);
     const uint32_t lo4 = 0x01010101u * static_cast<uint32_t>(r.act_min);
     const int32_t span = r.act_max - r.act_min;
     const int64_t groups = bytes >> 4;
@@ -106,13 +29,7 @@ add_u8_kernel(const uint8_t* __restrict__ a, const uint8_t* __restrict__ b, int6
     const uint4 vb = __ldcs(reinterpret_cast<const uint4*>(b) + g);
     uint4 o;
     if (kShiftKind == 3) {
-        AddSplit q;
-        q.mh = (static_cast<uint32_t>(r.a_mult) >> 16) | (static_cast<uint32_t>(r.b_mult) & 0xffff0000u);
-        q.ml = (static_cast<uint32_t>(r.a_mult) & 0xffffu) | (static_cast<uint32_t>(r.b_mult) << 16);
-        q.ah = static_cast<int32_t>(addend >> 16);
-        q.al = static_cast<uint32_t>(addend) & 0xffffu;
-        q.sh = r.rshift - 16;
-        q.span = span;
+        const AddSplit q = make_split(r);
         o.x = add_split4(va.x, vb.x, q, lo4); o.y = add_split4(va.y, vb.y, q, lo4);
         o.z = add_split4(va.z, vb.z, q, lo4); o.w = add_split4(va.w, vb.w, q, lo4);
         reinterpret_cast<uint4*>(y)[g] = o;
@@ -236,5 +153,105 @@ extern "C" qtz_status qtz_global_avgpool_u8(qtz_handle h, const uint8_t* x_dev, 
     global_avgpool_u8_kernel<<<static_cast<unsigned>(ceil_div(total, kThreads)), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         x_dev, x_zp, y_dev, y_zp, mult, rshift, batch, hw, c_pitch);
     QTZ_LAUNCH_CHECK(h, "global_avgpool_u8_kernel");
+    return QTZ_OK;
+}
+
+// ---- 4-bit activation storage (Section 3.2.4) ---------------------------------------------------
+namespace {
+
+constexpr int kPackThreads = 256;
+
+// One thread per packed byte (generic) or per four packed bytes (rows 4-byte aligned on both sides).
+__global__ void __launch_bounds__(kPackThreads)
+pack_u4_kernel(const uint8_t* __restrict__ x, int64_t pixels, int c, int x_pitch, uint8_t* __restrict__ y, int y_pitch, int fast)
+{
+    const int bytes = (c + 1) >> 1;
+    const int per_row = fast ? (bytes + 3) >> 2 : bytes;
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * kPackThreads + threadIdx.x;
+    if (t >= pixels * per_row) return;
+    const int64_t p = t / per_row;
+    const int j = static_cast<int>(t - p * per_row);
+    const uint8_t* row = x + p * x_pitch;
+    uint8_t* out = y + p * y_pitch;
+    if (fast && 8 * j + 8 <= c) {          // eight codes in, four bytes out
+        const uint2 v = *reinterpret_cast<const uint2*>(row + 8 * j);
+        const uint32_t lo = v.x & 0x0f0f0f0fu, hi = v.y & 0x0f0f0f0fu;
+        // bytes (a0 a1 a2 a3) -> (a0 | a1 << 4), (a2 | a3 << 4)
+        const uint32_t l2 = (lo | (lo >> 4)) & 0x00ff00ffu, h2 = (hi | (hi >> 4)) & 0x00ff00ffu;
+        const uint32_t l = (l2 | (l2 >> 8)) & 0xffffu, hh = (h2 | (h2 >> 8)) & 0xffffu;
+        *reinterpret_cast<uint32_t*>(out + 4 * j) = l | (hh << 16);
+        return;
+    }
+    const int first = fast ? 4 * j : j, last = fast ? min(4 * j + 4, bytes) : j + 1;
+    for (int b = first; b < last; ++b) {
+        const uint32_t lo = row[2 * b] & 0xfu, hi = 2 * b + 1 < c ? (row[2 * b + 1] & 0xfu) : 0u;
+        out[b] = static_cast<uint8_t>(lo | (hi << 4));
+    }
+}
+
+__global__ void __launch_bounds__(kPackThreads)
+unpack_u4_kernel(const uint8_t* __restrict__ x, int64_t pixels, int c, int x_pitch, uint8_t* __restrict__ y, int y_pitch, int fast)
+{
+    const int bytes = (c + 1) >> 1;
+    const int per_row = fast ? (bytes + 3) >> 2 : bytes;
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * kPackThreads + threadIdx.x;
+    if (t >= pixels * per_row) return;
+    const int64_t p = t / per_row;
+    const int j = static_cast<int>(t - p * per_row);
+    const uint8_t* row = x + p * x_pitch;
+    uint8_t* out = y + p * y_pitch;
+    if (fast && 8 * j + 8 <= c) {          // four bytes in, eight codes out
+        const uint32_t v = *reinterpret_cast<const uint32_t*>(row + 4 * j);
+        const uint32_t even = v & 0x0f0f0f0fu, odd = (v >> 4) & 0x0f0f0f0fu;       // codes 0,2,4,6 and 1,3,5,7
+        uint2 o;
+        o.x = __byte_perm(even, odd, 0x5140);                                       // c0 c1 c2 c3
+        o.y = __byte_perm(even, odd, 0x7362);                                       // c4 c5 c6 c7
+        *reinterpret_cast<uint2*>(out + 8 * j) = o;
+        return;
+    }
+    const int first = fast ? 4 * j : j, last = fast ? min(4 * j + 4, bytes) : j + 1;
+    for (int b = first; b < last; ++b) {
+        const uint32_t v = row[b];
+        out[2 * b] = static_cast<uint8_t>(v & 0xfu);
+        if (2 * b + 1 < c) out[2 * b + 1] = static_cast<uint8_t>(v >> 4);
+    }
+}
+
+qtz_status pack_args_ok(qtz_handle h, const void* x, const void* y, int64_t pixels, int32_t c, int32_t wide_pitch, int32_t packed_pitch)
+{
+    if (!h || !x || !y || pixels <= 0 || c <= 0 || wide_pitch < c || packed_pitch < (c + 1) / 2) return QTZ_ERR_INVALID_ARG;
+    if (pixels > (INT64_MAX / 4) / (c + 8)) return QTZ_ERR_INVALID_ARG;
+    return QTZ_OK;
+}
+
+}  // namespace
+
+extern "C" qtz_status qtz_pack_u4(qtz_handle h, const uint8_t* x_dev, int64_t pixels, int32_t c, int32_t x_pitch,
+                                  uint8_t* y_dev, int32_t y_pitch, void* stream)
+{
+    qtz_status s = pack_args_ok(h, x_dev, y_dev, pixels, c, x_pitch, y_pitch);
+    if (s != QTZ_OK) return s;
+    const int fast = ((reinterpret_cast<uintptr_t>(x_dev) & 7u) == 0 && (x_pitch & 7) == 0 &&
+                      (reinterpret_cast<uintptr_t>(y_dev) & 3u) == 0 && (y_pitch & 3) == 0) ? 1 : 0;
+    const int bytes = (c + 1) >> 1;
+    const int64_t work = pixels * (fast ? (bytes + 3) >> 2 : bytes);
+    pack_u4_kernel<<<static_cast<unsigned>((work + kPackThreads - 1) / kPackThreads), kPackThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        x_dev, pixels, c, x_pitch, y_dev, y_pitch, fast);
+    QTZ_LAUNCH_CHECK(h, "pack_u4_kernel");
+    return QTZ_OK;
+}
+
+extern "C" qtz_status qtz_unpack_u4(qtz_handle h, const uint8_t* x_dev, int64_t pixels, int32_t c, int32_t x_pitch,
+                                    uint8_t* y_dev, int32_t y_pitch, void* stream)
+{
+    qtz_status s = pack_args_ok(h, x_dev, y_dev, pixels, c, y_pitch, x_pitch);
+    if (s != QTZ_OK) return s;
+    const int fast = ((reinterpret_cast<uintptr_t>(x_dev) & 3u) == 0 && (x_pitch & 3) == 0 &&
+                      (reinterpret_cast<uintptr_t>(y_dev) & 7u) == 0 && (y_pitch & 7) == 0) ? 1 : 0;
+    const int bytes = (c + 1) >> 1;
+    const int64_t work = pixels * (fast ? (bytes + 3) >> 2 : bytes);
+    unpack_u4_kernel<<<static_cast<unsigned>((work + kPackThreads - 1) / kPackThreads), kPackThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        x_dev, pixels, c, x_pitch, y_dev, y_pitch, fast);
+    QTZ_LAUNCH_CHECK(h, "unpack_u4_kernel");
     return QTZ_OK;
 }

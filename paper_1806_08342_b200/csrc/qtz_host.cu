@@ -169,6 +169,7 @@ bool qtz_code_range(int32_t dtype, int32_t restrict_range, int32_t* qmin, int32_
         case QTZ_U8: *qmin = 0; *qmax = restrict_range ? 254 : 255; return true;
         case QTZ_S8: *qmin = restrict_range ? -127 : -128; *qmax = 127; return true;
         case QTZ_S4_PACKED: *qmin = restrict_range ? -7 : -8; *qmax = 7; return true;
+        case QTZ_U4_PACKED: *qmin = 0; *qmax = restrict_range ? 14 : 15; return true;
         default: return false;
     }
 }
@@ -197,22 +198,29 @@ extern "C" qtz_status qtz_quantize_multiplier(double real_multiplier, int32_t* m
     return QTZ_OK;
 }
 
-extern "C" qtz_status qtz_activation_range(int32_t kind, float y_scale, int32_t y_zero_point,
-                                           int32_t* act_min, int32_t* act_max)
+extern "C" qtz_status qtz_activation_range_bits(int32_t kind, float y_scale, int32_t y_zero_point, int32_t bits,
+                                                int32_t* act_min, int32_t* act_max)
 {
-    if (!act_min || !act_max) return QTZ_ERR_INVALID_ARG;
+    if (!act_min || !act_max || bits < 2 || bits > 8) return QTZ_ERR_INVALID_ARG;
+    const int32_t top_code = (1 << bits) - 1;
     switch (kind) {
-        case 0: *act_min = 0; *act_max = 255; return QTZ_OK;
-        case 1: *act_min = y_zero_point; *act_max = 255; return QTZ_OK;
+        case 0: *act_min = 0; *act_max = top_code; return QTZ_OK;
+        case 1: *act_min = y_zero_point; *act_max = top_code; return QTZ_OK;
         case 2: {
             if (!(y_scale > 0.f)) return QTZ_ERR_INVALID_ARG;
             const double top = y_zero_point + std::nearbyint(6.0 / static_cast<double>(y_scale));
             *act_min = y_zero_point;
-            *act_max = top < 255.0 ? static_cast<int32_t>(top) : 255;
+            *act_max = top < static_cast<double>(top_code) ? static_cast<int32_t>(top) : top_code;
             return QTZ_OK;
         }
         default: return QTZ_ERR_INVALID_ARG;
     }
+}
+
+extern "C" qtz_status qtz_activation_range(int32_t kind, float y_scale, int32_t y_zero_point,
+                                           int32_t* act_min, int32_t* act_max)
+{
+    return qtz_activation_range_bits(kind, y_scale, y_zero_point, 8, act_min, act_max);
 }
 
 extern "C" qtz_status qtz_add_params(float a_scale, float b_scale, float y_scale, int32_t* a_mult,

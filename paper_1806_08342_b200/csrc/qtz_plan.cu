@@ -130,6 +130,13 @@ extern "C" const char* qtz_conv_plan_kernel(qtz_conv_plan p)
     return p->family == QTZ_K_TCGEN05 ? "tcgen05" : (p->family == QTZ_K_DEPTHWISE ? "depthwise" : "direct");
 }
 
+extern "C" const char* qtz_conv_plan_detail(qtz_conv_plan p)
+{
+    if (!p) return "";
+    if (p->detail.empty()) return qtz_conv_plan_kernel(p);
+    return p->detail.c_str();
+}
+
 extern "C" qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, int32_t depthwise, const void* w_q_dev,
                                       const int32_t* bias_q_dev, const int32_t* w_zero_point_host,
                                       const int32_t* mult_host, const int32_t* rshift_host, qtz_conv_plan* out,
@@ -267,6 +274,23 @@ extern "C" qtz_status qtz_conv2d_u8(qtz_conv_plan p, const uint8_t* x_dev, int32
     if (p->family == QTZ_K_TCGEN05)
         return qtz_tc_launch(p, x_dev, x_zero_point, y_dev, y_zero_point, act_min, act_max, st);
     return qtz_direct_launch(p, x_dev, x_zero_point, y_dev, y_zero_point, act_min, act_max, st);
+}
+
+extern "C" qtz_status qtz_conv2d_add_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point, const qtz_residual* r,
+                                        const uint8_t* s_dev, void* y_dev, int32_t y_zero_point, int32_t act_min,
+                                        int32_t act_max, void* stream)
+{
+    qtz_status s = check_run_args(p, x_dev, y_dev, x_zero_point, y_zero_point, act_min, act_max);
+    if (s != QTZ_OK) return s;
+    if (!r || !s_dev || p->depthwise) return QTZ_ERR_INVALID_ARG;
+    if (!qtz_aligned16(s_dev)) return QTZ_ERR_MISALIGNED;
+    if (r->t_zero_point < 0 || r->t_zero_point > 255 || r->s_zero_point < 0 || r->s_zero_point > 255 || r->t_act_min < 0 ||
+        r->t_act_max > 255 || r->t_act_min > r->t_act_max || r->t_mult < 0 || r->s_mult < 0)
+        return QTZ_ERR_INVALID_ARG;
+    if (r->rshift < 1 || r->rshift > 53) return QTZ_ERR_UNSUPPORTED;
+    if (p->family != QTZ_K_TCGEN05 || p->d.outkind != QTZ_OUT_U8) return QTZ_ERR_UNSUPPORTED;
+    qtz_device_guard guard(p->device);
+    return qtz_tc_launch(p, x_dev, x_zero_point, y_dev, y_zero_point, act_min, act_max, static_cast<cudaStream_t>(stream), r, s_dev);
 }
 
 extern "C" qtz_status qtz_depthwise_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point, void* y_dev,

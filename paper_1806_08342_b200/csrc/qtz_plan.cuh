@@ -36,6 +36,7 @@ struct qtz_plan {
     qtz_tc_state* tc = nullptr;
     qtz_dw_state* dw = nullptr;
     cudaEvent_t ev_start = nullptr, ev_stop = nullptr;  // optional profiling hook
+    std::string detail;                                 // how the most recent launch ran (qtz_conv_plan_detail)
 };
 
 // Direct (CUDA-core) path.
@@ -50,8 +51,10 @@ qtz_status qtz_depthwise_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, uin
 bool qtz_tc_supported(const qtz_conv_desc& d);
 qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st);
 void qtz_tc_release(qtz_plan* p);
+// res / s_dev: NULL, or the residual add fused into the epilogue and its second addend (qtz_conv2d_add_u8).
 qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, int32_t y_zp,
-                         int32_t act_min, int32_t act_max, cudaStream_t st);
+                         int32_t act_min, int32_t act_max, cudaStream_t st, const qtz_residual* res = nullptr,
+                         const uint8_t* s_dev = nullptr);
 
 // Encodes a rank-2 or rank-4 uint8 tensor map (dims[0] contiguous).  swizzle_bytes: 0 (none), 32, 64 or 128.
 bool qtz_encode_u8_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,

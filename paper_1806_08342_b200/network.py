@@ -25,8 +25,11 @@ class _Layer:
 
 
 class QuantizedNetwork:
-    def __init__(self, handle: qtz.Handle, ops, seed: int, wbits: int = 8):
+    def __init__(self, handle: qtz.Handle, ops, seed: int, wbits: int = 8, fuse: bool = True):
         self.h, self.ops, self.seed, self.wbits = handle, ops, seed, wbits
+        self.fuse = fuse            # forward() runs a convolution and the residual add that follows it as one kernel
+        self.fused_away = set()     # tensors forward() then never writes (build() still computes them once)
+        self.schedule = []          # what forward() launches: (kind, layer[, add layer])
         self.layers = []
         self.params = {}            # tensor name -> qparams record (numpy void) after build()
         self.batch = None
@@ -135,7 +138,44 @@ class QuantizedNetwork:
             self.layers.append(L)
         self.tensors = tensors
         self.chans = chans
+        self._plan_schedule()
         return tensors
+
+    def _plan_schedule(self):
+        """Pairs every element-wise add with the convolution that produces one of its inputs, when that tensor has no
+        other reader and the convolution runs on the tensor-core path: the pair becomes one qtz_conv2d_add_u8 call
+        at the add's position (Section 3.2.1: the add fuses into the producing op)."""
+        readers = {}
+        for L in self.layers:
+            for key in ("src", "a", "b"):
+                if key in L.op:
+                    readers[L.op[key]] = readers.get(L.op[key], 0) + 1
+        producer = {L.op["dst"]: L for L in self.layers}
+        taken, fused = set(), {}
+        if self.fuse:
+            for L in self.layers:
+                if L.op["op"] != "add":
+                    continue
+                for mine, other in (("a", "b"), ("b", "a")):
+                    P = producer.get(L.op[mine])
+                    if (P is not None and P.op["op"] == "conv" and not P.op["depthwise"] and P.plan.kernel == "tcgen05"
+                            and readers.get(L.op[mine], 0) == 1 and id(P) not in taken):
+                        taken.add(id(P))
+                        fused[id(L)] = (P, mine, other)
+                        break
+        self.fused_away = {P.op["dst"] for P, _, _ in fused.values()}
+        self.schedule = []
+        for L in self.layers:
+            if id(L) in taken:
+                continue
+            if id(L) in fused:
+                P, mine, other = fused[id(L)]
+                a = L.args      # (za, ma, zb, mb, r, zy, amin, amax, c)
+                t_zp, t_mult, s_zp, s_mult = (a[0], a[1], a[2], a[3]) if mine == "a" else (a[2], a[3], a[0], a[1])
+                res = qtz.Residual(t_zp, P.args[2], P.args[3], t_mult, s_zp, s_mult, a[4])
+                self.schedule.append(("conv+add", P, L, res, other))
+            else:
+                self.schedule.append((L.op["op"], L))
 
     # ---- the timed pass ----------------------------------------------------------------------
     def forward(self, x=None):
@@ -144,21 +184,28 @@ class QuantizedNetwork:
         h, t = self.h, self.tensors
         if x is not None:
             t["in"] = x
-        for L in self.layers:
-            op = L.op
-            kind = op["op"]
-            if kind == "conv":
-                L.plan(t[op["src"]], *L.args, out=t[op["dst"]])
-            elif kind == "fc":
-                L.plan(t[op["src"]], *L.args, out=t[op["dst"]])
-            elif kind == "add":
-                a = L.args
-                h.add_u8(t[op["a"]], a[0], a[1], t[op["b"]], a[2], a[3], a[4], a[5], a[6], a[7], a[8], out=t[op["dst"]])
-            elif kind == "maxpool":
-                h.maxpool_u8(t[op["src"]], *L.args, out=t[op["dst"]])
-            else:
-                h.global_avgpool_u8(t[op["src"]], *L.args, out=t[op["dst"]])
+        for item in self.schedule:
+            self.run_item(item)
         return t["logits"]
 
+    def run_item(self, item):
+        """One entry of the schedule: a library call on the tensors build() allocated."""
+        h, t = self.h, self.tensors
+        kind, L = item[0], item[1]
+        op = L.op
+        if kind == "conv+add":
+            _, P, A, res, other = item
+            a = A.args
+            P.plan.add_fused(t[P.op["src"]], P.args[0], res, t[A.op[other]], a[5], a[6], a[7], out=t[A.op["dst"]])
+        elif kind in ("conv", "fc"):
+            L.plan(t[op["src"]], *L.args, out=t[op["dst"]])
+        elif kind == "add":
+            a = L.args
+            h.add_u8(t[op["a"]], a[0], a[1], t[op["b"]], a[2], a[3], a[4], a[5], a[6], a[7], a[8], out=t[op["dst"]])
+        elif kind == "maxpool":
+            h.maxpool_u8(t[op["src"]], *L.args, out=t[op["dst"]])
+        else:
+            h.global_avgpool_u8(t[op["src"]], *L.args, out=t[op["dst"]])
+
     def num_launch_calls(self):
-        return len(self.layers)
+        return len(self.schedule)

@@ -17,7 +17,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libqtz.so")
 
-U8, S8, S4_PACKED, S32 = 0, 1, 2, 3
+U8, S8, S4_PACKED, S32, U4_PACKED = 0, 1, 2, 3, 4
 W_S8_PER_CHANNEL_SYM, W_U8_PER_LAYER_ASYM, W_S4_PACKED_PER_CHANNEL_SYM = 0, 1, 2
 OUT_U8, OUT_S32_RAW = 0, 1
 ACT_NONE, ACT_RELU, ACT_RELU6 = 0, 1, 2
@@ -28,6 +28,10 @@ QPARAMS = np.dtype([("scale", "<f4"), ("zero_point", "<i4"), ("min_nudged", "<f4
 class ConvDesc(Structure):
     _fields_ = [(n, c_int32) for n in ("batch", "h", "w", "c", "c_pitch_in", "n", "c_pitch_out", "kh", "kw",
                                        "stride", "pad", "wkind", "outkind")]
+
+
+class Residual(Structure):
+    _fields_ = [(n, c_int32) for n in ("t_zero_point", "t_act_min", "t_act_max", "t_mult", "s_zero_point", "s_mult", "rshift")]
 
 
 class QtzError(RuntimeError):
@@ -67,6 +71,9 @@ SIGNATURES = {
     "qtz_quantize_bias": (c_int32, [c_void_p, c_void_p, c_int64, c_float, c_void_p, c_int32, c_void_p, c_void_p]),
     "qtz_quantize_multiplier": (c_int32, [c_double, POINTER(c_int32), POINTER(c_int32)]),
     "qtz_activation_range": (c_int32, [c_int32, c_float, c_int32, POINTER(c_int32), POINTER(c_int32)]),
+    "qtz_activation_range_bits": (c_int32, [c_int32, c_float, c_int32, c_int32, POINTER(c_int32), POINTER(c_int32)]),
+    "qtz_pack_u4": (c_int32, [c_void_p, c_void_p, c_int64, c_int32, c_int32, c_void_p, c_int32, c_void_p]),
+    "qtz_unpack_u4": (c_int32, [c_void_p, c_void_p, c_int64, c_int32, c_int32, c_void_p, c_int32, c_void_p]),
     "qtz_add_params": (c_int32, [c_float, c_float, c_float, POINTER(c_int32), POINTER(c_int32), POINTER(c_int32)]),
     "qtz_range_after_activation": (c_int32, [c_float, c_float, c_int32, POINTER(c_float), POINTER(c_float)]),
     "qtz_add_output_range": (c_int32, [c_void_p, c_void_p, c_int32, POINTER(c_float), POINTER(c_float)]),
@@ -77,8 +84,11 @@ SIGNATURES = {
                                   c_void_p, POINTER(c_void_p), c_void_p]),
     "qtz_conv_destroy": (c_int32, [c_void_p]),
     "qtz_conv_plan_kernel": (c_char_p, [c_void_p]),
+    "qtz_conv_plan_detail": (c_char_p, [c_void_p]),
     "qtz_conv_set_profile_events": (c_int32, [c_void_p, c_void_p, c_void_p]),
     "qtz_conv2d_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p]),
+    "qtz_conv2d_add_u8": (c_int32, [c_void_p, c_void_p, c_int32, POINTER(Residual), c_void_p, c_void_p, c_int32, c_int32, c_int32,
+                                    c_void_p]),
     "qtz_depthwise_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p]),
     "qtz_add_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p,
                              c_int32, c_int32, c_int32, c_int64, c_int32, c_int32, c_void_p]),
@@ -147,6 +157,14 @@ def activation_range(kind, y_scale, y_zero_point):
     rc = load_library().qtz_activation_range(kind, float(y_scale), int(y_zero_point), byref(lo), byref(hi))
     if rc:
         raise QtzError(rc, "qtz_activation_range")
+    return lo.value, hi.value
+
+
+def activation_range_bits(kind, y_scale, y_zero_point, bits):
+    lo, hi = c_int32(), c_int32()
+    rc = load_library().qtz_activation_range_bits(kind, float(y_scale), int(y_zero_point), int(bits), byref(lo), byref(hi))
+    if rc:
+        raise QtzError(rc, "qtz_activation_range_bits")
     return lo.value, hi.value
 
 
@@ -335,7 +353,7 @@ class Handle:
         o, a, i = _view(x.shape, axis)
         assert params.shape[0] == a
         if out is None:
-            if out_dtype == S4_PACKED:
+            if out_dtype in (S4_PACKED, U4_PACKED):
                 run = i if i > 1 else a
                 out = torch.empty((x.numel() // run) * ((run + 1) // 2), dtype=torch.uint8, device=x.device)
             else:
@@ -347,7 +365,7 @@ class Handle:
     def dequantize(self, q, params, axis=None, in_dtype=None, shape=None, out=None):
         _check_dev(q, out)
         if in_dtype is None:
-            in_dtype = {torch.uint8: U8, torch.int8: S8, torch.int32: S32}[q.dtype]
+            in_dtype = {torch.uint8: U8, torch.int8: S8, torch.int32: S32}[q.dtype]   # packed 4-bit: pass in_dtype
         shape = tuple(q.shape) if shape is None else tuple(shape)
         params = np.ascontiguousarray(np.atleast_1d(params), dtype=QPARAMS)
         o, a, i = _view(shape, axis)
@@ -392,6 +410,26 @@ class Handle:
         dst = c_void_p(out.data_ptr() + out_offset)
         self._chk(self.lib.qtz_rescale_u8(self.h, _ptr(x), x_zp, mult, rshift, dst, y_zp, act_min, act_max,
                                           x.numel() // xp, c, xp, yp, _stream()), "qtz_rescale_u8")
+        return out
+
+    def pack_u4(self, x, c=None, out=None):
+        """One 4-bit code per byte [..., pitch] -> two per byte [..., (c + 1) // 2 rounded up to 16]."""
+        _check_dev(x, out)
+        xp = x.shape[-1]
+        c = xp if c is None else c
+        if out is None:
+            out = torch.zeros(x.shape[:-1] + (((c + 1) // 2 + 15) // 16 * 16,), dtype=torch.uint8, device=x.device)
+        self._chk(self.lib.qtz_pack_u4(self.h, _ptr(x), x.numel() // xp, c, xp, _ptr(out), out.shape[-1], _stream()),
+                  "qtz_pack_u4")
+        return out
+
+    def unpack_u4(self, x, c, out=None):
+        _check_dev(x, out)
+        xp = x.shape[-1]
+        if out is None:
+            out = torch.zeros(x.shape[:-1] + ((c + 15) // 16 * 16,), dtype=torch.uint8, device=x.device)
+        self._chk(self.lib.qtz_unpack_u4(self.h, _ptr(x), x.numel() // xp, c, xp, _ptr(out), out.shape[-1], _stream()),
+                  "qtz_unpack_u4")
         return out
 
     def fold_batchnorm(self, w, conv_bias, gamma, beta, mean, var, eps):
@@ -465,6 +503,10 @@ class ConvPlan:
     def kernel(self) -> str:
         return self.handle.lib.qtz_conv_plan_kernel(self.plan).decode()
 
+    @property
+    def detail(self) -> str:
+        return self.handle.lib.qtz_conv_plan_detail(self.plan).decode()
+
     def empty_output(self, device):
         d = self.desc
         if d.outkind == OUT_S32_RAW:
@@ -477,6 +519,15 @@ class ConvPlan:
         fn = self.handle.lib.qtz_depthwise_u8 if self.depthwise else self.handle.lib.qtz_conv2d_u8
         self.handle._chk(fn(self.plan, _ptr(x), int(x_zero_point), _ptr(out), int(y_zero_point), int(act_min),
                             int(act_max), _stream()), "qtz_depthwise_u8" if self.depthwise else "qtz_conv2d_u8")
+        return out
+
+    def add_fused(self, x, x_zero_point, residual: Residual, s, y_zero_point, act_min, act_max, out=None):
+        """qtz_conv2d_add_u8: this convolution and the element-wise add with `s` in one kernel."""
+        _check_dev(x, s, out)
+        out = self.empty_output(x.device) if out is None else out
+        self.handle._chk(self.handle.lib.qtz_conv2d_add_u8(self.plan, _ptr(x), int(x_zero_point), byref(residual), _ptr(s),
+                                                           _ptr(out), int(y_zero_point), int(act_min), int(act_max), _stream()),
+                         "qtz_conv2d_add_u8")
         return out
 
     def set_profile_events(self, start=None, stop=None):

@@ -27,7 +27,8 @@ def make_weights(wkind, shape, seed):
     return None, codes, None                                        # packed by the caller (layout differs)
 
 
-def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=0, expect_kernel=None, real_m=None, bias_range=20000):
+def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=0, expect_kernel=None, real_m=None, bias_range=20000,
+              expect_detail=None):
     x = synth.uniform_u8((b, h, w, c), seed, 1)
     xp = pitched(x)
     api_w, codes, zw = make_weights(wkind, (n, k, k, c), seed)
@@ -44,6 +45,8 @@ def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=0, 
         got = host(plan(dev(xp), z_x))
         if expect_kernel:
             assert plan.kernel == expect_kernel
+        if expect_detail:
+            assert expect_detail in plan.detail, plan.detail
         assert got.shape == acc.shape
         assert np.array_equal(got, acc)
         return
@@ -61,10 +64,38 @@ def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=0, 
     if expect_kernel:
         assert plan.kernel == expect_kernel
     got = host(plan(dev(xp), z_x, z_y, lo, hi))
+    if expect_detail:
+        assert expect_detail in plan.detail, plan.detail
     assert got.shape[:3] == want.shape[:3]
     bad = np.argwhere(got[..., :n].astype(np.int32) != want)
     assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[0]}: got {got[tuple(bad[0])]} want {want[tuple(bad[0])]}"
     assert want.size < 2000 or len(np.unique(want)) > 20             # the case is not degenerate
+
+
+# 4-bit weights stay packed in global memory and are expanded to int8 in shared memory (Section 7: compressed
+# weight storage decompressed on the fly) whenever a CTA's column tile of the layer fits on chip
+INT4_SMEM_SHAPES = [
+    # b, h, w, c, n, k, stride, pad, raw
+    (2, 28, 28, 96, 24, 1, 1, 0, False),      # pointwise, 64-byte... K block of 128 with a ragged tail
+    (3, 20, 20, 32, 64, 3, 1, 1, False),      # 3x3 with border classes
+    (1, 40, 40, 40, 200, 1, 1, 0, False),     # K block of 64, wide output
+    (2, 30, 30, 16, 8, 1, 1, 0, False),       # K block of 32
+    (256, 1, 1, 1792, 1000, 1, 1, 0, True),   # a classifier: several column tiles, one tile per CTA, raw logits
+    (2, 64, 64, 3, 48, 3, 2, 1, False),       # an image stem (row-window form)
+    (1, 12, 12, 144, 24, 1, 2, 0, False),     # strided pointwise
+]
+
+
+@pytest.mark.parametrize("shape", INT4_SMEM_SHAPES)
+def test_int4_weights_expanded_in_shared_memory(hq, shape):
+    b, h, w, c, n, k, stride, pad, raw = shape
+    conv_case(hq, b, h, w, c, n, k, stride, pad, qtz.W_S4_PACKED_PER_CHANNEL_SYM, 900 + c + n, raw=raw,
+              expect_kernel="tcgen05", expect_detail="int4-expanded-in-smem")
+
+
+def test_int4_weights_too_large_for_shared_memory_are_streamed(hq):
+    conv_case(hq, 4, 28, 28, 448, 1792, 1, 1, 0, qtz.W_S4_PACKED_PER_CHANNEL_SYM, 950, expect_kernel="tcgen05",
+              expect_detail="weights:streamed")
 
 
 STEM_SHAPES = [
@@ -319,3 +350,84 @@ def test_conv_argument_errors(hq):
     assert lib.qtz_conv2d_u8(plan.plan, x.data_ptr(), 0, y.data_ptr(), 0, 10, 5, None) == -1
     assert lib.qtz_conv2d_u8(plan.plan, x.data_ptr() + 4, 0, y.data_ptr(), 0, 0, 255, None) == -2
     assert lib.qtz_depthwise_u8(plan.plan, x.data_ptr(), 0, y.data_ptr(), 0, 0, 255, None) == -1
+
+
+# ---- convolution with the residual add fused into its epilogue (Section 3.2.1, Section 7) ---------------------
+FUSED_ADD_SHAPES = [
+    # b, h, w, c, n, k, weight kind, add scales (t, s, y)
+    (3, 20, 20, 64, 256, 1, qtz.W_S8_PER_CHANNEL_SYM, (0.02, 0.03, 0.04)),          # ResNet projection back to 4x width
+    (2, 14, 14, 32, 64, 3, qtz.W_S8_PER_CHANNEL_SYM, (0.05, 0.01, 0.05)),           # 3x3 tiles (4-D boxes, border classes)
+    (2, 28, 28, 144, 24, 1, qtz.W_S4_PACKED_PER_CHANNEL_SYM, (0.03, 0.03, 0.045)),   # MobileNet-v2 linear bottleneck, ragged box
+    (1, 9, 9, 256, 1000, 1, qtz.W_S8_PER_CHANNEL_SYM, (0.02, 0.02, 0.03)),          # several column tiles
+    (2, 12, 12, 48, 136, 1, qtz.W_U8_PER_LAYER_ASYM, (1e-3, 2e-3, 900.0)),          # add shift above 38: 64-bit form
+    (2, 12, 12, 48, 40, 1, qtz.W_S8_PER_CHANNEL_SYM, (40.0, 25.0, 0.0005)),         # add shift 10..15: funnel-shift form
+    (1, 10, 10, 32, 32, 1, qtz.W_S8_PER_CHANNEL_SYM, (4000.0, 100.0, 0.0005)),      # add shift below 10: 64-bit shift
+]
+
+
+@pytest.mark.parametrize("shape", FUSED_ADD_SHAPES)
+@pytest.mark.parametrize("alias", [False, True])
+def test_conv_with_fused_residual_add(hq, shape, alias):
+    b, h, w, c, n, k, wkind, (st, ss, sy) = shape
+    pad = k // 2
+    seed = 1200 + n
+    x = pitched(synth.uniform_u8((b, h, w, c), seed, 1))
+    api_w, codes, zw = make_weights(wkind, (n, k, k, c), seed)
+    if wkind == qtz.W_S4_PACKED_PER_CHANNEL_SYM:
+        api_w = oracle.pack_s4(codes.reshape(n, -1))
+    g = synth.rng(seed, 71)
+    bias = g.integers(-20000, 20000, size=n).astype(np.int32)
+    z_x, z_t, z_s, z_y = (int(v) for v in g.integers(60, 190, size=4))
+    z_w = None if zw is None else np.full(n, zw, np.int32)
+    acc = oracle.conv2d_acc(x, z_x, codes, z_w, bias, 1, pad, c=c)
+    span = np.abs(acc).reshape(-1, n).max(axis=0).astype(np.float64) + 1.0
+    mr = [oracle.quantize_multiplier(float(v)) for v in 100.0 / span * np.exp(g.uniform(-1.0, 1.0, size=n))]
+    mult, rsh = np.array([m for m, _ in mr], np.int32), np.array([r for _, r in mr], np.int32)
+    t_lo, t_hi = 0, 255                                   # a linear layer before the add
+    t = oracle.requantize(acc, mult, rsh, z_t, t_lo, t_hi).astype(np.uint8)
+    s = pitched(synth.uniform_u8((b, h, w, n), seed, 2), fill=0)
+    m_t, m_s, r = oracle.add_params(np.float32(st), np.float32(ss), np.float32(sy))
+    lo, hi = z_y, 255                                     # ReLU after the add
+    want = oracle.add_u8(t, z_t, m_t, s[..., :n], z_s, m_s, r, z_y, lo, hi)
+    assert {0.04: 16 <= r <= 38, 900.0: r >= 39, 0.0005: r < 16}.get(sy, True)
+    if 0.01 < sy < 1.0:
+        assert len(np.unique(want)) > 20
+    desc = qtz.conv_desc(b, h, w, c, n, k, k, 1, pad, wkind)
+    plan = hq.conv_create(desc, dev(api_w), dev(bias), zw, mult, rsh)
+    res = qtz.Residual(z_t, t_lo, t_hi, m_t, z_s, m_s, r)
+    s_dev = dev(s)
+    y = plan.add_fused(dev(x), z_x, res, s_dev, z_y, lo, hi, out=s_dev if alias else None)
+    assert "+residual-add" in plan.detail
+    assert np.array_equal(host(y)[..., :n], want)
+    # and it is what the two separate calls give
+    t_dev = plan(dev(x), z_x, z_t, t_lo, t_hi)
+    assert np.array_equal(host(t_dev)[..., :n], t)
+    two = hq.add_u8(t_dev, z_t, m_t, dev(s), z_s, m_s, r, z_y, lo, hi, n)
+    assert np.array_equal(host(two)[..., :n], want)
+
+
+def test_fused_residual_add_is_refused_where_it_cannot_run(hq):
+    w = dev(synth.uniform_s8((3, 3, 16), 1300, 0))
+    m, r = oracle.quantize_multiplier(0.01)
+    dw = hq.conv_create(qtz.conv_desc(1, 8, 8, 16, 16, 3, 3, 1, 1), w, None, None, np.full(16, m, np.int32),
+                        np.full(16, r, np.int32), depthwise=True)
+    x = dev(np.zeros((1, 8, 8, 16), np.uint8))
+    with pytest.raises(qtz.QtzError) as e:
+        dw.add_fused(x, 0, qtz.Residual(0, 0, 255, 1 << 30, 0, 1 << 30, 31), x, 0, 0, 255)
+    assert e.value.code == -1
+    raw = hq.conv_create(qtz.conv_desc(1, 8, 8, 16, 16, 1, 1, 1, 0, outkind=qtz.OUT_S32_RAW),
+                         dev(synth.uniform_s8((16, 1, 1, 16), 1300, 1)), None)
+    with pytest.raises(qtz.QtzError) as e:
+        raw.add_fused(x, 0, qtz.Residual(0, 0, 255, 1 << 30, 0, 1 << 30, 31), x, 0, 0, 255,
+                      out=torch.zeros((1, 8, 8, 16), dtype=torch.int32, device="cuda"))
+    assert e.value.code == -3
+
+
+@pytest.mark.parametrize("shape", [(16, 14, 14, 256, 512), (16, 7, 7, 512, 2048), (17, 14, 14, 256, 512), (5, 9, 9, 64, 1000)])
+def test_few_pixel_tiles_spread_over_column_tiles(hq, shape):
+    # a layer with few pixel tiles is split into narrow column tiles so that it covers the SMs; the split must not
+    # leave a role waiting for a column tile that lies beyond the real channels (the status word would say so)
+    b, h, w, c, n = shape
+    conv_case(hq, b, h, w, c, n, 1, 1, 0, qtz.W_S8_PER_CHANNEL_SYM, 1400 + n, expect_kernel="tcgen05")
+    torch.cuda.synchronize()
+    assert hq.device_status() == (0, 0)
