@@ -348,8 +348,9 @@ QTZ_API qtz_status qtz_avgpool_multiplier(int32_t hw, float x_scale, float y_sca
  *   mult_host, rshift_host  n entries: fixed-point form of Delta_x Delta_w[n] / Delta_y
  *               (ignored, may be NULL, with QTZ_OUT_S32_RAW).
  * The caller may free or overwrite all inputs once `stream` has passed this call.
- * Errors: QTZ_ERR_OVERFLOW when kh*kw*c > 32768; QTZ_ERR_UNSUPPORTED for depthwise layers
- * other than 3x3 / pad 1 / stride 1 or 2.                                                      */
+ * Errors: QTZ_ERR_OVERFLOW when kh*kw*c > 32768, or when kh*kw*c * 255 * max|w| + |bias_q[n]| (the
+ * largest accumulator any input can produce) does not fit int32; QTZ_ERR_UNSUPPORTED for
+ * depthwise layers other than 3x3 / pad 1 / stride 1 or 2.                                      */
 QTZ_API qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, int32_t depthwise,
                            const void* w_q_dev, const int32_t* bias_q_dev,
                            const int32_t* w_zero_point_host, const int32_t* mult_host,

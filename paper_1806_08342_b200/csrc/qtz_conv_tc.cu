@@ -8,13 +8,15 @@
 // One persistent CTA per SM, warp-specialised:
 //   warp 0      TMA producer: NHWC activation boxes (one shifted box per filter tap; out-of-image
 //               pixels arrive as zeros) and K-major weight tiles into a ring of swizzled stages
-//   warp 1      MMA issuer: one thread issues tcgen05.mma; two accumulators of up to 256 columns
-//               alternate in TMEM so that the epilogue of tile i overlaps the MMAs of tile i+1
-//   warps 2..17 epilogue, two groups of eight warps (one group per accumulator): tcgen05.ld, cross
-//               terms, requantise, clamp, pack to uint8 into a rotating set of swizzled staging boxes;
-//               the warps signal each filled box on an mbarrier and never wait for one another
-//   warps 18,19 one store thread per group: TMA store of every filled box (which also clips ragged
-//               tile edges), box handed back once the store has read it
+//   warp 1      MMA issuer: one elected lane issues tcgen05.mma; up to eight accumulators (512 TMEM columns / tile
+//               width) are used round robin, so the MMAs run several tiles ahead of the epilogue
+//   warps 2..17 epilogue: four groups of four warps (tiles up to 128 columns wide) or two groups of eight; the groups
+//               take the CTA's tiles in turn: tcgen05.ld, cross terms, requantise, clamp, pack to uint8 into a
+//               rotating set of swizzled staging boxes (optionally the residual add against a shortcut tile that the
+//               store lane fetched into the box); the warps signal each filled box on an mbarrier and never wait
+//               for one another.  For 4-bit layers the same warps first expand the packed weights into shared memory
+//   warp 18     one store lane per group: TMA store of every filled box (which also clips ragged tile edges), box
+//               handed back once the store has read it
 // Image stems (few channels, wide filters) run as "row-window" layers: a frame of the input padded
 // with z_x is staged one contiguous run per filter row (copied by the producer warp's lanes), and the MMA
 // reads the overlapping windows of 120 neighbouring output columns straight out of those runs (pad_copy_kernel).

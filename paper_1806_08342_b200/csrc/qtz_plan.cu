@@ -190,15 +190,23 @@ extern "C" qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, i
     PLAN_CUDA(cudaMalloc(reinterpret_cast<void**>(&p->bias), nb_alloc));
     PLAN_CUDA(cudaMemsetAsync(p->bias, 0, nb_alloc, st));
     if (bias_q_dev) PLAN_CUDA(cudaMemcpyAsync(p->bias, bias_q_dev, nb, cudaMemcpyDeviceToDevice, st));
-    if (!raw) {
-        // Largest accumulator any input can produce, and with it the largest requantised value: when
-        // that stays inside 32 bits for every channel, the epilogue may narrow before it clamps.
-        std::vector<int32_t> bias_host(static_cast<size_t>(d.n), 0);
-        if (bias_q_dev) {
-            PLAN_CUDA(cudaMemcpyAsync(bias_host.data(), bias_q_dev, nb, cudaMemcpyDeviceToHost, st));
-            PLAN_CUDA(cudaStreamSynchronize(st));
+    // Largest accumulator any input can produce: |acc| <= K 255 wmax + |bias|.  Beyond int32 the layer is refused
+    // (the accumulator of Eq. 4 is 32 bits wide); when even the requantised value stays inside 32 bits for every
+    // channel, the epilogue may narrow before it clamps.
+    std::vector<int32_t> bias_host(static_cast<size_t>(d.n), 0);
+    if (bias_q_dev) {
+        PLAN_CUDA(cudaMemcpyAsync(bias_host.data(), bias_q_dev, nb, cudaMemcpyDeviceToHost, st));
+        PLAN_CUDA(cudaStreamSynchronize(st));
+    }
+    const int64_t wmax = d.wkind == QTZ_W_S4_PACKED_PER_CHANNEL_SYM ? 8 : (d.wkind == QTZ_W_S8_PER_CHANNEL_SYM ? 128 : 255);
+    for (int i = 0; i < d.n; ++i) {
+        const int64_t bound = static_cast<int64_t>(p->k_total) * 255 * wmax + std::llabs(static_cast<long long>(bias_host[i]));
+        if (bound > 2147483647LL) {
+            qtz_conv_destroy(p);
+            return QTZ_ERR_OVERFLOW;
         }
-        const int64_t wmax = d.wkind == QTZ_W_S4_PACKED_PER_CHANNEL_SYM ? 8 : (d.wkind == QTZ_W_S8_PER_CHANNEL_SYM ? 128 : 255);
+    }
+    if (!raw) {
         p->narrow_ok = true;
         for (int i = 0; i < d.n; ++i) {
             const int64_t bound = static_cast<int64_t>(p->k_total) * 255 * wmax + std::llabs(static_cast<long long>(bias_host[i]));

@@ -30,8 +30,8 @@ struct qtz_plan {
     int32_t* bias = nullptr;      // [n + 16] (zeros when the layer has no bias); bias, mult, rshift are padded so that
                                   // 16-byte loads of a channel group never leave the array
     int32_t* wsum = nullptr;      // [classes][n] sum of int8 weight codes per border class
-    int32_t* mult = nullptr;      // [n]
-    int32_t* rshift = nullptr;    // [n]
+    int32_t* mult = nullptr;      // [n + 16], padded like bias (multiplier 0, shift 40 beyond n)
+    int32_t* rshift = nullptr;    // [n + 16]
     uint8_t* x_gather = nullptr;  // strided 1x1 layers: the sub-sampled input, pitched NHWC
     qtz_tc_state* tc = nullptr;
     qtz_dw_state* dw = nullptr;

@@ -431,3 +431,48 @@ def test_few_pixel_tiles_spread_over_column_tiles(hq, shape):
     conv_case(hq, b, h, w, c, n, 1, 1, 0, qtz.W_S8_PER_CHANNEL_SYM, 1400 + n, expect_kernel="tcgen05")
     torch.cuda.synchronize()
     assert hq.device_status() == (0, 0)
+
+
+# ---- requantisation forms the workloads rarely reach ---------------------------------------------------------
+@pytest.mark.parametrize("k,c,n", [(1, 32, 48), (3, 16, 32)])
+def test_requant_right_shifts_above_53(hq, k, c, n):
+    # real multipliers near 2e-8 give right shifts of 56 (the general 64-bit form); with int32 biases near +-1.9e9
+    # the outputs still spread over the code range
+    g = synth.rng(1500 + k, 0)
+    real_m = 2e-8 * np.exp(g.uniform(-0.6, 0.6, size=n))
+    assert all(54 <= oracle.quantize_multiplier(float(v))[1] <= 62 for v in real_m)
+    conv_case(hq, 2, 12, 12, c, n, k, 1, k // 2, qtz.W_S8_PER_CHANNEL_SYM, 1500 + k, real_m=real_m, bias_range=1_900_000_000)
+    torch.cuda.synchronize()
+    assert hq.device_status() == (0, 0)
+
+
+@pytest.mark.parametrize("k,c,n", [(1, 64, 40), (3, 32, 40)])
+def test_requant_large_values_with_small_shifts(hq, k, c, n):
+    # multipliers of 1..2 (right shift 30) and biases near 1e9: a requantised value can leave 32 bits before the
+    # clamp, so the narrow forms are not allowed and the 64-bit form must be taken
+    g = synth.rng(1510 + k, 0)
+    real_m = np.exp(g.uniform(0.05, 0.6, size=n))
+    assert all(oracle.quantize_multiplier(float(v))[1] == 30 for v in real_m)
+    conv_case(hq, 1, 6, 6, c, n, k, 1, k // 2, qtz.W_S8_PER_CHANNEL_SYM, 1510 + k, real_m=real_m, bias_range=1_000_000_000)
+    # the same multipliers with accumulators small enough for the narrow form (shift below 32, values within 32 bits)
+    conv_case(hq, 1, 6, 6, c, n, k, 1, k // 2, qtz.W_S8_PER_CHANNEL_SYM, 1520 + k, real_m=real_m / 4000.0, bias_range=2000)
+
+
+def test_layer_whose_accumulator_can_leave_int32_is_refused(hq):
+    # K 255 max|w| + |bias| beyond int32: the oracle reports overflow for the worst input, the library refuses the layer
+    c, n = 64, 16
+    w = np.full((n, 1, 1, c), 127, np.int8)
+    bias = np.full(n, 2_147_000_000, np.int32)
+    x = np.full((1, 2, 2, c), 255, np.uint8)
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.conv2d_acc(x, 0, w.astype(np.int32), None, bias, 1, 0)
+    assert e.value.code == -4
+    m, r = oracle.quantize_multiplier(1e-6)
+    with pytest.raises(qtz.QtzError) as e:
+        hq.conv_create(qtz.conv_desc(1, 2, 2, c, n, 1, 1, 1, 0), dev(w), dev(bias), None, np.full(n, m, np.int32), np.full(n, r, np.int32))
+    assert e.value.code == -4
+    with pytest.raises(qtz.QtzError) as e:
+        hq.conv_create(qtz.conv_desc(1, 2, 2, c, n, 1, 1, 1, 0, outkind=qtz.OUT_S32_RAW), dev(w), dev(bias))
+    assert e.value.code == -4
+    ok = hq.conv_create(qtz.conv_desc(1, 2, 2, c, n, 1, 1, 1, 0, outkind=qtz.OUT_S32_RAW), dev(w), dev(bias // 2))
+    assert np.array_equal(host(ok(dev(x), 0)), oracle.conv2d_acc(x, 0, w.astype(np.int32), None, bias // 2, 1, 0))

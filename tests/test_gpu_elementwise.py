@@ -162,7 +162,7 @@ def test_add_u8(hq, c, pixels):
         assert np.array_equal(got[:, :c], want[:, :c])
     # every shift range of the kernel: 16..38 (split multipliers), above 38, 10..15 and below 10
     for ma, mb, r in [(2147483647, 1518500250, 38), (1 << 30, 3 << 28, 16), (1 << 30, 3 << 28, 40), (1200, 700, 12), (37, 21, 5),
-                      (65535, 65536, 31), (0, 2147418113, 33)]:
+                      (65535, 65536, 31), (0, 2147418113, 33), (1 << 30, 3 << 28, 53), (2147483647, 1 << 29, 45), (1 << 30, 1 << 30, 39)]:
         want = oracle.add_u8(a, 200, ma, b, 13, mb, r, 77, 5, 250, c=c)
         got = host(hq.add_u8(dev(a), 200, ma, dev(b), 13, mb, r, 77, 5, 250, c))
         assert np.array_equal(got[:, :c], want[:, :c])
