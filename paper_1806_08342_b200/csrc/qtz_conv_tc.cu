@@ -124,6 +124,12 @@ struct TcArgs {
     // Fused residual add (Section 3.2.1): the convolution's own output code t (quantizer zy / act_min / act_max
     // above) is never stored; the shortcut tile s is brought into the output staging box by the store lane, and
     // the epilogue replaces it in place by clamp(z_y + ((t - z_t) m_t + (s - z_s) m_s + 2^(r-1)) >> r).
+    // CTA pairs (pointwise layers with wide tiles and a long reduction): two CTAs of a cluster work on one tile of
+    // 256 pixels x BN columns.  Each loads its own 128 pixel rows and its half of the weight tile (both CTAs' copies
+    // are counted on the first CTA's "full" barriers); the first CTA issues tcgen05.mma.cta_group::2 over both CTAs'
+    // shared memory (every weight K block is fetched from L2 by one of the two only), its commits arrive on both
+    // CTAs' barriers, and each CTA drains its own 128 accumulator rows.
+    int32_t pair;
     int32_t res;                            // 0: plain convolution
     int32_t res_kind;                       // arithmetic form of the add by its shift (see qtz_add_math.cuh)
     qtz_add::AddRule res_rule;
@@ -139,11 +145,11 @@ struct SmemLayout {
 // Operand ring (activations, and weights unless all `bres` weight blocks of the layer stay resident),
 // output staging boxes and one set of per-channel tables per epilogue group, barriers.
 __host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int groups, int obuf, int bres, int spb,
-                                                  int a_blk = 0)
+                                                  int a_blk = 0, int pair = 0)
 {
     SmemLayout L;
     L.a_blk = a_blk > 0 ? a_blk : kTileM * BK;   // one K block of activations (row-window layers: one run of the frame) / of weights
-    L.b_blk = BN * BK;
+    L.b_blk = (pair ? BN / 2 : BN) * BK;         // (a CTA of a pair holds half of the weight tile's columns)
     L.a_stage = (spb * L.a_blk + 1023u) & ~1023u;   // a ring stage holds spb consecutive K blocks; swizzled tiles behind the ring need 1 KB alignment
     L.b_stage = spb * L.b_blk;
     L.a_off = 0;
@@ -240,19 +246,21 @@ __device__ __forceinline__ void requant32(const uint32_t (&v)[32], const int32_t
 // Tile order: pixel tiles are taken in groups of group_m; inside a group the pixel tile varies
 // fastest, so the CTAs running at the same time share a band of A panels and a band of B panels
 // that together fit in L2.
-__device__ __forceinline__ void decode_tile(const TcArgs& a, uint32_t tile, uint32_t& m_tile, int& n_tile)
+__device__ __forceinline__ void decode_tile(const TcArgs& a, uint32_t tile, uint32_t& m_tile, int& n_tile, uint32_t prank)
 {
     if (a.n_tiles == 1) {                   // the usual case for a convolution layer: one column tile
         m_tile = tile;
         n_tile = 0;
-        return;
+    } else {
+        const uint32_t g = fdiv(tile, a.dv_per_group), r = tile - g * a.dv_per_group.d;
+        const uint32_t m_first = g * static_cast<uint32_t>(a.group_m);
+        const bool last = static_cast<uint32_t>(a.m_tiles) - m_first < static_cast<uint32_t>(a.group_m);   // a shorter final group
+        const uint32_t q = last ? fdiv(r, a.dv_group_last) : fdiv(r, a.dv_group_m);
+        m_tile = m_first + (r - q * (last ? a.dv_group_last.d : a.dv_group_m.d));
+        n_tile = static_cast<int>(q);
     }
-    const uint32_t g = fdiv(tile, a.dv_per_group), r = tile - g * a.dv_per_group.d;
-    const uint32_t m_first = g * static_cast<uint32_t>(a.group_m);
-    const bool last = static_cast<uint32_t>(a.m_tiles) - m_first < static_cast<uint32_t>(a.group_m);   // a shorter final group
-    const uint32_t q = last ? fdiv(r, a.dv_group_last) : fdiv(r, a.dv_group_m);
-    m_tile = m_first + (r - q * (last ? a.dv_group_last.d : a.dv_group_m.d));
-    n_tile = static_cast<int>(q);
+    // pair mode: the tile is a pair of pixel tiles, this CTA takes the one of its rank
+    if (a.pair) m_tile = 2 * m_tile + prank;
 }
 
 // First pixel (w0, h0, b0) of pixel tile m_tile.
@@ -271,6 +279,9 @@ __device__ __forceinline__ void tile_origin(const TcArgs& a, uint32_t m_tile, in
     }
 }
 
+// kPair: the CTA-pair form (launched as clusters of two; it contains cta_group::2 instructions, which a kernel
+// launched without clusters must not)
+template <bool kPair>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_s, const TcArgs a)
@@ -278,7 +289,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
-    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb, a.a_blk);
+    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb, a.a_blk, kPair);
 
     const uint32_t bar_full = base + L.bar_off;
     const uint32_t bar_empty = bar_full + 8 * kMaxStages;
@@ -289,6 +300,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t bar_wres = bar_oempty + 8 * kEpiGroups * kMaxObuf;         // resident weights have landed
     volatile uint32_t* const tmem_slot =
         reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + kNumBarriers * 8);
+    // pair mode: this CTA's place in its pair, and the pair's place among the pairs (tiles are dealt to pairs)
+    uint32_t prank = 0u;
+    if constexpr (kPair) prank = cluster_ctarank();
+    const uint32_t tile0 = kPair ? blockIdx.x >> 1 : blockIdx.x;
+    const uint32_t tile_step = kPair ? gridDim.x >> 1 : gridDim.x;
     volatile uint32_t* const abort_flag = tmem_slot + 1;
 
     // the shuffle tells the compiler that the warp index is the same in all lanes
@@ -301,7 +317,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int i = 0; i < kMaxAcc; ++i) {
             mbar_init(bar_tfull + 8 * i, 1);
-            mbar_init(bar_tempty + 8 * i, a.gwarps);
+            mbar_init(bar_tempty + 8 * i, kPair ? 2 * a.gwarps : a.gwarps);   // (a pair's accumulator is drained by both CTAs)
         }
         for (int i = 0; i < kEpiGroups * kMaxObuf; ++i) {
             mbar_init(bar_ofull + 8 * i, a.gwarps);
@@ -316,11 +332,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (a.res) prefetch_tensormap(&map_s);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
-        tmem_relinquish();
+        if constexpr (kPair) {
+            tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+            tmem_relinquish();
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (kPair) cluster_sync();      // both CTAs' barriers exist before anything arrives on them from the other CTA
     tc_fence_after();
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
 
@@ -334,12 +356,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // cycles per K block, which starves layers with a short reduction.)
         const uint32_t S = static_cast<uint32_t>(a.stages);
         const bool wres = a.bres > 0;
+        const int b_rows = kPair ? a.BN >> 1 : a.BN;      // weight rows (output channels) this CTA fetches per K block
         const uint32_t tx = static_cast<uint32_t>(a.spb) *
-                            static_cast<uint32_t>((a.cstride > 0 ? a.seg_bytes : a.rows * a.BK) + (wres ? 0 : a.BN * a.BK));
+                            static_cast<uint32_t>((a.cstride > 0 ? a.seg_bytes : a.rows * a.BK) + (wres ? 0 : b_rows * a.BK));
         const int nst = kblocks / a.spb;         // ring stages per tile
         uint32_t stage = 0, phase = 0;
         bool failed = false;
-        if (wres && a.w4 == nullptr && blockIdx.x < a.num_tiles) {
+        if (wres && a.w4 == nullptr && tile0 < a.num_tiles) {
             // the layer's weights are small: fetch all of their K blocks once, they stay for every tile
             if (elect_one()) {
                 mbar_arrive_expect_tx(bar_wres, static_cast<uint32_t>(a.bres) * L.b_blk);
@@ -356,10 +379,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // stages a signal trails its copies by (what may be in flight); two stages short of the ring so that the MMA
         // warp always has signalled stages ahead of it while the producer waits for a free one
         const uint32_t lag = max(1u, min(S - 3u, 6u));
-        for (uint32_t tile = blockIdx.x; a.lsu != 0 && !failed && tile < a.num_tiles; tile += gridDim.x) {
+        for (uint32_t tile = tile0; a.lsu != 0 && !failed && tile < a.num_tiles; tile += tile_step) {
             int n_tile, w0, h0, b0;
             uint32_t m_tile;
-            decode_tile(a, tile, m_tile, n_tile);
+            decode_tile(a, tile, m_tile, n_tile, prank);
             tile_origin(a, m_tile, w0, h0, b0);
             const int nrow = n_tile * a.BN;
             for (int st = 0; st < nst; ++st) {
@@ -414,12 +437,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             __syncwarp();
         }
-        for (uint32_t tile = blockIdx.x; a.lsu == 0 && !failed && tile < a.num_tiles; tile += gridDim.x) {
+        for (uint32_t tile = tile0; a.lsu == 0 && !failed && tile < a.num_tiles; tile += tile_step) {
             int n_tile, w0, h0, b0;
             uint32_t m_tile;
-            decode_tile(a, tile, m_tile, n_tile);
+            decode_tile(a, tile, m_tile, n_tile, prank);
             tile_origin(a, m_tile, w0, h0, b0);
-            const int nrow = n_tile * a.BN;
+            const int nrow = n_tile * a.BN + static_cast<int>(prank) * b_rows;   // (pair mode: this CTA's half of the columns)
             int tap_x = 0, tap_y = 0, kcol = 0, kc = 0;   // filter tap of the next K block, its first weight column, channel offset
             // row-window layers: the tile is a run of output columns of one output row; filter row tap_y
             // reads frame row h0 * cstride + tap_y from the byte where the window of column w0 starts (16 w0)
@@ -431,7 +454,28 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     break;
                 }
                 const bool leader = elect_one();
-                const uint32_t full = bar_full + 8 * stage;
+                uint32_t full = bar_full + 8 * stage;
+                if constexpr (kPair) {
+                    // both CTAs' copies are counted on the FIRST CTA's barrier, which its MMA warp waits on
+                    if (prank == 0) {
+                        if (leader) mbar_arrive_expect_tx(full, 2 * tx);
+                    } else {
+                        full = mapa_shared(full, 0u);
+                    }
+                    for (int j = 0; j < a.spb; ++j) {
+                        if (leader) {
+                            tma_load_2d_pair(base + L.a_off + stage * L.a_stage + j * L.a_blk, &map_a, full, kc, w0);
+                            tma_load_2d_pair(base + L.b_off + stage * L.b_stage + j * L.b_blk, &map_b, full, kcol + kc, nrow);
+                        }
+                        kc += a.BK;
+                    }
+                    __syncwarp();
+                    if (++stage == S) {
+                        stage = 0;
+                        phase ^= 1;
+                    }
+                    continue;
+                }
                 if (leader) mbar_arrive_expect_tx(full, tx);
                 for (int j = 0; j < a.spb; ++j) {
                     if (leader) {
@@ -489,15 +533,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t acc = 0, acc_phase = 0;     // accumulators are used round robin
         bool ok = true;
         const bool wres = a.bres > 0;
-        if (wres && blockIdx.x < a.num_tiles && !__all_sync(0xffffffffu, mbar_wait(bar_wres, 0, a.wait_budget, 64u))) {
+        if (wres && tile0 < a.num_tiles && !__all_sync(0xffffffffu, mbar_wait(bar_wres, 0, a.wait_budget, 64u))) {
             if (lane == 0) {
                 report_timeout(a.status, QTZ_SITE_TMA_FULL);
                 *abort_flag = 1;
             }
             ok = false;
         }
-        for (uint32_t tile = blockIdx.x; ok && tile < a.num_tiles; tile += gridDim.x) {
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget, 128u))) {
+        // (the second CTA of a pair issues no MMAs: its copies are counted on the first CTA's barriers, its stages are
+        //  freed and its accumulators published by the first CTA's commits, which arrive on both CTAs' barriers)
+        for (uint32_t tile = tile0; ok && (!kPair || prank == 0) && tile < a.num_tiles; tile += tile_step) {
+            if (!__all_sync(0xffffffffu, kPair ? mbar_wait_cluster(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget, 128u)
+                                             : mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, a.wait_budget, 128u))) {
                 if (lane == 0) {
                     report_timeout(a.status, QTZ_SITE_TMEM_EMPTY);
                     *abort_flag = 1;
@@ -507,7 +554,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * a.acc_stride;
             for (int st = 0; st < nst; ++st) {
-                if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8 * stage, phase, a.wait_budget, 64u))) {
+                const bool full = __all_sync(0xffffffffu, kPair ? mbar_wait_cluster(bar_full + 8 * stage, phase, a.wait_budget, 64u)
+                                                                : mbar_wait(bar_full + 8 * stage, phase, a.wait_budget, 64u));
+                if (!full) {
                     if (lane == 0) {
                         report_timeout(a.status, QTZ_SITE_TMA_FULL);
                         *abort_flag = 1;
@@ -520,17 +569,31 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     uint64_t da = desc_a0 + stage * a_step;
                     uint64_t db = desc_b0 + (wres ? static_cast<uint32_t>(st * a.spb) * b_blk : stage * b_step);
                     uint32_t accumulate = st > 0 ? 1u : 0u;      // the tile's first MMA overwrites the accumulator
-                    for (int j = 0; j < a.spb; ++j, da += a_blk, db += b_blk) {
-                        mma_i8(d_tmem, da, db, a.idesc, accumulate);
-                        if (mmas >= 2) mma_i8(d_tmem, da + 2, db + 2, a.idesc, 1u);
-                        if (mmas == 4) {
-                            mma_i8(d_tmem, da + 4, db + 4, a.idesc, 1u);
-                            mma_i8(d_tmem, da + 6, db + 6, a.idesc, 1u);
+                    if constexpr (kPair) {
+                        for (int j = 0; j < a.spb; ++j, da += a_blk, db += b_blk) {
+                            mma_i8_pair(d_tmem, da, db, a.idesc, accumulate);
+                            if (mmas >= 2) mma_i8_pair(d_tmem, da + 2, db + 2, a.idesc, 1u);
+                            if (mmas == 4) {
+                                mma_i8_pair(d_tmem, da + 4, db + 4, a.idesc, 1u);
+                                mma_i8_pair(d_tmem, da + 6, db + 6, a.idesc, 1u);
+                            }
+                            accumulate = 1u;
                         }
-                        accumulate = 1u;
+                        mma_commit_pair(bar_empty + 8 * stage);              // frees the stage in both CTAs
+                        if (st == nst - 1) mma_commit_pair(bar_tfull + 8 * acc);
+                    } else {
+                        for (int j = 0; j < a.spb; ++j, da += a_blk, db += b_blk) {
+                            mma_i8(d_tmem, da, db, a.idesc, accumulate);
+                            if (mmas >= 2) mma_i8(d_tmem, da + 2, db + 2, a.idesc, 1u);
+                            if (mmas == 4) {
+                                mma_i8(d_tmem, da + 4, db + 4, a.idesc, 1u);
+                                mma_i8(d_tmem, da + 6, db + 6, a.idesc, 1u);
+                            }
+                            accumulate = 1u;
+                        }
+                        mma_commit(bar_empty + 8 * stage);                     // frees the stage once these MMAs have read it
+                        if (st == nst - 1) mma_commit(bar_tfull + 8 * acc);
                     }
-                    mma_commit(bar_empty + 8 * stage);                     // frees the stage once these MMAs have read it
-                    if (st == nst - 1) mma_commit(bar_tfull + 8 * acc);
                 }
                 __syncwarp();
                 if (++stage == S) {
@@ -560,10 +623,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             };
             auto enter_tile = [&](BoxIter& it) {
                 // (a column tile that lies wholly beyond the real channels has no box at all: skip it)
-                for (; it.tile < a.num_tiles; it.tile += a.groups * gridDim.x) {
+                for (; it.tile < a.num_tiles; it.tile += a.groups * tile_step) {
                     int n_tile;
                     uint32_t m_tile;
-                    decode_tile(a, it.tile, m_tile, n_tile);
+                    decode_tile(a, it.tile, m_tile, n_tile, prank);
                     it.nn = n_tile * a.BN;
                     it.left = a.BN;
                     if (it.nn >= a.N) continue;
@@ -575,7 +638,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 it.nn += a.out_box;
                 it.left -= a.out_box;
                 if (!(it.left > 0 && it.nn < a.N)) {
-                    it.tile += a.groups * gridDim.x;
+                    it.tile += a.groups * tile_step;
                     enter_tile(it);
                 }
             };
@@ -588,7 +651,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 else
                     tma_load_2d(out_addr + slot_ * box_bytes, &map_s, oempty + 8 * slot_, it.nn, it.w0);
             };
-            BoxIter cur{blockIdx.x + grp * gridDim.x, 0, 0, 0, 0, 0};
+            BoxIter cur{tile0 + grp * tile_step, 0, 0, 0, 0, 0};
             enter_tile(cur);
             BoxIter ahead = cur;
             if (a.res)
@@ -676,13 +739,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int dr_h = a.is4d ? (row / a.tw) % a.th : 0;
         const int dr_b = a.is4d ? row / (a.tw * a.th) : 0;
         int staged_n_tile = -1;
-        if (a.w4 != nullptr && a.bres > 0 && blockIdx.x < a.num_tiles) {
+        if (a.w4 != nullptr && a.bres > 0 && tile0 < a.num_tiles) {
             // 4-bit weights: the layer's codes stay packed in global memory (two per byte along K); all sixteen
             // epilogue warps expand this CTA's column tile to int8 once, straight into the swizzled K blocks the
             // tensor cores read.  A thread takes 16 packed bytes = 32 codes = two 16-byte chunks of one row.
             int n_tile0;
             uint32_t m_tile0;
-            decode_tile(a, blockIdx.x, m_tile0, n_tile0);       // (a CTA with several tiles has a single column tile)
+            decode_tile(a, tile0, m_tile0, n_tile0, prank);       // (a CTA with several tiles has a single column tile)
             const int parts = a.BK >> 5;                        // 32-code pieces per row of a K block
             const int per_blk = a.BN * parts;
             const uint8_t* const src = a.w4 + static_cast<int64_t>(n_tile0) * a.BN * a.w4_row;
@@ -715,8 +778,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // with two groups in use, group g takes every other tile (accumulator g); with one, group 0 takes all
         // the CTA's i-th tile lives in accumulator i mod n_acc
         uint32_t next_acc = grp % a.n_acc, next_acc_phase = (grp / a.n_acc) & 1;
-        uint32_t tile = grp < a.groups ? blockIdx.x + grp * gridDim.x : a.num_tiles;
-        for (; tile < a.num_tiles; tile += a.groups * gridDim.x) {
+        uint32_t tile = grp < a.groups ? tile0 + grp * tile_step : a.num_tiles;
+        for (; tile < a.num_tiles; tile += a.groups * tile_step) {
             const uint32_t acc = next_acc, acc_phase = next_acc_phase;
             next_acc += a.groups;
             while (next_acc >= static_cast<uint32_t>(a.n_acc)) {
@@ -725,7 +788,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             int n_tile;
             uint32_t m_tile;
-            decode_tile(a, tile, m_tile, n_tile);
+            decode_tile(a, tile, m_tile, n_tile, prank);
             const int n0 = n_tile * a.BN;
 
             if (n_tile != staged_n_tile) {
@@ -812,7 +875,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+                if (lane == 0) {
+                    if (kPair && prank != 0) { if constexpr (kPair) mbar_arrive_remote(bar_tempty + 8 * acc, 0u); }
+                    else mbar_arrive(bar_tempty + 8 * acc);
+                }
                 continue;
             }
 
@@ -877,7 +943,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(ofull + 8 * slot);
-                    if (drained) mbar_arrive(bar_tempty + 8 * acc);   // accumulator back to the MMA warp
+                    if (drained) {                                    // accumulator back to the MMA warp (of the pair's first CTA)
+                        if (kPair && prank != 0) { if constexpr (kPair) mbar_arrive_remote(bar_tempty + 8 * acc, 0u); }
+                        else mbar_arrive(bar_tempty + 8 * acc);
+                    }
                 }
                 if (++slot == static_cast<uint32_t>(a.obuf)) {
                     slot = 0;
@@ -889,9 +958,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     tc_fence_before();
     __syncthreads();
+    if constexpr (kPair) cluster_sync();      // the other CTA's MMAs and arrivals no longer touch this CTA's shared memory
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, kTmemCols);
+        if constexpr (kPair) tmem_dealloc_pair(tmem_base, kTmemCols);
+        else tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -1168,6 +1239,9 @@ struct qtz_tc_state {
     size_t frame_bytes = 0;    // the frame with its slack
     int cs = 0;                // im2col: bytes per tap in the window matrix (channels rounded up to 4)
     CUtensorMap map_b{};
+    CUtensorMap map_b_half{};  // pair mode: boxes of half the column tile
+    bool pair = false;         // the layer runs on CTA pairs (clusters of two, tcgen05 cta_group::2)
+    int pair_clusters = 0;     // pairs that can be resident at once
     int8_t* w_packed = nullptr;
     uint8_t* w_packed4 = nullptr;   // 4-bit layers: the same re-laid rows with two codes per byte (what the kernel reads when
                                     // the layer's weights are expanded in shared memory)
@@ -1418,6 +1492,30 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     }
 
     a.m_tiles = static_cast<int32_t>(a.num_tiles / a.n_tiles);
+    // CTA pairs for GEMM-like pointwise layers: full-width column tiles, a reduction of at least 1024 and enough tiles
+    // to fill the SMs.  A pair works on 256 pixels x 256 columns, each CTA fetching half of every weight K block.
+    a.pair = 0;
+    if (pw && a.BN == 256 && d.c >= 1024 && a.num_tiles >= static_cast<uint32_t>(h->num_sms) && !h->no_pairs) {
+        int clusters = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(h->num_sms / 2 * 2));
+        cfg.blockDim = dim3(kThreadsTc);
+        cfg.dynamicSmemBytes = 227 * 1024;
+        cudaLaunchAttribute at;
+        at.id = cudaLaunchAttributeClusterDimension;
+        at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+        cfg.attrs = &at;
+        cfg.numAttrs = 1;
+        (void)cudaFuncSetAttribute(conv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (cudaOccupancyMaxActiveClusters(&clusters, conv_tc_kernel<true>, &cfg) == cudaSuccess && clusters >= h->num_sms / 4) {
+            a.pair = 1;
+            t->pair = true;
+            a.m_tiles = (a.m_tiles + 1) / 2;
+            a.num_tiles = static_cast<uint32_t>(a.m_tiles) * a.n_tiles;
+            t->pair_clusters = clusters;
+        }
+        (void)cudaGetLastError();
+    }
     a.group_m = std::max(1, std::min(a.m_tiles, 16));
     a.dv_per_group = make_fastdiv(static_cast<uint32_t>(a.group_m) * a.n_tiles);
     a.dv_group_m = make_fastdiv(static_cast<uint32_t>(a.group_m));
@@ -1436,7 +1534,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
 
     // instruction descriptor: s32 accumulate, A = u8, B = s8, both K-major, N and M of the tile
     a.idesc = (2u << 4) | (0u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) |
-              (static_cast<uint32_t>(kTileM >> 4) << 24);
+              (static_cast<uint32_t>((a.pair ? 2 * kTileM : kTileM) >> 4) << 24);
 
     // weights: re-lay, then the per-class sums
     const int64_t wbytes = static_cast<int64_t>(t->n_pad) * a.taps * a.c_pad;
@@ -1490,6 +1588,11 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
             h->last_error = "cuTensorMapEncodeTiled failed for the weight tensor";
             return QTZ_ERR_CUDA;
         }
+        const uint32_t half_box[2] = {static_cast<uint32_t>(a.BK), static_cast<uint32_t>(a.BN / 2)};
+        if (t->pair && !encode_map(&t->map_b_half, t->w_packed, 2, dims, strides, half_box, a.BK)) {
+            h->last_error = "cuTensorMapEncodeTiled failed for the weight tensor (half tiles)";
+            return QTZ_ERR_CUDA;
+        }
     }
     a.bias = p->bias;
     a.wsum = p->wsum;
@@ -1502,10 +1605,11 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.fold = 0;                             // decided per launch (it depends on the zero points)
     a.status = h->status_dev;
     a.wait_budget = h->wait_budget;
-    t->grid = static_cast<int>(std::min<int64_t>(a.num_tiles, h->num_sms));
+    t->grid = t->pair ? 2 * static_cast<int>(std::min<int64_t>(a.num_tiles, t->pair_clusters))
+                      : static_cast<int>(std::min<int64_t>(a.num_tiles, h->num_sms));
 
     // per device, so set for the device of this plan every time (the call is cheap)
-    QTZ_CUDA(h, cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    QTZ_CUDA(h, cudaFuncSetAttribute(conv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     return QTZ_OK;
 }
 
@@ -1619,7 +1723,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     auto depth = [&](int groups, int obuf) {
         int st_ = kMaxStages;
         for (; st_ >= 2; --st_)
-            if (make_layout(a.BK, a.BN, st_, a.ncls, a.out_box, groups, obuf, a.bres, a.spb, a.a_blk).total <= static_cast<uint32_t>(kSmemBudget)) break;
+            if (make_layout(a.BK, a.BN, st_, a.ncls, a.out_box, groups, obuf, a.bres, a.spb, a.a_blk, a.pair).total <= static_cast<uint32_t>(kSmemBudget)) break;
         return st_;
     };
     const int kblocks = a.taps * a.kb_per_tap;
@@ -1631,9 +1735,10 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
         a.bres = ((a.n_tiles == 1 || one_tile_each) && kblocks * a.BN * a.BK <= kResidentB4Max) ? kblocks : 0;
     else
         a.bres = (a.n_tiles == 1 && kblocks * a.BN * a.BK <= kResidentBMax) ? kblocks : 0;
+    if (a.pair) a.bres = 0;                          // a pair streams its weight halves
     // several K blocks share a ring stage (one barrier handshake for all of them) while the stage stays within 32 KB
     auto blocks_per_stage = [&]() {
-        const int blk = (a.a_blk > 0 ? a.a_blk : kTileM * a.BK) + (a.bres > 0 ? 0 : a.BN * a.BK);
+        const int blk = (a.a_blk > 0 ? a.a_blk : kTileM * a.BK) + (a.bres > 0 ? 0 : (a.pair ? a.BN / 2 : a.BN) * a.BK);
         int best = 1;
         for (int c = 2; c <= (a.a_blk > 0 ? 8 : 4); ++c)
             if (kblocks % c == 0 && c * blk <= 32 * 1024) best = c;
@@ -1641,6 +1746,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     };
     a.spb = blocks_per_stage();
     int need = std::min(4, kblocks / a.spb + 1);
+    if (a.pair) need = 6;                            // the pair's hand-offs cross SMs: a deeper ring, fewer staging boxes
     static const int choice[7][2] = {{4, 3}, {4, 2}, {2, 3}, {2, 2}, {1, 2}, {2, 1}, {1, 1}};
     // attempts: resident weights with several K blocks per stage; resident weights with one K block per stage (a
     // smaller ring beside a large resident tile); weights through the ring
@@ -1670,7 +1776,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.gwarps = a.groups == 4 ? 4 : 8;
     a.stages = depth(a.groups, a.obuf);
     if (a.stages < 2) return QTZ_ERR_UNSUPPORTED;
-    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb, a.a_blk).total + 1024;
+    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb, a.a_blk, a.pair).total + 1024;
     // folded form: shifts 32..53 (the high word of the 64-bit sum, shifted on by r - 32)
     // (2: shifts below 32 as well, given that no requantised value can leave 32 bits)
     a.fold = 0;
@@ -1686,9 +1792,23 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.w4_row = (a.taps * a.c_pad) >> 1;
     p->detail = std::string("tcgen05") + (t->rowwin ? " row-window" : (t->im2col ? " im2col" : (pw ? " pointwise" : " 3x3"))) +
                 (a.bres > 0 ? (a.w4 ? " weights:int4-expanded-in-smem" : " weights:resident") : " weights:streamed") +
-                (a.res ? " +residual-add" : "");
+                (a.pair ? " cta-pairs" : "") + (a.res ? " +residual-add" : "");
     if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
-    conv_tc_kernel<<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, map_s, a);
+    if (t->pair) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(t->grid));
+        cfg.blockDim = dim3(kThreadsTc);
+        cfg.dynamicSmemBytes = smem_bytes;
+        cfg.stream = st;
+        cudaLaunchAttribute at;
+        at.id = cudaLaunchAttributeClusterDimension;
+        at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+        cfg.attrs = &at;
+        cfg.numAttrs = 1;
+        QTZ_CUDA(h, cudaLaunchKernelEx(&cfg, conv_tc_kernel<true>, map_a, t->map_b_half, map_y, map_s, a));
+    } else {
+        conv_tc_kernel<false><<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, map_s, a);
+    }
     QTZ_LAUNCH_CHECK(h, "conv_tc_kernel");
     if (p->ev_stop) QTZ_CUDA(h, cudaEventRecord(p->ev_stop, st));
     return QTZ_OK;

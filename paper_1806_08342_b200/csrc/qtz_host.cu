@@ -1,6 +1,7 @@
 // Handle management and the host-side scalar rules of libqtz: quantizer parameters
 // from a range (Section 2.1-2.2), fixed-point multipliers, activation clamp ranges.
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -35,6 +36,7 @@ extern "C" qtz_status qtz_create(qtz_handle* out, int device)
     qtz_ctx* h = new (std::nothrow) qtz_ctx();
     if (!h) return QTZ_ERR_INVALID_ARG;
     h->device = device;
+    if (const char* v = std::getenv("QTZ_NO_PAIRS")) h->no_pairs = v[0] == '1';
     cudaError_t e = cudaSetDevice(device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) e = cudaMalloc(&h->status_dev, 2 * sizeof(int32_t));

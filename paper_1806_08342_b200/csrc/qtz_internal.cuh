@@ -24,6 +24,7 @@ struct qtz_ctx {
     int32_t* status_dev = nullptr;
     float* reduce_host = nullptr;  // pinned
     size_t reduce_host_bytes = 0;
+    bool no_pairs = false;                  // never run layers on CTA pairs (A/B comparisons; set by QTZ_NO_PAIRS=1)
     long long wait_budget = 2000000000LL;   // cycle budget of every bounded device-side wait (about one second)
     std::string last_error;
 };

@@ -267,6 +267,8 @@ def gemm_case(hq, m, n, k, seed=2, rows=None):
     assert np.array_equal(got[rows][:, :n].astype(np.int32), want)
     assert len(np.unique(want)) > 50
     assert plan.kernel == "tcgen05"
+    # GEMM-like layers (full-width column tiles, long reduction, at least a tile per SM) run on CTA pairs
+    assert ("cta-pairs" in plan.detail) == (n >= 256 and k >= 1024 and (m // 128) * (n // 256) >= 148), plan.detail
     return plan.kernel
 
 
