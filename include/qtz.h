@@ -358,7 +358,8 @@ QTZ_API qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, int3
 QTZ_API qtz_status qtz_conv_destroy(qtz_conv_plan p);
 /* Profiling hook: when both events (cudaEvent_t as void*) are non-NULL, every later
  * qtz_conv2d_u8 / qtz_depthwise_u8 call on this plan records them on the launch stream
- * immediately before and after its main kernel (pre-passes excluded).  NULL, NULL clears.   */
+ * immediately before and after its main kernel (pre-passes excluded, except the activation-sum
+ * pre-pass of asymmetric-weight layers, beside which the main kernel runs).  NULL, NULL clears. */
 QTZ_API qtz_status qtz_conv_set_profile_events(qtz_conv_plan p, void* start_event, void* stop_event);
 /* Name of the kernel family a plan dispatches to ("tcgen05", "direct", "depthwise").           */
 QTZ_API const char* qtz_conv_plan_kernel(qtz_conv_plan p);

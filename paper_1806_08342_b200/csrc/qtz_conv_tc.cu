@@ -739,6 +739,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int dr_h = a.is4d ? (row / a.tw) % a.th : 0;
         const int dr_b = a.is4d ? row / (a.tw * a.th) : 0;
         int staged_n_tile = -1;
+        // the activation sums come from the kernel launched just before this one, which may still be running
+        if (a.zw != 0) grid_dependency_wait();
         if (a.w4 != nullptr && a.bres > 0 && tile0 < a.num_tiles) {
             // 4-bit weights: the layer's codes stay packed in global memory (two per byte along K); all sixteen
             // epilogue warps expand this CTA's column tile to int8 once, straight into the swizzled K blocks the
@@ -1039,6 +1041,9 @@ class_sums_kernel(const int8_t* __restrict__ wp, int n, int taps, int kw, int c_
 __global__ void __launch_bounds__(kPrepThreads)
 pixel_sum_kernel(const uint8_t* __restrict__ x, int64_t pixels, int c, int pitch, int32_t* __restrict__ xsum)
 {
+    // the convolution that follows needs these sums only in its epilogue: let it start now (its copies and MMAs run
+    // beside this kernel; its epilogue waits for this grid before the first read of xsum)
+    grid_launch_dependents();
     const int warps_per_block = kPrepThreads / 32;
     const int lane = threadIdx.x & 31;
     for (int64_t p = static_cast<int64_t>(blockIdx.x) * warps_per_block + (threadIdx.x >> 5); p < pixels;
@@ -1492,10 +1497,12 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     }
 
     a.m_tiles = static_cast<int32_t>(a.num_tiles / a.n_tiles);
-    // CTA pairs for GEMM-like pointwise layers: full-width column tiles, a reduction of at least 1024 and enough tiles
-    // to fill the SMs.  A pair works on 256 pixels x 256 columns, each CTA fetching half of every weight K block.
+    // CTA pairs for GEMM-like pointwise layers: full-width column tiles, a reduction and a width of at least 2048 and
+    // at least two tiles per SM.  A pair works on 256 pixels x 256 columns, each CTA fetching half of every weight K block.
     a.pair = 0;
-    if (pw && a.BN == 256 && d.c >= 1024 && a.num_tiles >= static_cast<uint32_t>(h->num_sms) && !h->no_pairs) {
+    // (measured: layers of the networks with K = 1024..2048 and a few hundred tiles, which are bound by HBM and by
+    //  latency rather than by the tensor cores, run about 10 % slower on pairs, so the bar is set above them)
+    if (pw && a.BN == 256 && d.c >= 2048 && d.n >= 2048 && a.num_tiles >= 2 * static_cast<uint32_t>(h->num_sms) && !h->no_pairs) {
         int clusters = 0;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(static_cast<unsigned>(h->num_sms / 2 * 2));
@@ -1653,6 +1660,9 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
         xin = p->x_gather;
     }
     if (a.zw != 0) {
+        // the convolution starts beside this pre-pass (programmatic dependent launch), so the profiling events
+        // bracket the two together
+        if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
         const int blocks = static_cast<int>(std::min<int64_t>((t->in_pixels + 7) / 8, static_cast<int64_t>(h->num_sms) * 16));
         pixel_sum_kernel<<<blocks, kPrepThreads, 0, st>>>(xin, t->in_pixels, d.c, d.c_pitch_in, t->xsum);
         QTZ_LAUNCH_CHECK(h, "pixel_sum_kernel");
@@ -1793,21 +1803,32 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     p->detail = std::string("tcgen05") + (t->rowwin ? " row-window" : (t->im2col ? " im2col" : (pw ? " pointwise" : " 3x3"))) +
                 (a.bres > 0 ? (a.w4 ? " weights:int4-expanded-in-smem" : " weights:resident") : " weights:streamed") +
                 (a.pair ? " cta-pairs" : "") + (a.res ? " +residual-add" : "");
-    if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
-    if (t->pair) {
+    if (p->ev_start && a.zw == 0) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
+    {
+        // cluster of two for the pair form; early start beside pixel_sum_kernel when that kernel was just launched
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(static_cast<unsigned>(t->grid));
         cfg.blockDim = dim3(kThreadsTc);
         cfg.dynamicSmemBytes = smem_bytes;
         cfg.stream = st;
-        cudaLaunchAttribute at;
-        at.id = cudaLaunchAttributeClusterDimension;
-        at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
-        cfg.attrs = &at;
-        cfg.numAttrs = 1;
-        QTZ_CUDA(h, cudaLaunchKernelEx(&cfg, conv_tc_kernel<true>, map_a, t->map_b_half, map_y, map_s, a));
-    } else {
-        conv_tc_kernel<false><<<t->grid, kThreadsTc, smem_bytes, st>>>(map_a, t->map_b, map_y, map_s, a);
+        cudaLaunchAttribute at[2];
+        unsigned n_at = 0;
+        if (t->pair) {
+            at[n_at].id = cudaLaunchAttributeClusterDimension;
+            at[n_at].val.clusterDim.x = 2; at[n_at].val.clusterDim.y = 1; at[n_at].val.clusterDim.z = 1;
+            ++n_at;
+        }
+        if (a.zw != 0) {
+            at[n_at].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            at[n_at].val.programmaticStreamSerializationAllowed = 1;
+            ++n_at;
+        }
+        cfg.attrs = at;
+        cfg.numAttrs = n_at;
+        if (t->pair)
+            QTZ_CUDA(h, cudaLaunchKernelEx(&cfg, conv_tc_kernel<true>, map_a, t->map_b_half, map_y, map_s, a));
+        else
+            QTZ_CUDA(h, cudaLaunchKernelEx(&cfg, conv_tc_kernel<false>, map_a, t->map_b, map_y, map_s, a));
     }
     QTZ_LAUNCH_CHECK(h, "conv_tc_kernel");
     if (p->ev_stop) QTZ_CUDA(h, cudaEventRecord(p->ev_stop, st));

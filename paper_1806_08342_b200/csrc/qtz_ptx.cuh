@@ -153,6 +153,14 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t columns)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(columns) : "memory");
 }
 
+// ---- programmatic dependent launch -----------------------------------------------------------------------
+// A kernel launched with the programmatic-serialization attribute may start while the kernel before it in the
+// stream is still running; grid_dependency_wait() blocks until that kernel has finished and its writes are
+// visible (it returns at once in a normal launch).  The earlier kernel allows the early start with
+// grid_launch_dependents().
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- CTA pairs (thread-block clusters of two, tcgen05 cta_group::2) --------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {

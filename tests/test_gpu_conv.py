@@ -268,7 +268,7 @@ def gemm_case(hq, m, n, k, seed=2, rows=None):
     assert len(np.unique(want)) > 50
     assert plan.kernel == "tcgen05"
     # GEMM-like layers (full-width column tiles, long reduction, at least a tile per SM) run on CTA pairs
-    assert ("cta-pairs" in plan.detail) == (n >= 256 and k >= 1024 and (m // 128) * (n // 256) >= 148), plan.detail
+    assert ("cta-pairs" in plan.detail) == (n >= 2048 and k >= 2048 and (m // 128) * (n // 256) >= 296), plan.detail
     return plan.kernel
 
 
