@@ -330,6 +330,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         prefetch_tensormap(&map_b);
         prefetch_tensormap(&map_y);
         if (a.res) prefetch_tensormap(&map_s);
+        // the next kernel of the stream may be scheduled as this one's CTAs leave (it waits for this grid before it
+        // touches activations: grid_dependency_wait below)
+        grid_launch_dependents();
     }
     if (warp == 1) {
         if constexpr (kPair) {
@@ -373,6 +376,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             __syncwarp();
         }
+        // This kernel may have started while the kernel before it in the stream was still running (programmatic
+        // dependent launch): everything above touched only the layer's own constants; activations wait.
+        grid_dependency_wait();
         // ---- thread copies: every lane copies 16-byte pieces of the stage's activations; a stage is signalled
         // `lag` stages late, once this warp's copies for it have landed and been fenced for the tensor cores
         uint32_t issued = 0, signalled = 0, sig_stage = 0;
@@ -611,6 +617,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // One lane per epilogue group turns filled staging boxes into TMA stores and hands each box
         // back once its store has read it, so the warps doing arithmetic never wait on a store.
         const int grp = lane;
+        grid_dependency_wait();          // the output may alias a buffer the previous kernel still reads; so may the shortcut
         if (grp < a.groups && !a.raw) {
             const uint32_t box_bytes = kTileM * a.out_box;
             const uint32_t out_addr = base + L.out_off + grp * a.obuf * box_bytes;
@@ -739,8 +746,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int dr_h = a.is4d ? (row / a.tw) % a.th : 0;
         const int dr_b = a.is4d ? row / (a.tw * a.th) : 0;
         int staged_n_tile = -1;
-        // the activation sums come from the kernel launched just before this one, which may still be running
-        if (a.zw != 0) grid_dependency_wait();
+        // the activation sums come from the kernel launched just before this one, which may still be running; raw
+        // accumulators are stored by these warps themselves
+        if (a.zw != 0 || a.raw) grid_dependency_wait();
         if (a.w4 != nullptr && a.bres > 0 && tile0 < a.num_tiles) {
             // 4-bit weights: the layer's codes stay packed in global memory (two per byte along K); all sixteen
             // epilogue warps expand this CTA's column tile to int8 once, straight into the swizzled K blocks the
@@ -958,6 +966,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     }
 
+    if (threadIdx.x == 0) grid_dependency_wait();   // even a CTA without tiles leaves only after the previous grid
     tc_fence_before();
     __syncthreads();
     if constexpr (kPair) cluster_sync();      // the other CTA's MMAs and arrivals no longer touch this CTA's shared memory
@@ -1818,7 +1827,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
             at[n_at].val.clusterDim.x = 2; at[n_at].val.clusterDim.y = 1; at[n_at].val.clusterDim.z = 1;
             ++n_at;
         }
-        if (a.zw != 0) {
+        {   // early start beside the tail of the previous kernel (fully serial unless that kernel allows dependents)
             at[n_at].id = cudaLaunchAttributeProgrammaticStreamSerialization;
             at[n_at].val.programmaticStreamSerializationAllowed = 1;
             ++n_at;

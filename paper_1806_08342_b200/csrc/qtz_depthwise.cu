@@ -270,8 +270,12 @@ depthwise3x3_kernel(const __grid_constant__ CUtensorMap map_x, const DwArgs a)
         }
         fence_barrier_init();
         prefetch_tensormap(&map_x);
+        grid_launch_dependents();     // the next kernel may be scheduled as this one's blocks leave
     }
     __syncthreads();
+    // started, perhaps, before the previous kernel of the stream has finished (programmatic dependent launch): its
+    // output is this kernel's input, and this kernel's output may alias what it still reads
+    grid_dependency_wait();
 
     if (threadIdx.x < 32) {
         // ---- producer: lane 0 streams tiles into the ring ----
@@ -615,7 +619,19 @@ qtz_status qtz_depthwise_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, uin
     const bool clamp = !(act_min == 0 && act_max == 255);
     const DwKernel kernel = pick_kernel(d.stride, p->w_zp_signed != 0, mode, clamp);
     if (p->ev_start) QTZ_CUDA(p->h, cudaEventRecord(p->ev_start, st));
-    kernel<<<static_cast<unsigned>(p->dw->grid), static_cast<unsigned>(p->dw->threads), p->dw->smem_bytes, st>>>(map, a);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(p->dw->grid));
+        cfg.blockDim = dim3(static_cast<unsigned>(p->dw->threads));
+        cfg.dynamicSmemBytes = p->dw->smem_bytes;
+        cfg.stream = st;
+        cudaLaunchAttribute at;
+        at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &at;
+        cfg.numAttrs = 1;
+        QTZ_CUDA(p->h, cudaLaunchKernelEx(&cfg, kernel, map, a));
+    }
     QTZ_LAUNCH_CHECK(p->h, "depthwise3x3_kernel");
     if (p->ev_stop) QTZ_CUDA(p->h, cudaEventRecord(p->ev_stop, st));
     return QTZ_OK;
