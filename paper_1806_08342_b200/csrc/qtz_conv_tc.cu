@@ -1053,6 +1053,9 @@ pixel_sum_kernel(const uint8_t* __restrict__ x, int64_t pixels, int c, int pitch
     // the convolution that follows needs these sums only in its epilogue: let it start now (its copies and MMAs run
     // beside this kernel; its epilogue waits for this grid before the first read of xsum)
     grid_launch_dependents();
+    // this kernel itself may have started beside the tail of the kernel before it: its input may be that kernel's
+    // output, and xsum may still be read by an earlier launch of the same plan
+    grid_dependency_wait();
     const int warps_per_block = kPrepThreads / 32;
     const int lane = threadIdx.x & 31;
     for (int64_t p = static_cast<int64_t>(blockIdx.x) * warps_per_block + (threadIdx.x >> 5); p < pixels;
@@ -1080,6 +1083,7 @@ __global__ void __launch_bounds__(kPrepThreads)
 stride_gather_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, int batch, int h, int w, int pitch,
                      int stride, int oh, int ow)
 {
+    grid_launch_dependents();      // the convolution launched next may set itself up beside this pre-pass (it waits for it before its first copy)
     const int chunks = pitch >> 4;
     const int64_t t = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
     if (t >= static_cast<int64_t>(batch) * oh * ow * chunks) return;
@@ -1106,6 +1110,7 @@ __global__ void __launch_bounds__(kPrepThreads)
 pad_copy_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ xp, int batch, int h, int w, int c, int hp, int wp,
                 int pad, int zx, int fp)
 {
+    grid_launch_dependents();      // the convolution launched next may set itself up beside this pre-pass (it waits for it before its first copy)
     const int ppc = 16 / fp;                         // pixels per 16-byte chunk
     const int chunks = wp / ppc;                     // wp is a multiple of ppc
     const int xc = blockIdx.x * blockDim.x + threadIdx.x;      // grid: (chunks of a row, frame rows, images)
@@ -1168,6 +1173,7 @@ __global__ void __launch_bounds__(kPrepThreads)
 im2col_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, int h, int w, int c, int cs, int pitch, int kh,
               int kw, int stride, int pad, int oh, int ow, int tp, int k_total, int k_pitch, int zx)
 {
+    grid_launch_dependents();      // the convolution launched next may set itself up beside this pre-pass (it waits for it before its first copy)
     extern __shared__ __align__(16) uint8_t im_s[];
     const int kwords = k_pitch >> 2;
     uint16_t* const off_s = reinterpret_cast<uint16_t*>(im_s);          // [kwords] word offset of output word k in the staged rows
@@ -1673,7 +1679,16 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
         // bracket the two together
         if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
         const int blocks = static_cast<int>(std::min<int64_t>((t->in_pixels + 7) / 8, static_cast<int64_t>(h->num_sms) * 16));
-        pixel_sum_kernel<<<blocks, kPrepThreads, 0, st>>>(xin, t->in_pixels, d.c, d.c_pitch_in, t->xsum);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+        cfg.blockDim = dim3(kPrepThreads);
+        cfg.stream = st;
+        cudaLaunchAttribute at;
+        at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &at;
+        cfg.numAttrs = 1;
+        QTZ_CUDA(h, cudaLaunchKernelEx(&cfg, pixel_sum_kernel, xin, t->in_pixels, static_cast<int>(d.c), static_cast<int>(d.c_pitch_in), t->xsum));
         QTZ_LAUNCH_CHECK(h, "pixel_sum_kernel");
     }
 

@@ -478,3 +478,47 @@ def test_layer_whose_accumulator_can_leave_int32_is_refused(hq):
     assert e.value.code == -4
     ok = hq.conv_create(qtz.conv_desc(1, 2, 2, c, n, 1, 1, 1, 0, outkind=qtz.OUT_S32_RAW), dev(w), dev(bias // 2))
     assert np.array_equal(host(ok(dev(x), 0)), oracle.conv2d_acc(x, 0, w.astype(np.int32), None, bias // 2, 1, 0))
+
+
+def test_back_to_back_layers_on_ping_pong_buffers(hq):
+    """Kernels of consecutive layers are launched as programmatic dependents: a layer's prologue may run while the
+    layer before it is still finishing, but no activation may be read, and no output written, before that layer is
+    done.  Four layers alternate between two buffers (each layer's output overwrites the input of the layer before
+    it) and are enqueued back to back several times; every result must be the oracle's."""
+    b, h, w, c = 32, 40, 40, 64
+    g = synth.rng(1700, 0)
+    x0 = synth.uniform_u8((b, h, w, c), 1700, 1)
+    m, r = oracle.quantize_multiplier(1.0 / 900.0)
+    mult, rsh = np.full(c, m, np.int32), np.full(c, r, np.int32)
+    md, rd = oracle.quantize_multiplier(1.0 / 120.0)
+    multd, rshd = np.full(c, md, np.int32), np.full(c, rd, np.int32)
+    layers, want, cur = [], [], x0
+    for i in range(4):
+        if i % 2 == 0:
+            wq = g.integers(-127, 128, size=(c, 1, 1, c)).astype(np.int8)
+            plan = hq.conv_create(qtz.conv_desc(b, h, w, c, c, 1, 1, 1, 0), dev(wq), None, None, mult, rsh)
+            acc = oracle.conv2d_acc(cur, 0, wq.astype(np.int32), None, None, 1, 0)
+            cur = oracle.requantize(acc, mult, rsh, 0, 0, 255).astype(np.uint8)
+        else:
+            wq = g.integers(-127, 128, size=(3, 3, c)).astype(np.int8)
+            plan = hq.conv_create(qtz.conv_desc(b, h, w, c, c, 3, 3, 1, 1), dev(wq), None, None, multd, rshd, depthwise=True)
+            acc = oracle.depthwise_acc(cur, 0, wq.astype(np.int32), None, None, 1, 1)
+            cur = oracle.requantize(acc, multd, rshd, 0, 0, 255).astype(np.uint8)
+        layers.append(plan)
+        want.append(cur)
+    assert len(np.unique(want[-1])) > 30
+    bufs = [torch.empty((b, h, w, c), dtype=torch.uint8, device="cuda") for _ in range(2)]
+    x_dev = dev(x0)
+    for rep in range(5):
+        bufs[0].copy_(x_dev)
+        outs = []
+        for i, plan in enumerate(layers):                     # buffer 0 -> 1 -> 0 -> 1 -> 0, nothing in between
+            plan(bufs[i % 2], 0, 0, 0, 255, out=bufs[(i + 1) % 2])
+        torch.cuda.synchronize()
+        assert np.array_equal(host(bufs[0]), want[3]), rep      # the last layer wrote buffer 0
+        # and every intermediate, one layer at a time
+        bufs[0].copy_(x_dev)
+        for i, plan in enumerate(layers):
+            plan(bufs[i % 2], 0, 0, 0, 255, out=bufs[(i + 1) % 2])
+            assert np.array_equal(host(bufs[(i + 1) % 2]), want[i]), (rep, i)
+    assert hq.device_status() == (0, 0)
