@@ -291,6 +291,9 @@ def time_hbm_kernels(hq, qtz, torch, peaks):
         res[key]["frac_of_alu_peak"] = round(y.numel() / secs / alu_peak, 3)
         res[key]["sm_mhz"] = mhz
         plan.close()
+    res["requant_alu_probe (outputs per clock and SM)"] = {
+        "three_dp4a": round(hq.probe_requant_rate(0)[0], 2), "multiply_shift_clamp": round(hq.probe_requant_rate(1)[0], 2),
+        "both": round(hq.probe_requant_rate(2)[0], 2), "derived_ceiling_used": round(DW_ALU_OUT_PER_CLK_SM, 2)}
     a = torch.randint(0, 256, (1 << 28,), dtype=torch.uint8, device="cuda").view(-1, 64)
     b = torch.randint(0, 256, (1 << 28,), dtype=torch.uint8, device="cuda").view(-1, 64)
     ma, mb, r = qtz.add_params(0.02, 0.03, 0.04)

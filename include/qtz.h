@@ -115,6 +115,13 @@ QTZ_API qtz_status qtz_selftest_wait_timeout(qtz_handle h, int64_t budget_cycles
 QTZ_API qtz_status qtz_probe_int8_peak(qtz_handle h, int32_t mmas_per_cta, int32_t launches, double* tops_out,
                                        float* ms_out, void* stream);
 
+/* Measures the CUDA cores' rate for the integer arithmetic of an output code, on register operands:
+ * kind 0 three dp4a (the nine taps of a depthwise output); kind 1 one requantisation (32x32->64
+ * multiply-add, shift of the high word, clamp: the y of Eq. 4's rescale); kind 2 both.  Writes outputs
+ * per clock and SM (at the device's maximum SM clock) and, if not NULL, outputs per second.  BLOCKS. */
+QTZ_API qtz_status qtz_probe_requant_rate(qtz_handle h, int32_t kind, double* outputs_per_clock_sm,
+                                          double* outputs_per_second, void* stream);
+
 /* ---- quantizer parameters (Sections 2.1, 2.2, 2.5, 2.6) ------------------------------- */
 
 /* Range estimation by min/max (Section 2.5) followed by parameter derivation.

@@ -5,6 +5,9 @@
 //    tcgen05.mma kind::i8 (M = 128, N = 256, K = 32) back to back into two TMEM accumulators;
 //    nothing is loaded inside the loop, so the figure is the ceiling a u8 x s8 -> s32
 //    contraction (Eq. 5, first term) can reach on this part at the clocks it holds.
+//  * qtz_probe_requant_rate: the rate at which the CUDA cores produce requantised outputs (three dp4a and
+//    one 32x32->64 multiply-shift-clamp each), which is the ceiling of the depthwise kernel and of every
+//    requantising epilogue.
 //  * qtz_selftest_wait_timeout: one CTA waits, with a small cycle budget, on an mbarrier that
 //    nobody ever signals.  The wait gives up by itself, records (QTZ_ERR_DEVICE_TIMEOUT, site)
 //    in the handle's status word and the kernel returns: the path every bounded wait of the
@@ -98,7 +101,92 @@ selftest_wait_kernel(long long budget, int32_t* status)
     if (!done && threadIdx.x == 0 && atomicCAS(status, 0, QTZ_ERR_DEVICE_TIMEOUT) == 0) status[1] = QTZ_SITE_SELFTEST;
 }
 
+// Integer-issue rate of the requantising arithmetic: every thread runs independent chains of
+//   kind 0: three dp4a per output (a depthwise output's nine taps)
+//   kind 1: the 32x32->64 multiply-add, the shift of its high word and the clamp (one requantisation)
+//   kind 2: both (a depthwise output from taps to code)
+// on register operands, eight outputs per loop pass.  Nothing touches memory inside the loop.
+template <int kKind>
+__global__ void __launch_bounds__(256)
+probe_requant_kernel(const uint32_t* __restrict__ seed, int32_t* __restrict__ sink_out, int iters, int32_t m, int sh, long long add64)
+{
+    const int tid = blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t x0 = seed[tid & 255], x1 = seed[(tid + 1) & 255], x2 = seed[(tid + 2) & 255];
+    const uint32_t w0 = seed[(tid + 3) & 255], w1 = seed[(tid + 4) & 255], w2 = seed[(tid + 5) & 255];
+    int32_t sink = 0;
+    for (int it = 0; it < iters; ++it) {
+        int32_t acc[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (kKind != 1) {
+                int32_t d0, d1, d2;
+                asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d0) : "r"(x0 + u), "r"(w0), "r"(0));
+                asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d1) : "r"(x1 + u), "r"(w1), "r"(d0));
+                asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d2) : "r"(x2 + u), "r"(w2), "r"(d1));
+                acc[u] = d2;
+            } else {
+                acc[u] = static_cast<int32_t>(x0 + 77u * u);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            int32_t y = acc[u];
+            if (kKind != 0) {
+                const long long p = static_cast<long long>(acc[u]) * m + add64;
+                y = __vimin_s32_relu(static_cast<int32_t>(p >> 32) >> sh, 255);
+            }
+            sink ^= y;
+        }
+        x0 += sink & 1; x1 += 3; x2 += 5;
+    }
+    sink_out[tid] = sink;
+}
+
 }  // namespace
+
+extern "C" qtz_status qtz_probe_requant_rate(qtz_handle h, int32_t kind, double* outputs_per_clock_sm, double* outputs_per_second,
+                                             void* stream)
+{
+    if (!h || !outputs_per_clock_sm || kind < 0 || kind > 2) return QTZ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    qtz_device_guard guard(h->device);
+    const int blocks = h->num_sms * 8, threads = 256, iters = 4000;
+    qtz_status s = qtz_ensure_reduce(h, sizeof(int32_t) * (static_cast<size_t>(blocks) * threads + 256));
+    if (s != QTZ_OK) return s;
+    uint32_t* seed = reinterpret_cast<uint32_t*>(h->reduce_dev);
+    int32_t* sink = reinterpret_cast<int32_t*>(h->reduce_dev) + 256;
+    uint32_t host_seed[256];
+    for (int i = 0; i < 256; ++i) host_seed[i] = static_cast<uint32_t>(i + 1) * 2654435761u;
+    QTZ_CUDA(h, cudaMemcpyAsync(seed, host_seed, sizeof(host_seed), cudaMemcpyHostToDevice, st));
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    QTZ_CUDA(h, cudaEventCreate(&e0));
+    QTZ_CUDA(h, cudaEventCreate(&e1));
+    const int32_t m = 1518500250;
+    const long long add64 = 1ll << 39;
+    auto launch = [&](int n) {
+        if (kind == 0) probe_requant_kernel<0><<<blocks, threads, 0, st>>>(seed, sink, n, m, 8, add64);
+        else if (kind == 1) probe_requant_kernel<1><<<blocks, threads, 0, st>>>(seed, sink, n, m, 8, add64);
+        else probe_requant_kernel<2><<<blocks, threads, 0, st>>>(seed, sink, n, m, 8, add64);
+    };
+    launch(10);
+    cudaError_t e = cudaEventRecord(e0, st);
+    launch(iters);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaEventRecord(e1, st);
+    if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    int khz = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, h->device);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (e != cudaSuccess) return qtz_cuda_fail(h, e, "probe_requant_kernel");
+    const double outputs = static_cast<double>(blocks) * threads * iters * 8.0;
+    const double per_second = outputs / (static_cast<double>(ms) * 1e-3);
+    if (outputs_per_second) *outputs_per_second = per_second;
+    *outputs_per_clock_sm = per_second / h->num_sms / (static_cast<double>(khz) * 1e3);   // at the maximum SM clock
+    return QTZ_OK;
+}
 
 extern "C" qtz_status qtz_probe_int8_peak(qtz_handle h, int32_t mmas_per_cta, int32_t launches, double* tops_out,
                                           float* ms_out, void* stream)

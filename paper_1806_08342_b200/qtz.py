@@ -52,6 +52,7 @@ SIGNATURES = {
     "qtz_set_wait_budget": (c_int32, [c_void_p, c_int64]),
     "qtz_selftest_wait_timeout": (c_int32, [c_void_p, c_int64, c_void_p]),
     "qtz_probe_int8_peak": (c_int32, [c_void_p, c_int32, c_int32, POINTER(c_double), POINTER(c_float), c_void_p]),
+    "qtz_probe_requant_rate": (c_int32, [c_void_p, c_int32, POINTER(c_double), POINTER(c_double), c_void_p]),
     "qtz_calibrate_minmax": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int32, c_int32, c_void_p,
                                        c_void_p]),
     "qtz_minmax": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_void_p]),
@@ -303,6 +304,12 @@ class Handle:
         self._chk(self.lib.qtz_probe_int8_peak(self.h, int(mmas_per_cta), int(launches), byref(tops), byref(ms), _stream()),
                   "qtz_probe_int8_peak")
         return tops.value, ms.value
+
+    def probe_requant_rate(self, kind):
+        """(outputs per clock and SM at the maximum clock, outputs per second) of the requantising arithmetic."""
+        a, b = c_double(), c_double()
+        self._chk(self.lib.qtz_probe_requant_rate(self.h, int(kind), byref(a), byref(b), _stream()), "qtz_probe_requant_rate")
+        return a.value, b.value
 
     def calibrate_minmax(self, x, axis=None, bits=8, symmetric=False):
         _check_dev(x)

@@ -58,3 +58,15 @@ def test_int8_tensor_core_probe_reports_a_plausible_rate():
     # measurement, anything else means the loop did not do the work it counts
     assert 900.0 < tops < 5200.0, (tops, ms)
     hq.close()
+
+
+def test_requant_rate_probe_orders_its_three_kinds():
+    hq = qtz.Handle(0)
+    taps, _ = hq.probe_requant_rate(0)
+    requant, _ = hq.probe_requant_rate(1)
+    both, per_s = hq.probe_requant_rate(2)
+    # taps and requantisation share one pipe: together they are slower than either, and no faster than their
+    # harmonic sum by more than the loop overhead they share
+    assert both < min(taps, requant) and both > 0.8 / (1.0 / taps + 1.0 / requant), (taps, requant, both)
+    assert 4.0 < both < 20.0 and per_s > 1e12
+    hq.close()
