@@ -20,7 +20,9 @@
  *  - Activations are uint8, NHWC, with a channel pitch: pixel p, channel c lives at
  *    base[p * c_pitch + c].  Pitches are multiples of 16 and base pointers 16-byte
  *    aligned (else QTZ_ERR_MISALIGNED).  Bytes in [c, c_pitch) are never read as data;
- *    outputs leave them unspecified.
+ *    outputs leave them unspecified.  One exception: the INPUT of an image stem (a k x k
+ *    convolution, k > 1, over at most 8 channels with kh*kw*c <= 1024) may have a pitch of 4 or
+ *    8 bytes, so that a 3-channel image need not be stored at 16 bytes per pixel.
  *  - Tensors handed to calibrate / quantize / dequantize are viewed as
  *    x[outer][axis_len][inner] (row-major); one quantizer per index of the middle axis.
  *    axis_len == 1 is per-layer quantization (Section 2.6).

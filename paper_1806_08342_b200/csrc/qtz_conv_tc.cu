@@ -1108,7 +1108,7 @@ stride_gather_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ out, i
 // ever materialised.  No border classes: padding is data.  One thread writes 16 bytes of the frame.
 __global__ void __launch_bounds__(kPrepThreads)
 pad_copy_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ xp, int batch, int h, int w, int c, int hp, int wp,
-                int pad, int zx, int fp)
+                int pad, int zx, int fp, int in_words)
 {
     grid_launch_dependents();      // the convolution launched next may set itself up beside this pre-pass (it waits for it before its first copy)
     const int ppc = 16 / fp;                         // pixels per 16-byte chunk
@@ -1129,7 +1129,7 @@ pad_copy_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ xp, int bat
             const int ix = xc * ppc + j - pad;
             const int live = c - 4 * q;              // real channel bytes in this word
             if (ix < 0 || ix >= w || live <= 0) continue;
-            uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(x) + ((b * h + iy) * w + ix) * 4 + q);   // input pitch: 16 bytes
+            uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(x) + ((b * h + iy) * w + ix) * in_words + q);   // input pitch: 4 in_words bytes
             if (live < 4) {
                 const uint32_t keep = 0xffffffffu >> (8 * (4 - live));
                 v = (v & keep) | (zx4 & ~keep);
@@ -1349,7 +1349,8 @@ int rowwin_run_bytes(const qtz_conv_desc& d)
 bool wants_rowwin(const qtz_conv_desc& d, int w_zp_signed)
 {
     if (is_pointwise(d) || (is_3x3(d) && d.c >= 8)) return false;
-    return d.c_pitch_in == 16 && rowwin_run_bytes(d) != 0 && d.kh <= 16 && d.stride <= 4 && w_zp_signed == 0;
+    return (d.c_pitch_in == 16 || d.c_pitch_in == 8 || d.c_pitch_in == 4) && rowwin_run_bytes(d) != 0 && d.kh <= 16 &&
+           d.stride <= 4 && w_zp_signed == 0;
 }
 
 }  // namespace
@@ -1411,6 +1412,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     t->eff = p->d;
     t->rowwin = wants_rowwin(p->d, p->w_zp_signed);
     t->im2col = !t->rowwin && wants_im2col(p->d);
+    if ((p->d.c_pitch_in & 15) && !t->rowwin && !t->im2col) return QTZ_ERR_MISALIGNED;   // only the repacking paths take narrow pixels
     if (t->im2col) {
         const qtz_conv_desc& o = p->d;
         t->cs = (o.c + 3) / 4 * 4;
@@ -1652,7 +1654,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
         const int threads = std::min(kPrepThreads, (chunks + 31) / 32 * 32);
         pad_copy_kernel<<<dim3(static_cast<unsigned>((chunks + threads - 1) / threads), static_cast<unsigned>(t->hp),
                                static_cast<unsigned>(d.batch)), threads, 0, st>>>(
-            x, p->x_gather, d.batch, d.h, d.w, d.c, t->hp, t->wp, d.pad, x_zp, t->fp);
+            x, p->x_gather, d.batch, d.h, d.w, d.c, t->hp, t->wp, d.pad, x_zp, t->fp, d.c_pitch_in / 4);
         QTZ_LAUNCH_CHECK(h, "pad_copy_kernel");
         xin = p->x_gather;
     } else if (t->im2col) {

@@ -76,7 +76,9 @@ qtz_status validate_desc(const qtz_conv_desc& d, int depthwise)
         return QTZ_ERR_INVALID_ARG;
     if (d.wkind < QTZ_W_S8_PER_CHANNEL_SYM || d.wkind > QTZ_W_S4_PACKED_PER_CHANNEL_SYM) return QTZ_ERR_INVALID_ARG;
     if (d.outkind != QTZ_OUT_U8 && d.outkind != QTZ_OUT_S32_RAW) return QTZ_ERR_INVALID_ARG;
-    if (d.c_pitch_in & 15) return QTZ_ERR_MISALIGNED;
+    // (image tensors of up to 8 channels may come at a pixel pitch of 4 or 8 bytes: the stem paths repack them anyway)
+    const bool narrow_image = !depthwise && (d.c_pitch_in == 4 || d.c_pitch_in == 8) && !(d.kh == 1 && d.kw == 1);
+    if ((d.c_pitch_in & 15) && !narrow_image) return QTZ_ERR_MISALIGNED;
     if (d.outkind == QTZ_OUT_U8) {
         if (d.c_pitch_out < d.n) return QTZ_ERR_INVALID_ARG;
         if (d.c_pitch_out & 15) return QTZ_ERR_MISALIGNED;
@@ -242,6 +244,10 @@ extern "C" qtz_status qtz_conv_create(qtz_handle h, const qtz_conv_desc* desc, i
             return s;
         }
     } else {
+        if (d.c_pitch_in & 15) {                     // the direct path reads whole 16-byte channel groups
+            qtz_conv_destroy(p);
+            return QTZ_ERR_MISALIGNED;
+        }
         p->family = QTZ_K_DIRECT;
         p->k_padded = (p->k_total + 15) & ~15;
         p->n_padded = (d.n + 63) & ~63;

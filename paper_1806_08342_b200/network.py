@@ -69,7 +69,7 @@ class QuantizedNetwork:
         h = self.h
         batch = images_u8.shape[0]
         self.batch = batch
-        x0 = np.zeros(images_u8.shape[:3] + (16,), np.uint8)
+        x0 = np.zeros(images_u8.shape[:3] + (4,), np.uint8)          # images at 4 bytes per pixel (the stem repacks them)
         x0[..., :3] = images_u8
         tensors = {"in": torch.from_numpy(x0).cuda()}
         chans = {"in": 3}

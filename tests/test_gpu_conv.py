@@ -28,9 +28,9 @@ def make_weights(wkind, shape, seed):
 
 
 def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=0, expect_kernel=None, real_m=None, bias_range=20000,
-              expect_detail=None):
+              expect_detail=None, in_pitch=None):
     x = synth.uniform_u8((b, h, w, c), seed, 1)
-    xp = pitched(x)
+    xp = pitched(x, in_pitch)
     api_w, codes, zw = make_weights(wkind, (n, k, k, c), seed)
     if wkind == qtz.W_S4_PACKED_PER_CHANNEL_SYM:
         api_w = oracle.pack_s4(codes.reshape(n, -1))
@@ -39,7 +39,7 @@ def conv_case(hq, b, h, w, c, n, k, stride, pad, wkind, seed, raw=False, act=0, 
     z_x = int(g.integers(64, 192))
     z_w = None if zw is None else np.full(n, zw, np.int32)
     acc = oracle.conv2d_acc(xp, z_x, codes, z_w, bias, stride, pad, c=c)
-    desc = qtz.conv_desc(b, h, w, c, n, k, k, stride, pad, wkind, qtz.OUT_S32_RAW if raw else qtz.OUT_U8)
+    desc = qtz.conv_desc(b, h, w, c, n, k, k, stride, pad, wkind, qtz.OUT_S32_RAW if raw else qtz.OUT_U8, c_pitch_in=in_pitch)
     if raw:
         plan = hq.conv_create(desc, dev(api_w), dev(bias), zw)
         got = host(plan(dev(xp), z_x))
@@ -522,3 +522,28 @@ def test_back_to_back_layers_on_ping_pong_buffers(hq):
             plan(bufs[i % 2], 0, 0, 0, 255, out=bufs[(i + 1) % 2])
             assert np.array_equal(host(bufs[(i + 1) % 2]), want[i]), (rep, i)
     assert hq.device_status() == (0, 0)
+
+
+@pytest.mark.parametrize("case", [
+    # b, h, w, c, n, k, stride, weight kind, input pitch, expected form
+    (2, 64, 64, 3, 32, 3, 2, qtz.W_S8_PER_CHANNEL_SYM, 4, "row-window"),      # MobileNet stem, images at 4 bytes per pixel
+    (2, 60, 60, 3, 64, 7, 2, qtz.W_S8_PER_CHANNEL_SYM, 4, "row-window"),      # ResNet stem
+    (1, 33, 31, 3, 48, 3, 2, qtz.W_S4_PACKED_PER_CHANNEL_SYM, 4, "row-window"),
+    (2, 30, 30, 6, 24, 3, 2, qtz.W_S8_PER_CHANNEL_SYM, 8, "row-window"),      # 8-byte pixels
+    (2, 30, 30, 3, 24, 3, 2, qtz.W_U8_PER_LAYER_ASYM, 4, "im2col"),           # asymmetric weights: explicit im2col
+    (1, 20, 20, 4, 16, 5, 1, qtz.W_S8_PER_CHANNEL_SYM, 4, "row-window"),      # stride 1: 16-byte frame pixels
+])
+def test_image_stems_take_narrow_pixel_pitches(hq, case):
+    b, h, w, c, n, k, stride, wkind, pitch, form = case
+    conv_case(hq, b, h, w, c, n, k, stride, k // 2, wkind, 1800 + c + n + k, expect_kernel="tcgen05", expect_detail=form, in_pitch=pitch)
+    conv_case(hq, b, h, w, c, n, k, stride, k // 2, wkind, 1900 + c + n + k, raw=True, in_pitch=pitch)
+
+
+def test_narrow_pixel_pitch_is_refused_elsewhere(hq):
+    m, r = oracle.quantize_multiplier(0.01)
+    for args, dw in [((1, 8, 8, 4, 16, 1, 1, 1, 0), False), ((1, 8, 8, 8, 8, 3, 3, 1, 1), True)]:
+        w = dev(synth.uniform_s8((3, 3, 8) if dw else (16, 1, 1, 4), 1990, 0))
+        n = args[4]
+        with pytest.raises(qtz.QtzError) as e:
+            hq.conv_create(qtz.conv_desc(*args, c_pitch_in=args[3]), w, None, None, np.full(n, m, np.int32), np.full(n, r, np.int32), depthwise=dw)
+        assert e.value.code == -2
