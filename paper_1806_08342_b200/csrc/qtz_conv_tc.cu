@@ -1062,9 +1062,8 @@ pixel_sum_kernel(const uint8_t* __restrict__ x, int64_t pixels, int c, int pitch
          p += static_cast<int64_t>(gridDim.x) * warps_per_block) {
         const uint8_t* row = x + p * pitch;
         uint32_t s = 0;
-        for (int off = lane * 16; off < c; off += 32 * 16) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(row + off));
-            uint32_t words[4] = {v.x, v.y, v.z, v.w};
+        auto take = [&](const uint4& v, int off) {
+            const uint32_t words[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int first = off + 4 * i;
@@ -1072,7 +1071,17 @@ pixel_sum_kernel(const uint8_t* __restrict__ x, int64_t pixels, int c, int pitch
                 if (first + 4 > c) word = first >= c ? 0u : (word & (0xffffffffu >> (8 * (first + 4 - c))));
                 s = __dp4a(word, 0x01010101u, s);
             }
+        };
+        int off = lane * 16;
+        // four 16-byte loads of a lane in flight at a time (2 KB of the row per warp and step)
+        for (; off + 3 * 512 < c; off += 4 * 512) {
+            const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(row + off));
+            const uint4 v1 = __ldg(reinterpret_cast<const uint4*>(row + off + 512));
+            const uint4 v2 = __ldg(reinterpret_cast<const uint4*>(row + off + 1024));
+            const uint4 v3 = __ldg(reinterpret_cast<const uint4*>(row + off + 1536));
+            take(v0, off); take(v1, off + 512); take(v2, off + 1024); take(v3, off + 1536);
         }
+        for (; off < c; off += 512) take(__ldg(reinterpret_cast<const uint4*>(row + off)), off);
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
         if (lane == 0) xsum[p] = static_cast<int32_t>(s);
     }
