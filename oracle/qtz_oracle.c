@@ -71,7 +71,7 @@ int orc_minmax(const float* x, int64_t outer, int64_t axis_len, int64_t inner,
 /* ------------------------------------------------------------------------- */
 int orc_affine_params(float lo, float hi, int bits, orc_qparams* q)
 {
-    if (bits < 2 || bits > 8) return ORC_ERR_INVALID;
+    if (bits < 2 || bits > 16) return ORC_ERR_INVALID;   /* Section 7: 4, 8 and 16 bits */
     if (!isfinite(lo) || !isfinite(hi)) return ORC_ERR_NONFINITE;
     if (lo > hi) return ORC_ERR_INVALID;
     if (lo > 0.0f) lo = 0.0f;
@@ -101,7 +101,7 @@ int orc_affine_params(float lo, float hi, int bits, orc_qparams* q)
 /* All-zero channel: Delta = 1.                                                */
 int orc_symmetric_params(float lo, float hi, int bits, orc_qparams* q)
 {
-    if (bits < 2 || bits > 8) return ORC_ERR_INVALID;
+    if (bits < 2 || bits > 16) return ORC_ERR_INVALID;   /* Section 7: 4, 8 and 16 bits */
     if (!isfinite(lo) || !isfinite(hi)) return ORC_ERR_NONFINITE;
     float a = fabsf(lo) > fabsf(hi) ? fabsf(lo) : fabsf(hi);
     const int P = (1 << (bits - 1)) - 1;
@@ -133,7 +133,7 @@ int orc_calibrate_minmax(const float* x, int64_t outer, int64_t axis_len, int64_
 /* symmetric), Eq. 10 (signed symmetric with the restricted range).            */
 int orc_code_range(int bits, int is_signed, int restrict_range, int32_t* qmin, int32_t* qmax)
 {
-    if (bits < 2 || bits > 8) return ORC_ERR_INVALID;
+    if (bits < 2 || bits > 16) return ORC_ERR_INVALID;   /* Section 7: 4, 8 and 16 bits */
     if (is_signed) {
         *qmax = (1 << (bits - 1)) - 1;
         *qmin = restrict_range ? -*qmax : -(1 << (bits - 1));

@@ -67,7 +67,7 @@ def test_sqnr_hand_computed():
     assert abs(oracle.sqnr(4 * w, 4 * wh)[0] - oracle.sqnr(w, wh)[0]) < 1e-12
 
 
-@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("bits", [4, 8, 16])
 def test_sqnr_of_a_uniform_signal_is_the_textbook_value(bits):
     # uniform on [0, R] quantized over exactly that range: noise power Delta^2 / 12, signal power R^2 / 3,
     # so SQNR = 20 log10(2 (2^b - 1))  (about 6.02 dB per bit)
