@@ -261,7 +261,11 @@ def time_hbm_kernels(hq, qtz, torch, peaks):
     entry("dequantize_u8_to_f32 (5 B/elem)", timed(lambda: hq.dequantize(q, p, out=x)), 5.0 * n)
     y = torch.empty_like(x)
     entry("simquant_f32 (8 B/elem)", timed(lambda: hq.simquant(x, p, out=y)), 8.0 * n)
-    del x, q, y
+    p16 = hq.calibrate_minmax(x, bits=16)
+    q16 = hq.quantize_tensor(x, p16, out_dtype=qtz.U16)
+    entry("quantize_f32_to_u16 (6 B/elem)", timed(lambda: hq.quantize_tensor(x, p16, out_dtype=qtz.U16, out=q16)), 6.0 * n)
+    entry("dequantize_u16_to_f32 (6 B/elem)", timed(lambda: hq.dequantize(q16, p16, out=y)), 6.0 * n)
+    del x, q, y, q16
     # MobileNet-v1 depthwise layers at batch 128: (H, C, stride, zero points and clamp).  "ranged": z_x = 3,
     # z_y = 10, clamp [10,255] (border cells refilled with z_x, explicit clamp); "relu6": the case between two
     # ReLU6 tensors, z_x = z_y = 0 and the whole byte as the range.  At stride 1 the kernel is bound by integer

@@ -65,7 +65,10 @@ typedef struct {
     float max_nudged;   /* real value of the highest code, (L - z) * Delta  */
 } qtz_qparams;
 
-typedef enum { QTZ_U8 = 0, QTZ_S8 = 1, QTZ_S4_PACKED = 2, QTZ_S32 = 3, QTZ_U4_PACKED = 4 } qtz_dtype;
+typedef enum {
+    QTZ_U8 = 0, QTZ_S8 = 1, QTZ_S4_PACKED = 2, QTZ_S32 = 3, QTZ_U4_PACKED = 4,
+    QTZ_U16 = 5, QTZ_S16 = 6   /* 16-bit codes (Section 7: 4, 8 and 16 bits), stored as uint16_t / int16_t */
+} qtz_dtype;
 
 typedef enum {
     QTZ_W_S8_PER_CHANNEL_SYM = 0,       /* int8 codes, one scale per output channel, z_w = 0 */
@@ -133,7 +136,7 @@ QTZ_API qtz_status qtz_probe_requant_rate(qtz_handle h, int32_t kind, double* ou
  * Symmetric (Section 2.2): z = 0, Delta = max|x| / (2^(bits-1) - 1).
  * A tensor (or channel) that is all zero gets Delta = 1, z = 0.
  * Reads x_dev (fp32, device, outer*axis_len*inner values), writes axis_len entries to
- * out_host.  BLOCKS until `stream` has finished.  bits in [2,8].
+ * out_host.  BLOCKS until `stream` has finished.  bits in [2,16].
  * Errors: QTZ_ERR_NONFINITE if any value is NaN/Inf (out_host is then unspecified).       */
 QTZ_API qtz_status qtz_calibrate_minmax(qtz_handle h, const float* x_dev, int64_t outer,
                                 int64_t axis_len, int64_t inner, int32_t bits,
@@ -209,7 +212,11 @@ QTZ_API qtz_status qtz_params_from_range(float lo, float hi, int32_t bits, int32
  * The quotient is one IEEE fp32 division and round() is round-half-to-even.  Code ranges:
  *   QTZ_U8 [0,255] (restrict_range: [0,254]); QTZ_S8 [-128,127] (restrict_range, Eq. 10:
  *   [-127,127]); QTZ_S4_PACKED [-8,7] (restrict_range: [-7,7]); QTZ_U4_PACKED [0,15]
- *   (restrict_range: [0,14]) -- 4-bit activations, Section 3.2.4.
+ *   (restrict_range: [0,14]) -- 4-bit activations, Section 3.2.4; QTZ_U16 [0,65535] (restrict_range:
+ *   [0,65534]) and QTZ_S16 [-32768,32767] (restrict_range: [-32767,32767]) -- the 16-bit precision of
+ *   Section 7, two bytes per code, q_dev 2-byte aligned.  (fp32 holds every 16-bit code exactly; the
+ *   quotient x / Delta is then good to 2^-8 of a step, so a value within that distance of a tie may
+ *   round either way against exact arithmetic, never against these fp32 steps.)
  * NaN maps to the lowest code, +-Inf saturate.
  * params_host: axis_len entries, read before the call returns.
  * QTZ_S4_PACKED / QTZ_U4_PACKED: nibbles (two's complement / unsigned) packed along the innermost run of the view
@@ -233,7 +240,7 @@ QTZ_API qtz_status qtz_dequantize(qtz_handle h, const void* q_dev, int32_t in_dt
  *   y = (clamp(round(x / Delta) + z, qmin, qmax) - z) * Delta
  * with exactly the fp32 steps of qtz_quantize_tensor and qtz_dequantize (the paper prints the
  * formula with the sign of z flipped; this is Eq. 3 applied to Eq. 1-2).  fp32 in, fp32 out,
- * same view and parameter conventions; code_dtype (QTZ_U8 / QTZ_S8 / QTZ_S4_PACKED) and
+ * same view and parameter conventions; code_dtype (any qtz_dtype but QTZ_S32) and
  * restrict_range only select the code range [qmin, qmax].  y_dev may alias x_dev.           */
 QTZ_API qtz_status qtz_simquant(qtz_handle h, const float* x_dev, int64_t outer, int64_t axis_len,
                                 int64_t inner, const qtz_qparams* params_host, int32_t code_dtype,

@@ -137,6 +137,38 @@ quantize_flat_kernel(const float* __restrict__ x, int64_t n, QuantRule q, uint8_
     }
 }
 
+// Per-layer, 16-bit output (uint16 or int16 share the low half word): 8 values per thread,
+// 2 x 16-byte loads and one 16-byte store.  Needs both pointers 16-byte aligned.
+__global__ void __launch_bounds__(kThreads)
+quantize_flat16_kernel(const float* __restrict__ x, int64_t n, QuantRule q, uint16_t* __restrict__ out)
+{
+    const int64_t groups = n >> 3;
+    const int64_t g = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+    if (g < groups) {
+        const float4* xv = reinterpret_cast<const float4*>(x) + 2 * g;
+        const float4 a = __ldcs(xv), b = __ldcs(xv + 1);
+        auto two = [&](float lo, float hi) {
+            return (static_cast<uint32_t>(quant1(lo, q)) & 0xffffu) | (static_cast<uint32_t>(quant1(hi, q)) << 16);
+        };
+        uint4 o;
+        o.x = two(a.x, a.y); o.y = two(a.z, a.w); o.z = two(b.x, b.y); o.w = two(b.z, b.w);
+        reinterpret_cast<uint4*>(out)[g] = o;
+    } else if (g == groups) {
+        for (int64_t i = groups << 3; i < n; ++i) out[i] = static_cast<uint16_t>(quant1(x[i], q));
+    }
+}
+
+// Any view, 16-bit output: one value per thread.
+__global__ void __launch_bounds__(kThreads)
+quantize_axis16_kernel(const float* __restrict__ x, int64_t total, int64_t axis_len, int64_t inner,
+                       const QuantRule* __restrict__ rules, uint16_t* __restrict__ out)
+{
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+    if (i >= total) return;
+    const int64_t a = (i / inner) % axis_len;
+    out[i] = static_cast<uint16_t>(quant1(x[i], rules[a]));
+}
+
 // Any view, byte output: one value per thread, the rule fetched per axis index.
 __global__ void __launch_bounds__(kThreads)
 quantize_axis_kernel(const float* __restrict__ x, int64_t total, int64_t axis_len, int64_t inner,
@@ -211,6 +243,27 @@ dequantize_flat_kernel(const uint8_t* __restrict__ q, int64_t n, DequantRule rul
     }
 }
 
+// Per-layer 16-bit codes: 8 values per thread (one 16-byte load, two 16-byte stores).
+template <bool kSigned>
+__global__ void __launch_bounds__(kThreads)
+dequantize_flat16_kernel(const uint16_t* __restrict__ q, int64_t n, DequantRule rule, float* __restrict__ x)
+{
+    const int64_t groups = n >> 3;
+    const int64_t g = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+    auto one = [&](uint32_t half) {
+        const int32_t c = kSigned ? static_cast<int32_t>(static_cast<int16_t>(half)) : static_cast<int32_t>(half & 0xffffu);
+        return __fmul_rn(static_cast<float>(c - rule.zp), rule.scale);
+    };
+    if (g < groups) {
+        const uint4 v = __ldcs(reinterpret_cast<const uint4*>(q) + g);
+        float4* xv = reinterpret_cast<float4*>(x) + 2 * g;
+        __stcs(xv, make_float4(one(v.x), one(v.x >> 16), one(v.y), one(v.y >> 16)));
+        __stcs(xv + 1, make_float4(one(v.z), one(v.z >> 16), one(v.w), one(v.w >> 16)));
+    } else if (g == groups) {
+        for (int64_t i = groups << 3; i < n; ++i) x[i] = one(q[i]);
+    }
+}
+
 // Any view and any code type: one value per thread.
 __global__ void __launch_bounds__(kThreads)
 dequantize_axis_kernel(const void* __restrict__ q, int32_t dtype, int64_t total, int64_t axis_len,
@@ -227,6 +280,10 @@ dequantize_axis_kernel(const void* __restrict__ q, int32_t dtype, int64_t total,
         code = static_cast<const int8_t*>(q)[i];
     } else if (dtype == QTZ_S32) {
         code = static_cast<const int32_t*>(q)[i];
+    } else if (dtype == QTZ_U16) {
+        code = static_cast<const uint16_t*>(q)[i];
+    } else if (dtype == QTZ_S16) {
+        code = static_cast<const int16_t*>(q)[i];
     } else {  // packed 4-bit: locate the byte inside the element's run
         const int64_t run = i / run_len, e = i - run * run_len;
         const uint32_t byte = static_cast<const uint8_t*>(q)[run * ((run_len + 1) >> 1) + (e >> 1)];
@@ -415,7 +472,7 @@ extern "C" qtz_status qtz_range_finish(qtz_handle h, const void* state_dev, int6
                                        void* stream)
 {
     if (!h || !state_dev || qtz_range_state_bytes(axis_len) == 0) return QTZ_ERR_INVALID_ARG;
-    if (params_host && (bits < 2 || bits > 8)) return QTZ_ERR_INVALID_ARG;
+    if (params_host && (bits < 2 || bits > 16)) return QTZ_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t bytes = static_cast<size_t>(qtz_range_state_bytes(axis_len));
     std::vector<char> host(bytes);
@@ -447,7 +504,7 @@ extern "C" qtz_status qtz_calibrate_minmax(qtz_handle h, const float* x_dev, int
     if (!h) return QTZ_ERR_INVALID_ARG;
     qtz_status s = check_view(x_dev, out_host, outer, axis_len, inner);
     if (s != QTZ_OK) return s;
-    if (bits < 2 || bits > 8) return QTZ_ERR_INVALID_ARG;
+    if (bits < 2 || bits > 16) return QTZ_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(x_dev) & 3u) return QTZ_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     s = launch_minmax(h, x_dev, outer, axis_len, inner, st);
@@ -488,7 +545,16 @@ extern "C" qtz_status qtz_quantize_tensor(qtz_handle h, const float* x_dev, int6
                              static_cast<float>(qmax - p.zero_point), p.zero_point};
     }
     const bool packed4 = out_dtype == QTZ_S4_PACKED || out_dtype == QTZ_U4_PACKED;
-    if (axis_len == 1 && !packed4 && qtz_aligned16(x_dev) && qtz_aligned16(q_dev)) {
+    const bool wide = out_dtype == QTZ_U16 || out_dtype == QTZ_S16;
+    if (wide && (reinterpret_cast<uintptr_t>(q_dev) & 1u)) return QTZ_ERR_MISALIGNED;
+    if (axis_len == 1 && wide && qtz_aligned16(x_dev) && qtz_aligned16(q_dev)) {
+        const int64_t groups = (total >> 3) + 1;
+        quantize_flat16_kernel<<<static_cast<unsigned>(ceil_div(groups, kThreads)), kThreads, 0, st>>>(
+            x_dev, total, rules[0], static_cast<uint16_t*>(q_dev));
+        QTZ_LAUNCH_CHECK(h, "quantize_flat16_kernel");
+        return QTZ_OK;
+    }
+    if (axis_len == 1 && !packed4 && !wide && qtz_aligned16(x_dev) && qtz_aligned16(q_dev)) {
         const int64_t groups = (total >> 4) + 1;
         quantize_flat_kernel<<<static_cast<unsigned>(ceil_div(groups, kThreads)), kThreads, 0, st>>>(
             x_dev, total, rules[0], static_cast<uint8_t*>(q_dev));
@@ -507,6 +573,10 @@ extern "C" qtz_status qtz_quantize_tensor(qtz_handle h, const float* x_dev, int6
         quantize_s4_kernel<<<static_cast<unsigned>(ceil_div(work, kThreads)), kThreads, 0, st>>>(
             x_dev, runs, run_len, axis_len, inner, rules_dev, static_cast<uint8_t*>(q_dev));
         QTZ_LAUNCH_CHECK(h, "quantize_s4_kernel");
+    } else if (wide) {
+        quantize_axis16_kernel<<<static_cast<unsigned>(ceil_div(total, kThreads)), kThreads, 0, st>>>(
+            x_dev, total, axis_len, inner, rules_dev, static_cast<uint16_t*>(q_dev));
+        QTZ_LAUNCH_CHECK(h, "quantize_axis16_kernel");
     } else {
         quantize_axis_kernel<<<static_cast<unsigned>(ceil_div(total, kThreads)), kThreads, 0, st>>>(
             x_dev, total, axis_len, inner, rules_dev, static_cast<uint8_t*>(q_dev));
@@ -524,8 +594,10 @@ extern "C" qtz_status qtz_dequantize(qtz_handle h, const void* q_dev, int32_t in
     if (!h || !params_host) return QTZ_ERR_INVALID_ARG;
     qtz_status s = check_view(q_dev, x_dev, outer, axis_len, inner);
     if (s != QTZ_OK) return s;
-    if (in_dtype < QTZ_U8 || in_dtype > QTZ_U4_PACKED) return QTZ_ERR_INVALID_ARG;
+    if (in_dtype < QTZ_U8 || in_dtype > QTZ_S16) return QTZ_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(x_dev) & 3u) return QTZ_ERR_MISALIGNED;
+    const bool wide = in_dtype == QTZ_U16 || in_dtype == QTZ_S16;
+    if (wide && (reinterpret_cast<uintptr_t>(q_dev) & 1u)) return QTZ_ERR_MISALIGNED;
     if (in_dtype == QTZ_S32 && (reinterpret_cast<uintptr_t>(q_dev) & 3u)) return QTZ_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t total = outer * axis_len * inner;
@@ -542,6 +614,16 @@ extern "C" qtz_status qtz_dequantize(qtz_handle h, const void* q_dev, int32_t in
         else
             dequantize_flat_kernel<false><<<blocks, kThreads, 0, st>>>(static_cast<const uint8_t*>(q_dev), total, rules[0], x_dev);
         QTZ_LAUNCH_CHECK(h, "dequantize_flat_kernel");
+        return QTZ_OK;
+    }
+    if (axis_len == 1 && wide && qtz_aligned16(q_dev) && qtz_aligned16(x_dev)) {
+        const int64_t groups = (total >> 3) + 1;
+        const unsigned blocks = static_cast<unsigned>(ceil_div(groups, kThreads));
+        if (in_dtype == QTZ_S16)
+            dequantize_flat16_kernel<true><<<blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(q_dev), total, rules[0], x_dev);
+        else
+            dequantize_flat16_kernel<false><<<blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(q_dev), total, rules[0], x_dev);
+        QTZ_LAUNCH_CHECK(h, "dequantize_flat16_kernel");
         return QTZ_OK;
     }
     const size_t bytes = sizeof(DequantRule) * rules.size();

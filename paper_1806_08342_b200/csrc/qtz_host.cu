@@ -121,7 +121,7 @@ qtz_status qtz_ensure_reduce(qtz_ctx* h, size_t bytes)
 // zero point is the (integer) code that real 0 falls on.
 qtz_status qtz_host_affine_params(float lo, float hi, int bits, qtz_qparams* q)
 {
-    if (!q || bits < 2 || bits > 8) return QTZ_ERR_INVALID_ARG;
+    if (!q || bits < 2 || bits > 16) return QTZ_ERR_INVALID_ARG;
     if (!std::isfinite(lo) || !std::isfinite(hi)) return QTZ_ERR_NONFINITE;
     if (hi < lo) return QTZ_ERR_INVALID_ARG;
     const double levels = static_cast<double>((1 << bits) - 1);
@@ -145,7 +145,7 @@ qtz_status qtz_host_affine_params(float lo, float hi, int bits, qtz_qparams* q)
 // Section 2.2: zero point fixed at 0, the largest magnitude maps to the top positive code.
 qtz_status qtz_host_symmetric_params(float lo, float hi, int bits, qtz_qparams* q)
 {
-    if (!q || bits < 2 || bits > 8) return QTZ_ERR_INVALID_ARG;
+    if (!q || bits < 2 || bits > 16) return QTZ_ERR_INVALID_ARG;
     if (!std::isfinite(lo) || !std::isfinite(hi)) return QTZ_ERR_NONFINITE;
     const int top = (1 << (bits - 1)) - 1;
     const float amax = std::fmax(std::fabs(lo), std::fabs(hi));
@@ -172,6 +172,8 @@ bool qtz_code_range(int32_t dtype, int32_t restrict_range, int32_t* qmin, int32_
         case QTZ_S8: *qmin = restrict_range ? -127 : -128; *qmax = 127; return true;
         case QTZ_S4_PACKED: *qmin = restrict_range ? -7 : -8; *qmax = 7; return true;
         case QTZ_U4_PACKED: *qmin = 0; *qmax = restrict_range ? 14 : 15; return true;
+        case QTZ_U16: *qmin = 0; *qmax = restrict_range ? 65534 : 65535; return true;
+        case QTZ_S16: *qmin = restrict_range ? -32767 : -32768; *qmax = 32767; return true;
         default: return false;
     }
 }

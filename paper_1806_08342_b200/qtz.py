@@ -17,7 +17,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libqtz.so")
 
-U8, S8, S4_PACKED, S32, U4_PACKED = 0, 1, 2, 3, 4
+U8, S8, S4_PACKED, S32, U4_PACKED, U16, S16 = 0, 1, 2, 3, 4, 5, 6
 W_S8_PER_CHANNEL_SYM, W_U8_PER_LAYER_ASYM, W_S4_PACKED_PER_CHANNEL_SYM = 0, 1, 2
 OUT_U8, OUT_S32_RAW = 0, 1
 ACT_NONE, ACT_RELU, ACT_RELU6 = 0, 1, 2
@@ -364,7 +364,8 @@ class Handle:
                 run = i if i > 1 else a
                 out = torch.empty((x.numel() // run) * ((run + 1) // 2), dtype=torch.uint8, device=x.device)
             else:
-                out = torch.empty(x.shape, dtype=torch.uint8 if out_dtype == U8 else torch.int8, device=x.device)
+                out = torch.empty(x.shape, dtype={U8: torch.uint8, S8: torch.int8, U16: torch.uint16, S16: torch.int16}[out_dtype],
+                                  device=x.device)
         self._chk(self.lib.qtz_quantize_tensor(self.h, _ptr(x), o, a, i, _np(params), out_dtype,
                                                int(restrict_range), _ptr(out), _stream()), "qtz_quantize_tensor")
         return out
@@ -372,7 +373,8 @@ class Handle:
     def dequantize(self, q, params, axis=None, in_dtype=None, shape=None, out=None):
         _check_dev(q, out)
         if in_dtype is None:
-            in_dtype = {torch.uint8: U8, torch.int8: S8, torch.int32: S32}[q.dtype]   # packed 4-bit: pass in_dtype
+            in_dtype = {torch.uint8: U8, torch.int8: S8, torch.int32: S32, torch.uint16: U16,
+                        torch.int16: S16}[q.dtype]                                    # packed 4-bit: pass in_dtype
         shape = tuple(q.shape) if shape is None else tuple(shape)
         params = np.ascontiguousarray(np.atleast_1d(params), dtype=QPARAMS)
         o, a, i = _view(shape, axis)

@@ -79,7 +79,7 @@ def test_params_from_range_matches_oracle(qtz):
         lo = float(np.float32(g.normal() * 10 ** g.uniform(-4, 4)))
         cases.append((lo, float(np.float32(lo + abs(g.normal()) * 10 ** g.uniform(-4, 4)))))
     for lo, hi in cases:
-        for bits in (4, 8):
+        for bits in (4, 8, 16):
             a, b = qtz.params_from_range(lo, hi, bits, False), oracle.affine_params(lo, hi, bits)
             assert a.tobytes() == b.tobytes(), (lo, hi, bits, a, b)
             a, b = qtz.params_from_range(lo, hi, bits, True), oracle.symmetric_params(lo, hi, bits)

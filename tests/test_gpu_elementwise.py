@@ -194,7 +194,7 @@ def test_argument_errors(hq):
     pp = p.ctypes.data
     assert lib.qtz_calibrate_minmax(h, None, 1, 1, 64, 8, 0, pp, None) == -1
     assert lib.qtz_calibrate_minmax(h, x.data_ptr(), 1, 1, 0, 8, 0, pp, None) == -1
-    assert lib.qtz_calibrate_minmax(h, x.data_ptr(), 1, 1, 64, 9, 0, pp, None) == -1
+    assert lib.qtz_calibrate_minmax(h, x.data_ptr(), 1, 1, 64, 17, 0, pp, None) == -1     # bits in [2,16]
     assert lib.qtz_quantize_tensor(h, x.data_ptr(), 1, 1, 64, pp, 7, 0, out.data_ptr(), None) == -1
     assert lib.qtz_quantize_tensor(h, x.data_ptr() + 2, 1, 1, 32, pp, 0, 0, out.data_ptr(), None) == -2
     p["scale"] = 0.0
