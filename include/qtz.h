@@ -416,6 +416,21 @@ typedef struct {
 QTZ_API qtz_status qtz_conv2d_add_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point,
                                      const qtz_residual* r_host, const uint8_t* s_dev, void* y_dev,
                                      int32_t y_zero_point, int32_t act_min, int32_t act_max, void* stream);
+/* A depthwise-separable block in one kernel (Section 7 recommends fusing operators): the 3x3 depthwise
+ * plan `dw` followed by the pointwise plan `pw`, whose input is the depthwise output.  Computes exactly
+ * what qtz_depthwise_u8 (output zero point mid_zero_point, clamp [mid_act_min, mid_act_max]) followed by
+ * qtz_conv2d_u8 (input zero point mid_zero_point) computes, bit for bit; the intermediate tensor is
+ * produced chunk of channels by chunk of channels in shared memory, as the activation operand of the
+ * tensor cores, and never stored.  x_dev follows the geometry of `dw`, y_dev that of `pw`.
+ * Errors: QTZ_ERR_INVALID_ARG when the plans do not chain (channels, batch, extent); QTZ_ERR_UNSUPPORTED
+ * when this pair cannot run fused -- run the two calls separately then.  Fused are: symmetric int8
+ * weights on both layers, depthwise stride 1 or 2 with right shifts 32..53, a stride-1 pointwise layer on
+ * the tensor-core path with at most 256 output channels whose 8-bit weights fit in shared memory
+ * (channels x outputs <= 80 KB).                                                                    */
+QTZ_API qtz_status qtz_conv2d_dw_pw_u8(qtz_conv_plan dw, qtz_conv_plan pw, const uint8_t* x_dev, int32_t x_zero_point,
+                                       int32_t mid_zero_point, int32_t mid_act_min, int32_t mid_act_max, void* y_dev,
+                                       int32_t y_zero_point, int32_t act_min, int32_t act_max, void* stream);
+
 /* Depthwise form of the same (depth multiplier 1; Section 3.1.3 networks): the sum runs over
  * the kh x kw taps of one channel.  Plan must have been created with depthwise != 0.           */
 QTZ_API qtz_status qtz_depthwise_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point,

@@ -35,6 +35,7 @@
 
 #include "qtz_add_math.cuh"
 #include "qtz_device_util.cuh"
+#include "qtz_dw_math.cuh"
 #include "qtz_plan.cuh"
 #include "qtz_ptx.cuh"
 
@@ -51,7 +52,9 @@ constexpr int kStoreWarp = 2 + kEpiWarps;            // its lane g issues the ou
 constexpr int kThreadsTc = 32 * (kStoreWarp + 1);    // producer warp, MMA warp, epilogue warps, store warp
 constexpr int kMaxObuf = 4;
 constexpr int kMaxStages = 8;
-constexpr int kNumBarriers = 2 * kMaxStages + 2 * kMaxAcc + 2 * kEpiGroups * kMaxObuf + 1;
+constexpr int kDwWarps = 8;          // fused depthwise -> pointwise: epilogue warps 2..9 compute the depthwise layer instead
+constexpr int kDwinStages = 2;       // ... from a ring of this many input tiles
+constexpr int kNumBarriers = 2 * kMaxStages + 2 * kMaxAcc + 2 * kEpiGroups * kMaxObuf + 1 + 2 * kDwinStages;
 constexpr int kResidentBMax = 80 * 1024;   // weights of a whole layer stay in shared memory up to this size
 constexpr int kResidentB4Max = 128 * 1024; // ... and up to this size when they arrive as packed 4-bit codes
 constexpr int kMaxCls = 16;
@@ -82,6 +85,25 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f)
 {
     return f.d > 1 ? (__umulhi(n, f.mul) >> f.shr) : n;
 }
+
+// A 3x3 depthwise layer computed in front of a pointwise layer inside the same kernel (Section 7 recommends fusing
+// operators; the intermediate tensor of a depthwise-separable block then never leaves the SM).  A tile is a box of
+// tw x th x tb output pixels; for every K block of the pointwise layer (a chunk of BK depthwise channels) the producer
+// brings the box of input pixels with its halo into shared memory, eight warps compute the depthwise outputs of the
+// chunk, requantise them to the codes of the intermediate tensor (exactly what the stand-alone depthwise kernel
+// stores) and write them as the swizzled activation K block the tensor cores read.
+struct DwFront {
+    const uint32_t* taps;   // [3][tap_pitch]: per filter row and channel, bytes (k0, k1, k2, 0) as int8
+    const int32_t* wsum;
+    const int32_t* bias;
+    const int32_t* mult;
+    const int32_t* rshift;
+    int32_t tap_pitch, c, h, w;             // channels and extent of the depthwise input
+    int32_t zx, zy, act_min, act_max;       // its zero point; quantizer and clamp of the intermediate tensor
+    int32_t twin, thin;                     // input columns / rows of a tile
+    uint32_t stage_bytes, stage_stride;     // one input tile in the ring
+    int32_t gp, pairs, spi, rps, items;     // thread mapping: channel groups, column pairs, row slots per image, rows per slot
+};
 
 struct TcArgs {
     FastDiv dv_per_group, dv_group_m, dv_group_last, dv_tiles_w, dv_tiles_h;
@@ -135,17 +157,18 @@ struct TcArgs {
     qtz_add::AddRule res_rule;
     qtz_add::AddSplit res_split;
     int64_t res_addend;
+    DwFront dw;                             // used by the kernels instantiated with a depthwise front only
 };
 
 struct SmemLayout {
-    uint32_t a_off, b_off, out_off, tbl_off, tbl_stride, mult_rel, sh_rel, addhi_rel, bar_off, total;
+    uint32_t a_off, b_off, out_off, tbl_off, tbl_stride, mult_rel, sh_rel, addhi_rel, dwin_off, bar_off, total;
     uint32_t a_stage, b_stage, a_blk, b_blk;
 };
 
 // Operand ring (activations, and weights unless all `bres` weight blocks of the layer stay resident),
 // output staging boxes and one set of per-channel tables per epilogue group, barriers.
 __host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, int ncls, int out_box, int groups, int obuf, int bres, int spb,
-                                                  int a_blk = 0, int pair = 0)
+                                                  int a_blk = 0, int pair = 0, uint32_t dwin_bytes = 0)
 {
     SmemLayout L;
     L.a_blk = a_blk > 0 ? a_blk : kTileM * BK;   // one K block of activations (row-window layers: one run of the frame) / of weights
@@ -160,7 +183,8 @@ __host__ __device__ inline SmemLayout make_layout(int BK, int BN, int stages, in
     L.sh_rel = L.mult_rel + BN * 4;
     L.addhi_rel = L.sh_rel + BN * 4;
     L.tbl_stride = L.addhi_rel + BN * 4;
-    L.bar_off = L.tbl_off + groups * L.tbl_stride;
+    L.dwin_off = (L.tbl_off + groups * L.tbl_stride + 127u) & ~127u;   // ring of depthwise input tiles (fused front only)
+    L.bar_off = L.dwin_off + dwin_bytes;
     L.total = L.bar_off + kNumBarriers * 8 + 16;
     return L;
 }
@@ -281,7 +305,8 @@ __device__ __forceinline__ void tile_origin(const TcArgs& a, uint32_t m_tile, in
 
 // kPair: the CTA-pair form (launched as clusters of two; it contains cta_group::2 instructions, which a kernel
 // launched without clusters must not)
-template <bool kPair>
+// kFused: 0, or the stride (1 or 2) of a 3x3 depthwise layer computed in front of this pointwise layer (see DwFront)
+template <bool kPair, int kFused>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_s, const TcArgs a)
@@ -289,7 +314,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const smem = smem_raw + (base - smem_u32(smem_raw));
-    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb, a.a_blk, kPair);
+    const SmemLayout L = make_layout(a.BK, a.BN, a.stages, a.ncls, a.out_box, a.groups, a.obuf, a.bres, a.spb, a.a_blk, kPair,
+                                     kFused != 0 ? kDwinStages * a.dw.stage_stride : 0u);
 
     const uint32_t bar_full = base + L.bar_off;
     const uint32_t bar_empty = bar_full + 8 * kMaxStages;
@@ -298,6 +324,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t bar_ofull = bar_tempty + 8 * kMaxAcc;                               // [group][box]: box written
     const uint32_t bar_oempty = bar_ofull + 8 * kEpiGroups * kMaxObuf;        // [group][box]: box read by its store
     const uint32_t bar_wres = bar_oempty + 8 * kEpiGroups * kMaxObuf;         // resident weights have landed
+    const uint32_t bar_dfull = bar_wres + 8;                                  // [input tile stage]: landed
+    const uint32_t bar_dempty = bar_dfull + 8 * kDwinStages;                  // ... read by all depthwise warps
     volatile uint32_t* const tmem_slot =
         reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + kNumBarriers * 8);
     // pair mode: this CTA's place in its pair, and the pair's place among the pairs (tiles are dealt to pairs)
@@ -324,6 +352,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             mbar_init(bar_oempty + 8 * i, 1);
         }
         mbar_init(bar_wres, a.w4 ? kEpiWarps : 1);    // one arrival per expanding warp, or the producer's expect_tx
+        for (int s = 0; s < kDwinStages; ++s) {
+            mbar_init(bar_dfull + 8 * s, 1);
+            mbar_init(bar_dempty + 8 * s, kDwWarps);
+        }
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_a);
@@ -379,13 +411,48 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // This kernel may have started while the kernel before it in the stream was still running (programmatic
         // dependent launch): everything above touched only the layer's own constants; activations wait.
         grid_dependency_wait();
+        if constexpr (kFused != 0) {
+            // ---- depthwise front: one input tile (with its halo; cells outside the image arrive as zeros) per K block
+            uint32_t ds = 0, dphase = 0;
+            for (uint32_t tile = tile0; !failed && tile < a.num_tiles; tile += tile_step) {
+                int n_tile, w0, h0, b0;
+                uint32_t m_tile;
+                decode_tile(a, tile, m_tile, n_tile, prank);
+                tile_origin(a, m_tile, w0, h0, b0);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(bar_dempty + 8 * ds, dphase ^ 1, a.wait_budget, 64u)) || *abort_flag != 0) {
+                        failed = true;
+                        break;
+                    }
+                    if (elect_one()) {
+                        mbar_arrive_expect_tx(bar_dfull + 8 * ds, a.dw.stage_bytes);
+                        tma_load_4d(base + L.dwin_off + ds * a.dw.stage_stride, &map_a, bar_dfull + 8 * ds, kb * a.BK, w0 * kFused - 1,
+                                    h0 * kFused - 1, b0);
+                    }
+                    __syncwarp();
+                    if (++ds == kDwinStages) {
+                        ds = 0;
+                        dphase ^= 1;
+                    }
+                }
+            }
+            if (failed) {
+                if (lane == 0) {
+                    report_timeout(a.status, QTZ_SITE_SMEM_EMPTY);
+                    *abort_flag = 1;
+                }
+                const uint32_t last = ds == 0 ? kDwinStages - 1 : ds - 1;       // the most recent copy gets a bounded time to land
+                (void)mbar_wait(bar_dfull + 8 * last, ds == 0 ? dphase ^ 1 : dphase, 20000000LL);
+                failed = false;
+            }
+        }
         // ---- thread copies: every lane copies 16-byte pieces of the stage's activations; a stage is signalled
         // `lag` stages late, once this warp's copies for it have landed and been fenced for the tensor cores
         uint32_t issued = 0, signalled = 0, sig_stage = 0;
         // stages a signal trails its copies by (what may be in flight); two stages short of the ring so that the MMA
         // warp always has signalled stages ahead of it while the producer waits for a free one
         const uint32_t lag = max(1u, min(S - 3u, 6u));
-        for (uint32_t tile = tile0; a.lsu != 0 && !failed && tile < a.num_tiles; tile += tile_step) {
+        for (uint32_t tile = tile0; kFused == 0 && a.lsu != 0 && !failed && tile < a.num_tiles; tile += tile_step) {
             int n_tile, w0, h0, b0;
             uint32_t m_tile;
             decode_tile(a, tile, m_tile, n_tile, prank);
@@ -443,7 +510,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             __syncwarp();
         }
-        for (uint32_t tile = tile0; a.lsu == 0 && !failed && tile < a.num_tiles; tile += tile_step) {
+        for (uint32_t tile = tile0; kFused == 0 && a.lsu == 0 && !failed && tile < a.num_tiles; tile += tile_step) {
             int n_tile, w0, h0, b0;
             uint32_t m_tile;
             decode_tile(a, tile, m_tile, n_tile, prank);
@@ -706,6 +773,178 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             tma_store_wait_all();
         }
+    } else if (kFused != 0 && warp >= 2 && warp < 2 + kDwWarps) {
+        // ------------------------------ depthwise front ----------------------------
+        // Eight warps turn every input tile of the ring into one activation K block.  A piece of work is 4 channels x
+        // 2 adjacent output columns x rps output rows (as in the stand-alone depthwise kernel: three byte-transposed
+        // input rows rotate through registers, a filter row is one dp4a); the lanes of a warp take neighbouring channel
+        // groups, so the reads of the tile and the writes of the K block run along shared-memory rows.
+        if constexpr (kFused != 0) {
+            using namespace qtz_dw;
+            const DwFront& f = a.dw;
+            const int wt = threadIdx.x - 64;                 // 0 .. 255
+            const int cb = a.BK;
+            const uint32_t row_bytes = static_cast<uint32_t>(f.twin * cb);
+            WinOffsets wo;
+            wo.o1 = cb; wo.o2 = 2 * cb; wo.o3 = 3 * cb; wo.o4 = 4 * cb;
+            ChanConst<kModeFast> k;
+            k.off = f.zy - f.act_min;
+            k.span = f.act_max - f.act_min;
+            k.lo4 = 0x01010101u * static_cast<uint32_t>(f.act_min);
+            k.zw = 0;
+            const uint32_t fill = 0x01010101u * static_cast<uint32_t>(f.zx);
+            const uint32_t S = static_cast<uint32_t>(a.stages);
+            uint32_t stage = 0, phase = 0, ds = 0, dphase = 0;
+            bool ok = true;
+            for (uint32_t tile = tile0; ok && tile < a.num_tiles; tile += tile_step) {
+                int n_tile, w0, h0, b0;
+                uint32_t m_tile;
+                decode_tile(a, tile, m_tile, n_tile, prank);
+                tile_origin(a, m_tile, w0, h0, b0);
+                const int ih0 = h0 * kFused - 1, iw0 = w0 * kFused - 1;
+                const bool border = f.zx != 0 && (ih0 < 0 || iw0 < 0 || ih0 + f.thin > f.h || iw0 + f.twin > f.w);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    // the input tile has landed and the K block's place in the ring is free
+                    bool got = __all_sync(0xffffffffu, mbar_wait(bar_dfull + 8 * ds, dphase, a.wait_budget, 64u)) &&
+                               __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * stage, phase ^ 1, a.wait_budget, 64u));
+                    // (a tile that needs its padding refilled has a barrier among these warps below: they decide
+                    //  together, so that no warp is left alone at it when another one's wait ran out)
+                    if (border) got = named_barrier_and(9, 32 * kDwWarps, got);
+                    if (!got) {
+                        if (lane == 0) {
+                            report_timeout(a.status, QTZ_SITE_TMA_FULL);
+                            *abort_flag = 1;
+                        }
+                        ok = false;
+                        break;
+                    }
+                    uint8_t* const tile_s = smem + L.dwin_off + ds * f.stage_stride;
+                    if (border) {
+                        // padding is real zero = the code z_x: overwrite the cells that lie outside the image
+                        const int rows_in = min(f.thin, f.h - ih0), first_row = ih0 < 0 ? 1 : 0;
+                        const int cols_in = min(f.twin, f.w - iw0), first_col = iw0 < 0 ? 1 : 0;
+                        const int lane8 = 8 * lane, warp_id = wt >> 5;
+                        for (int img = 0; img < a.tb; ++img) {
+                            uint8_t* const img_s = tile_s + img * f.thin * row_bytes;
+                            if (first_row)
+                                for (uint32_t i = 8 * wt; i < row_bytes; i += 8 * 32 * kDwWarps) *reinterpret_cast<uint2*>(img_s + i) = make_uint2(fill, fill);
+                            for (int ri = rows_in; ri < f.thin; ++ri)
+                                for (uint32_t i = 8 * wt; i < row_bytes; i += 8 * 32 * kDwWarps)
+                                    *reinterpret_cast<uint2*>(img_s + ri * row_bytes + i) = make_uint2(fill, fill);
+                            if (first_col + f.twin - cols_in > 0) {
+                                for (int ri = first_row + warp_id; ri < rows_in; ri += kDwWarps) {
+                                    uint8_t* const row = img_s + ri * row_bytes;
+                                    if (first_col)
+                                        for (int i = lane8; i < cb; i += 256) *reinterpret_cast<uint2*>(row + i) = make_uint2(fill, fill);
+                                    for (int i = lane8; i < (f.twin - cols_in) * cb; i += 256)
+                                        *reinterpret_cast<uint2*>(row + cols_in * cb + i) = make_uint2(fill, fill);
+                                }
+                            }
+                        }
+                        named_barrier(8, 32 * kDwWarps);
+                    }
+                    uint8_t* const a_stage = smem + L.a_off + stage * L.a_stage;
+                    const uint32_t tile_addr = base + L.dwin_off + ds * f.stage_stride;
+                    for (int item = wt; item < f.items; item += 32 * kDwWarps) {
+                        const int g = item % f.gp, rest = item / f.gp;
+                        const int pr = rest % f.pairs, slot = rest / f.pairs;
+                        const int img = slot / f.spi, part = slot - img * f.spi;
+                        const int c0 = kb * cb + 4 * g;
+                        const int ow0 = 2 * pr;
+                        const bool second = ow0 + 1 < a.tw;
+                        const int r_begin = part * f.rps;
+                        int n = min(a.th, r_begin + f.rps) - r_begin;            // output rows of this piece
+                        if (n <= 0) continue;
+                        uint32_t arow = static_cast<uint32_t>((img * a.th + r_begin) * a.tw + ow0);   // row of the K block: the tile's pixel
+                        if (c0 >= f.c) {                                           // channels beyond the layer's: zero codes
+                            for (; n > 0; --n, arow += a.tw) {
+                                *reinterpret_cast<uint32_t*>(a_stage + swz(arow, 4 * g, cb)) = 0u;
+                                if (second) *reinterpret_cast<uint32_t*>(a_stage + swz(arow + 1, 4 * g, cb)) = 0u;
+                            }
+                            continue;
+                        }
+                        // per-channel constants of the piece's four channels
+#pragma unroll
+                        for (int i = 0; i < 3; ++i) {
+                            const uint4 w = __ldg(reinterpret_cast<const uint4*>(f.taps + static_cast<int64_t>(i) * f.tap_pitch + c0));
+                            k.wa[i][0] = w.x; k.wa[i][1] = w.y; k.wa[i][2] = w.z; k.wa[i][3] = w.w;
+#pragma unroll
+                            for (int ch = 0; ch < 4; ++ch) k.wb[i][ch] = k.wa[i][ch] << 8;
+                        }
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            const int32_t r = __ldg(f.rshift + c0 + ch);
+                            const int32_t bse = __ldg(f.bias + c0 + ch) - f.zx * __ldg(f.wsum + c0 + ch);
+                            k.m[ch] = __ldg(f.mult + c0 + ch);
+                            k.sh[ch] = r - 32;
+                            k.add[ch] = (static_cast<int64_t>(2 * k.off + 1) << (r - 1)) + static_cast<int64_t>(bse) * k.m[ch];
+                        }
+                        auto emit = [&](const RowState<kFused>& r0, const RowState<kFused>& r1, const RowState<kFused>& r2) {
+                            int32_t acc[2][4];
+                            mac3<kFused, false, kModeFast>(r0, r1, r2, k, acc);
+                            const uint32_t y0 = requant_pixel<kModeFast, true>(acc[0], k);
+                            const uint32_t y1 = requant_pixel<kModeFast, true>(acc[1], k);
+                            *reinterpret_cast<uint32_t*>(a_stage + swz(arow, 4 * g, cb)) = y0;
+                            if (second) *reinterpret_cast<uint32_t*>(a_stage + swz(arow + 1, 4 * g, cb)) = y1;
+                            arow += a.tw;
+                        };
+                        uint32_t cell = tile_addr + ((img * f.thin + r_begin * kFused) * f.twin + ow0 * kFused) * cb + 4 * g;
+                        if constexpr (kFused == 1) {
+                            RowState<1> r0, r1, r2;
+                            load_row<1>(cell, wo, r0); cell += row_bytes;
+                            load_row<1>(cell, wo, r1); cell += row_bytes;
+                            for (; n >= 3; n -= 3) {
+                                load_row<1>(cell, wo, r2); cell += row_bytes;
+                                emit(r0, r1, r2);
+                                load_row<1>(cell, wo, r0); cell += row_bytes;
+                                emit(r1, r2, r0);
+                                load_row<1>(cell, wo, r1); cell += row_bytes;
+                                emit(r2, r0, r1);
+                            }
+                            if (n >= 1) {
+                                load_row<1>(cell, wo, r2); cell += row_bytes;
+                                emit(r0, r1, r2);
+                                if (n == 2) {
+                                    load_row<1>(cell, wo, r0);
+                                    emit(r1, r2, r0);
+                                }
+                            }
+                        } else {
+                            RowState<2> top, mid, bot;
+                            load_row<2>(cell, wo, top); cell += row_bytes;
+                            for (; n >= 2; n -= 2) {
+                                load_row<2>(cell, wo, mid); cell += row_bytes;
+                                load_row<2>(cell, wo, bot); cell += row_bytes;
+                                emit(top, mid, bot);
+                                load_row<2>(cell, wo, mid); cell += row_bytes;
+                                load_row<2>(cell, wo, top); cell += row_bytes;
+                                emit(bot, mid, top);
+                            }
+                            if (n == 1) {
+                                load_row<2>(cell, wo, mid); cell += row_bytes;
+                                load_row<2>(cell, wo, bot);
+                                emit(top, mid, bot);
+                            }
+                        }
+                    }
+                    // the K block is written (generic proxy) for the tensor cores (async proxy); the input tile is free
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(bar_full + 8 * stage);
+                        mbar_arrive(bar_dempty + 8 * ds);
+                    }
+                    if (++stage == S) {
+                        stage = 0;
+                        phase ^= 1;
+                    }
+                    if (++ds == kDwinStages) {
+                        ds = 0;
+                        dphase ^= 1;
+                    }
+                }
+            }
+        }
     } else {
         // ------------------------------ epilogue ----------------------------------
         // Sixteen warps as four groups of four (narrow tiles: more work per warp and tile, so the per-tile
@@ -715,7 +954,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // the columns of every staging box in halves.  The warps of a group run free of one another: a
         // warp waits for a staging box to be empty, fills its part and signals the box's barrier; the
         // group's store lane issues the store once all warps of the group have signalled.
-        const int et = threadIdx.x - 64;             // 0..511
+        const int et = threadIdx.x - 64 - (kFused != 0 ? 32 * kDwWarps : 0);   // 0..511 (0..255 behind a depthwise front)
         const int gthreads = 32 * a.gwarps;          // 128 or 256 threads per group
         const int grp = et / gthreads;
         const int gt = et - grp * gthreads;          // thread within the group
@@ -1539,8 +1778,8 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
         at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
         cfg.attrs = &at;
         cfg.numAttrs = 1;
-        (void)cudaFuncSetAttribute(conv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (cudaOccupancyMaxActiveClusters(&clusters, conv_tc_kernel<true>, &cfg) == cudaSuccess && clusters >= h->num_sms / 4) {
+        (void)cudaFuncSetAttribute(conv_tc_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (cudaOccupancyMaxActiveClusters(&clusters, conv_tc_kernel<true, 0>, &cfg) == cudaSuccess && clusters >= h->num_sms / 4) {
             a.pair = 1;
             t->pair = true;
             a.m_tiles = (a.m_tiles + 1) / 2;
@@ -1642,7 +1881,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
                       : static_cast<int>(std::min<int64_t>(a.num_tiles, h->num_sms));
 
     // per device, so set for the device of this plan every time (the call is cheap)
-    QTZ_CUDA(h, cudaFuncSetAttribute(conv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    QTZ_CUDA(h, cudaFuncSetAttribute(conv_tc_kernel<false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     return QTZ_OK;
 }
 
@@ -1861,11 +2100,179 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
         cfg.attrs = at;
         cfg.numAttrs = n_at;
         if (t->pair)
-            QTZ_CUDA(h, cudaLaunchKernelEx(&cfg, conv_tc_kernel<true>, map_a, t->map_b_half, map_y, map_s, a));
+            QTZ_CUDA(h, cudaLaunchKernelEx(&cfg, conv_tc_kernel<true, 0>, map_a, t->map_b_half, map_y, map_s, a));
         else
-            QTZ_CUDA(h, cudaLaunchKernelEx(&cfg, conv_tc_kernel<false>, map_a, t->map_b, map_y, map_s, a));
+            QTZ_CUDA(h, cudaLaunchKernelEx(&cfg, conv_tc_kernel<false, 0>, map_a, t->map_b, map_y, map_s, a));
     }
     QTZ_LAUNCH_CHECK(h, "conv_tc_kernel");
+    if (p->ev_stop) QTZ_CUDA(h, cudaEventRecord(p->ev_stop, st));
+    return QTZ_OK;
+}
+
+// Depthwise 3x3 -> pointwise in one kernel (see DwFront).  QTZ_ERR_UNSUPPORTED when this pair of layers cannot run
+// that way; the caller then runs the two plans one after the other, with the same result.
+qtz_status qtz_tc_launch_dw_pw(qtz_plan* dwp, qtz_plan* p, const uint8_t* x, int32_t x_zp, int32_t mid_zp, int32_t mid_min,
+                               int32_t mid_max, void* y, int32_t y_zp, int32_t act_min, int32_t act_max, cudaStream_t st)
+{
+    qtz_ctx* h = p->h;
+    qtz_tc_state* t = p->tc;
+    const qtz_conv_desc& d = p->d;       // the pointwise layer
+    const qtz_conv_desc& dd = dwp->d;    // the depthwise layer
+    if (!t || t->rowwin || t->im2col || t->pair || t->w_packed4 || !is_pointwise(d) || d.stride != 1) return QTZ_ERR_UNSUPPORTED;
+    if (d.outkind != QTZ_OUT_U8 || dd.outkind != QTZ_OUT_U8 || p->w_zp_signed != 0 || dwp->w_zp_signed != 0) return QTZ_ERR_UNSUPPORTED;
+    if (dwp->rshift_min < 32 || dwp->rshift_max > 53 || (dd.stride != 1 && dd.stride != 2)) return QTZ_ERR_UNSUPPORTED;
+    if (d.c != dd.c || d.batch != dd.batch || d.h != dwp->oh || d.w != dwp->ow || (dd.c & 3)) return QTZ_ERR_INVALID_ARG;
+    TcArgs a = t->args;
+    a.wait_budget = h->wait_budget;
+    // one column tile over all output channels (several would each repeat the depthwise work of their pixels), whatever
+    // split the plan chose for the pointwise layer alone
+    if (d.n > 256) return QTZ_ERR_UNSUPPORTED;
+    a.n_tiles = 1;
+    a.BN = (d.n + 31) / 32 * 32;
+    a.out_box = (a.BN % 128 == 0 || a.BN > 128) ? 128 : 64;
+    a.n_acc = std::min(kMaxAcc, kTmemCols / a.BN);
+    a.acc_stride = a.BN;
+    a.idesc = (2u << 4) | (0u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
+    if (a.BN > t->n_pad) return QTZ_ERR_UNSUPPORTED;
+    CUtensorMap map_b;
+    {
+        const uint64_t dims[2] = {static_cast<uint64_t>(a.taps) * a.c_pad, static_cast<uint64_t>(t->n_pad)};
+        const uint64_t strides[1] = {static_cast<uint64_t>(a.taps) * a.c_pad};
+        const uint32_t box[2] = {static_cast<uint32_t>(a.BK), static_cast<uint32_t>(a.BN)};
+        if (!encode_map(&map_b, t->w_packed, 2, dims, strides, box, a.BK)) return QTZ_ERR_CUDA;
+    }
+    const int kblocks = a.kb_per_tap;
+    if (static_cast<int64_t>(kblocks) * a.BN * a.BK > kResidentBMax) return QTZ_ERR_UNSUPPORTED;
+    a.bres = kblocks;
+    a.spb = 1;
+    a.is4d = 1;
+    a.W = p->ow; a.H = p->oh; a.B = d.batch;
+    a.zx = mid_zp; a.zy = y_zp; a.act_min = act_min; a.act_max = act_max;
+    a.res = 0; a.raw = 0; a.ncls = 1; a.lsu = 0; a.w4 = nullptr; a.src = nullptr;
+    a.full_count = kDwWarps;
+    a.groups = 2; a.gwarps = 4;
+    a.fold = p->rshift_max <= 53 ? (p->rshift_min >= 32 ? 1 : (p->narrow_ok ? 2 : 0)) : 0;
+    DwFront& f = a.dw;
+    f.taps = dwp->dw_taps; f.wsum = dwp->dw_wsum; f.bias = dwp->bias; f.mult = dwp->mult; f.rshift = dwp->rshift;
+    f.tap_pitch = dd.c_pitch_in; f.c = dd.c; f.h = dd.h; f.w = dd.w;
+    f.zx = x_zp; f.zy = mid_zp; f.act_min = mid_min; f.act_max = mid_max;
+    f.gp = a.BK / 4;
+    const int sd = dd.stride;
+    // Tile: the box of output pixels (at most 128) that costs the depthwise warps least over the whole layer, among
+    // those whose ring of input tiles fits beside at least two operand stages and one staging box per group.
+    double best = 0.0;
+    bool found = false;
+    int bt[3] = {0, 0, 0};
+    for (int tw = 2; tw <= std::min(a.W + (a.W & 1), kTileM); tw += 2) {
+        if (tw > a.W + 1) break;
+        for (int th = 1; th <= std::min(a.H, kTileM / tw); ++th) {
+            const int tb = (tw >= a.W && th >= a.H) ? std::min(a.B, kTileM / (tw * th)) : 1;
+            const int twin = (tw - 1) * sd + 3, thin = (th - 1) * sd + 3;
+            if (twin > 256 || thin > 256) continue;
+            const uint32_t sbytes = static_cast<uint32_t>(a.BK) * twin * thin * tb;
+            const uint32_t sstride = (sbytes + 127u) & ~127u;
+            if (make_layout(a.BK, a.BN, 2, 1, a.out_box, 2, 1, a.bres, 1, 0, 0, kDwinStages * sstride).total > static_cast<uint32_t>(kSmemBudget)) continue;
+            const int pairs = tw / 2;
+            const int spi = std::max(1, std::min(th, 32 * kDwWarps / std::max(1, f.gp * pairs * tb)));
+            const int rps = (th + spi - 1) / spi;
+            const int items = f.gp * pairs * tb * spi;
+            const int iters = (items + 32 * kDwWarps - 1) / (32 * kDwWarps);
+            const int64_t tiles = static_cast<int64_t>((a.W + tw - 1) / tw) * ((a.H + th - 1) / th) * ((a.B + tb - 1) / tb);
+            const int64_t rounds = (tiles + h->num_sms - 1) / h->num_sms;
+            const double cost = static_cast<double>(rounds) * kblocks * (iters * (rps + (sd == 1 ? 0.7 : 1.0)) + 0.8);
+            if (!found || cost < best) {
+                found = true;
+                best = cost;
+                bt[0] = tw; bt[1] = th; bt[2] = tb;
+            }
+        }
+    }
+    if (!found) return QTZ_ERR_UNSUPPORTED;
+    a.tw = bt[0]; a.th = bt[1]; a.tb = bt[2];
+    a.rows = a.tw * a.th * a.tb;
+    a.tiles_w = (a.W + a.tw - 1) / a.tw;
+    a.tiles_h = (a.H + a.th - 1) / a.th;
+    const int64_t tiles = static_cast<int64_t>(a.tiles_w) * a.tiles_h * ((a.B + a.tb - 1) / a.tb);
+    if (tiles > 0x7fffffff) return QTZ_ERR_UNSUPPORTED;
+    a.num_tiles = static_cast<uint32_t>(tiles);
+    a.m_tiles = static_cast<int32_t>(tiles);
+    a.group_m = std::max(1, std::min(a.m_tiles, 16));
+    a.dv_per_group = make_fastdiv(static_cast<uint32_t>(a.group_m));
+    a.dv_group_m = make_fastdiv(static_cast<uint32_t>(a.group_m));
+    a.dv_group_last = make_fastdiv(static_cast<uint32_t>(std::max(1, a.m_tiles % a.group_m)));
+    a.dv_tiles_w = make_fastdiv(static_cast<uint32_t>(a.tiles_w));
+    a.dv_tiles_h = make_fastdiv(static_cast<uint32_t>(a.tiles_h));
+    f.twin = (a.tw - 1) * sd + 3;
+    f.thin = (a.th - 1) * sd + 3;
+    f.stage_bytes = static_cast<uint32_t>(a.BK) * f.twin * f.thin * a.tb;
+    f.stage_stride = (f.stage_bytes + 127u) & ~127u;
+    f.pairs = a.tw / 2;
+    f.spi = std::max(1, std::min(a.th, 32 * kDwWarps / std::max(1, f.gp * f.pairs * a.tb)));
+    f.rps = (a.th + f.spi - 1) / f.spi;
+    f.items = f.gp * f.pairs * a.tb * f.spi;
+    // ring depth and staging boxes from what is left of shared memory
+    const uint32_t dwin_bytes = kDwinStages * f.stage_stride;
+    a.obuf = 1;
+    a.stages = 2;
+    for (int ob = 2; ob >= 1 && a.obuf == 1; --ob)
+        for (int st_ = 4; st_ >= 3; --st_)
+            if (make_layout(a.BK, a.BN, st_, 1, a.out_box, 2, ob, a.bres, 1, 0, 0, dwin_bytes).total <= static_cast<uint32_t>(kSmemBudget)) {
+                a.obuf = ob;
+                a.stages = st_;
+                break;
+            }
+    if (a.obuf == 1)
+        for (int st_ = 4; st_ >= 2; --st_)
+            if (make_layout(a.BK, a.BN, st_, 1, a.out_box, 2, 1, a.bres, 1, 0, 0, dwin_bytes).total <= static_cast<uint32_t>(kSmemBudget)) {
+                a.stages = st_;
+                break;
+            }
+    const uint32_t smem_bytes = make_layout(a.BK, a.BN, a.stages, 1, a.out_box, 2, a.obuf, a.bres, 1, 0, 0, dwin_bytes).total + 1024;
+    if (smem_bytes > 227u * 1024u) return QTZ_ERR_UNSUPPORTED;
+
+    CUtensorMap map_a, map_y;
+    {
+        const uint64_t pitch = static_cast<uint64_t>(dd.c_pitch_in);
+        const uint64_t dims[4] = {static_cast<uint64_t>(dd.c), static_cast<uint64_t>(dd.w), static_cast<uint64_t>(dd.h),
+                                  static_cast<uint64_t>(dd.batch)};
+        const uint64_t strides[3] = {pitch, pitch * dd.w, pitch * dd.w * dd.h};
+        const uint32_t box[4] = {static_cast<uint32_t>(a.BK), static_cast<uint32_t>(f.twin), static_cast<uint32_t>(f.thin),
+                                 static_cast<uint32_t>(a.tb)};
+        if (!encode_map(&map_a, x, 4, dims, strides, box, 0)) return QTZ_ERR_CUDA;
+    }
+    {
+        const uint64_t opitch = static_cast<uint64_t>(d.c_pitch_out);
+        const uint64_t dims[4] = {static_cast<uint64_t>(d.n), static_cast<uint64_t>(p->ow), static_cast<uint64_t>(p->oh),
+                                  static_cast<uint64_t>(d.batch)};
+        const uint64_t strides[3] = {opitch, opitch * p->ow, opitch * p->ow * p->oh};
+        const uint32_t box[4] = {static_cast<uint32_t>(a.out_box), static_cast<uint32_t>(a.tw), static_cast<uint32_t>(a.th),
+                                 static_cast<uint32_t>(a.tb)};
+        if (!encode_map(&map_y, y, 4, dims, strides, box, a.out_box)) return QTZ_ERR_CUDA;
+    }
+    const int grid = static_cast<int>(std::min<int64_t>(a.num_tiles, h->num_sms));
+    p->detail = std::string("tcgen05 pointwise weights:resident depthwise-front stride ") + std::to_string(sd) + " tile " +
+                std::to_string(a.tw) + "x" + std::to_string(a.th) + "x" + std::to_string(a.tb);
+    if (p->ev_start) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(grid));
+        cfg.blockDim = dim3(kThreadsTc);
+        cfg.dynamicSmemBytes = smem_bytes;
+        cfg.stream = st;
+        cudaLaunchAttribute at;
+        at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &at;
+        cfg.numAttrs = 1;
+        if (sd == 1) {
+            QTZ_CUDA(h, cudaFuncSetAttribute(conv_tc_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            QTZ_CUDA(h, cudaLaunchKernelEx(&cfg, conv_tc_kernel<false, 1>, map_a, map_b, map_y, map_b, a));
+        } else {
+            QTZ_CUDA(h, cudaFuncSetAttribute(conv_tc_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            QTZ_CUDA(h, cudaLaunchKernelEx(&cfg, conv_tc_kernel<false, 2>, map_a, map_b, map_y, map_b, a));
+        }
+    }
+    QTZ_LAUNCH_CHECK(h, "conv_tc_kernel (depthwise front)");
     if (p->ev_stop) QTZ_CUDA(h, cudaEventRecord(p->ev_stop, st));
     return QTZ_OK;
 }

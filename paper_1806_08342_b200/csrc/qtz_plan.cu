@@ -307,6 +307,22 @@ extern "C" qtz_status qtz_conv2d_add_u8(qtz_conv_plan p, const uint8_t* x_dev, i
     return qtz_tc_launch(p, x_dev, x_zero_point, y_dev, y_zero_point, act_min, act_max, static_cast<cudaStream_t>(stream), r, s_dev);
 }
 
+extern "C" qtz_status qtz_conv2d_dw_pw_u8(qtz_conv_plan dw, qtz_conv_plan pw, const uint8_t* x_dev, int32_t x_zero_point,
+                                          int32_t mid_zero_point, int32_t mid_act_min, int32_t mid_act_max, void* y_dev,
+                                          int32_t y_zero_point, int32_t act_min, int32_t act_max, void* stream)
+{
+    if (!dw) return QTZ_ERR_INVALID_ARG;
+    qtz_status s = check_run_args(pw, x_dev, y_dev, x_zero_point, y_zero_point, act_min, act_max);
+    if (s != QTZ_OK) return s;
+    if (!dw->depthwise || pw->depthwise || dw->h != pw->h || dw->device != pw->device) return QTZ_ERR_INVALID_ARG;
+    if (mid_zero_point < 0 || mid_zero_point > 255 || mid_act_min < 0 || mid_act_max > 255 || mid_act_min > mid_act_max)
+        return QTZ_ERR_INVALID_ARG;
+    if (pw->family != QTZ_K_TCGEN05 || dw->family != QTZ_K_DEPTHWISE) return QTZ_ERR_UNSUPPORTED;
+    qtz_device_guard guard(pw->device);
+    return qtz_tc_launch_dw_pw(dw, pw, x_dev, x_zero_point, mid_zero_point, mid_act_min, mid_act_max, y_dev, y_zero_point,
+                               act_min, act_max, static_cast<cudaStream_t>(stream));
+}
+
 extern "C" qtz_status qtz_depthwise_u8(qtz_conv_plan p, const uint8_t* x_dev, int32_t x_zero_point, void* y_dev,
                                        int32_t y_zero_point, int32_t act_min, int32_t act_max, void* stream)
 {

@@ -56,6 +56,11 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
                          int32_t act_min, int32_t act_max, cudaStream_t st, const qtz_residual* res = nullptr,
                          const uint8_t* s_dev = nullptr);
 
+// A 3x3 depthwise plan and the pointwise plan that follows it, in one kernel (the intermediate tensor, with zero point
+// mid_zp and clamp [mid_min, mid_max], stays in shared memory).  QTZ_ERR_UNSUPPORTED when the pair cannot run that way.
+qtz_status qtz_tc_launch_dw_pw(qtz_plan* dw, qtz_plan* pw, const uint8_t* x, int32_t x_zp, int32_t mid_zp, int32_t mid_min,
+                               int32_t mid_max, void* y, int32_t y_zp, int32_t act_min, int32_t act_max, cudaStream_t st);
+
 // Encodes a rank-2 or rank-4 uint8 tensor map (dims[0] contiguous).  swizzle_bytes: 0 (none), 32, 64 or 128.
 bool qtz_encode_u8_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                        const uint32_t* box, int swizzle_bytes);

@@ -91,6 +91,8 @@ SIGNATURES = {
     "qtz_conv2d_add_u8": (c_int32, [c_void_p, c_void_p, c_int32, POINTER(Residual), c_void_p, c_void_p, c_int32, c_int32, c_int32,
                                     c_void_p]),
     "qtz_depthwise_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p]),
+    "qtz_conv2d_dw_pw_u8": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p, c_int32, c_int32,
+                                      c_int32, c_void_p]),
     "qtz_add_u8": (c_int32, [c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p,
                              c_int32, c_int32, c_int32, c_int64, c_int32, c_int32, c_void_p]),
     "qtz_simquant": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int32, c_int32, c_void_p, c_void_p]),
@@ -537,6 +539,18 @@ class ConvPlan:
         self.handle._chk(self.handle.lib.qtz_conv2d_add_u8(self.plan, _ptr(x), int(x_zero_point), byref(residual), _ptr(s),
                                                            _ptr(out), int(y_zero_point), int(act_min), int(act_max), _stream()),
                          "qtz_conv2d_add_u8")
+        return out
+
+    def after_depthwise(self, dw_plan, x, x_zero_point, mid_zero_point, mid_act_min, mid_act_max, y_zero_point, act_min,
+                        act_max, out=None):
+        """qtz_conv2d_dw_pw_u8: the 3x3 depthwise plan `dw_plan` and this pointwise plan in one kernel.  Raises
+        QtzError (code ERR_UNSUPPORTED) when the pair cannot run fused."""
+        _check_dev(x, out)
+        out = self.empty_output(x.device) if out is None else out
+        self.handle._chk(self.handle.lib.qtz_conv2d_dw_pw_u8(dw_plan.plan, self.plan, _ptr(x), int(x_zero_point),
+                                                             int(mid_zero_point), int(mid_act_min), int(mid_act_max), _ptr(out),
+                                                             int(y_zero_point), int(act_min), int(act_max), _stream()),
+                         "qtz_conv2d_dw_pw_u8")
         return out
 
     def set_profile_events(self, start=None, stop=None):
