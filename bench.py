@@ -432,7 +432,7 @@ def time_networks(hq, qtz, torch, peaks, reps=10, detail=False):
             rows = []
             for i, item in enumerate(net.schedule):
                 L = item[2] if item[0] == "conv+add" else item[1]
-                kern = item[1].plan.detail if item[0] in ("conv", "fc", "conv+add") else item[0]
+                kern = item[1].plan.detail if item[0] in ("conv", "fc", "conv+add", "dw+pw") else item[0]
                 rows.append((round(evs[i].elapsed_time(evs[i + 1]) * 1e3, 1), L.op.get("dst"), kern,
                              tuple(t[L.op["dst"]].shape)))
             entry["layers_us"] = rows

@@ -795,6 +795,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t fill = 0x01010101u * static_cast<uint32_t>(f.zx);
             const uint32_t S = static_cast<uint32_t>(a.stages);
             uint32_t stage = 0, phase = 0, ds = 0, dphase = 0;
+            int loaded_c0 = -1;
             bool ok = true;
             for (uint32_t tile = tile0; ok && tile < a.num_tiles; tile += tile_step) {
                 int n_tile, w0, h0, b0;
@@ -863,7 +864,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             }
                             continue;
                         }
-                        // per-channel constants of the piece's four channels
+                        // per-channel constants of the piece's four channels (kept while the thread stays on them)
+                        if (c0 != loaded_c0) {
+                        loaded_c0 = c0;
 #pragma unroll
                         for (int i = 0; i < 3; ++i) {
                             const uint4 w = __ldg(reinterpret_cast<const uint4*>(f.taps + static_cast<int64_t>(i) * f.tap_pitch + c0));
@@ -878,6 +881,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             k.m[ch] = __ldg(f.mult + c0 + ch);
                             k.sh[ch] = r - 32;
                             k.add[ch] = (static_cast<int64_t>(2 * k.off + 1) << (r - 1)) + static_cast<int64_t>(bse) * k.m[ch];
+                        }
                         }
                         auto emit = [&](const RowState<kFused>& r0, const RowState<kFused>& r1, const RowState<kFused>& r2) {
                             int32_t acc[2][4];
@@ -2179,7 +2183,9 @@ qtz_status qtz_tc_launch_dw_pw(qtz_plan* dwp, qtz_plan* p, const uint8_t* x, int
             const int iters = (items + 32 * kDwWarps - 1) / (32 * kDwWarps);
             const int64_t tiles = static_cast<int64_t>((a.W + tw - 1) / tw) * ((a.H + th - 1) / th) * ((a.B + tb - 1) / tb);
             const int64_t rounds = (tiles + h->num_sms - 1) / h->num_sms;
-            const double cost = static_cast<double>(rounds) * kblocks * (iters * (rps + (sd == 1 ? 0.7 : 1.0)) + 0.8);
+            // (per K block: the pieces' row steps, and the tile's input cells through the copy engine and shared memory)
+            const double cost = static_cast<double>(rounds) * kblocks *
+                                (iters * (rps + (sd == 1 ? 0.7 : 1.0)) + 0.8 + 0.02 * twin * thin * tb);
             if (!found || cost < best) {
                 found = true;
                 best = cost;

@@ -25,9 +25,12 @@ class _Layer:
 
 
 class QuantizedNetwork:
-    def __init__(self, handle: qtz.Handle, ops, seed: int, wbits: int = 8, fuse: bool = True):
+    def __init__(self, handle: qtz.Handle, ops, seed: int, wbits: int = 8, fuse: bool = True, fuse_depthwise: bool = False):
         self.h, self.ops, self.seed, self.wbits = handle, ops, seed, wbits
         self.fuse = fuse            # forward() runs a convolution and the residual add that follows it as one kernel
+        # forward() runs a 3x3 depthwise layer and the pointwise layer after it as one kernel where the library can
+        # (qtz_conv2d_dw_pw_u8).  Off by default: on the networks here the two separate kernels are faster.
+        self.fuse_depthwise = fuse_depthwise
         self.fused_away = set()     # tensors forward() then never writes (build() still computes them once)
         self.schedule = []          # what forward() launches: (kind, layer[, add layer])
         self.layers = []
@@ -164,11 +167,34 @@ class QuantizedNetwork:
                         fused[id(L)] = (P, mine, other)
                         break
         self.fused_away = {P.op["dst"] for P, _, _ in fused.values()}
+        # depthwise -> pointwise pairs: the depthwise output has the pointwise layer as its only reader; the library
+        # decides whether the pair can run as one kernel (a first call here, into the pointwise layer's own output)
+        blocks = {}
+        if self.fuse_depthwise:
+            t = self.tensors
+            for D in self.layers:
+                if D.op["op"] != "conv" or not D.op["depthwise"] or readers.get(D.op["dst"], 0) != 1:
+                    continue
+                P = next((L for L in self.layers if L.op.get("src") == D.op["dst"]), None)
+                if (P is None or P.op["op"] != "conv" or P.op["depthwise"] or P.op["k"] != 1 or P.op["stride"] != 1
+                        or id(P) in taken or P.plan.kernel != "tcgen05"):
+                    continue
+                try:
+                    P.plan.after_depthwise(D.plan, t[D.op["src"]], *D.args, *P.args[1:], out=t[P.op["dst"]])
+                except qtz.QtzError as e:
+                    if e.code != -3:        # QTZ_ERR_UNSUPPORTED: the pair stays two kernels
+                        raise
+                    continue
+                blocks[id(P)] = D
+                taken.add(id(D))
+                self.fused_away.add(D.op["dst"])
         self.schedule = []
         for L in self.layers:
             if id(L) in taken:
                 continue
-            if id(L) in fused:
+            if id(L) in blocks:
+                self.schedule.append(("dw+pw", L, blocks[id(L)]))
+            elif id(L) in fused:
                 P, mine, other = fused[id(L)]
                 a = L.args      # (za, ma, zb, mb, r, zy, amin, amax, c)
                 t_zp, t_mult, s_zp, s_mult = (a[0], a[1], a[2], a[3]) if mine == "a" else (a[2], a[3], a[0], a[1])
@@ -197,6 +223,9 @@ class QuantizedNetwork:
             _, P, A, res, other = item
             a = A.args
             P.plan.add_fused(t[P.op["src"]], P.args[0], res, t[A.op[other]], a[5], a[6], a[7], out=t[A.op["dst"]])
+        elif kind == "dw+pw":
+            D = item[2]
+            L.plan.after_depthwise(D.plan, t[D.op["src"]], *D.args, *L.args[1:], out=t[op["dst"]])
         elif kind in ("conv", "fc"):
             L.plan(t[op["src"]], *L.args, out=t[op["dst"]])
         elif kind == "add":

@@ -68,6 +68,29 @@ def test_network_small_batch_every_layer(hq, name):
     assert "tcgen05" in kinds                                         # stems included (explicit im2col)
 
 
+def test_network_with_fused_depthwise_blocks(hq):
+    """MobileNet-v1 with every depthwise -> pointwise pair the library can fuse run as one kernel: the tensors the
+    timed pass still writes equal the oracle's, the intermediate tensors are never stored."""
+    ops = synth.NETWORKS["mobilenet_v1"]()
+    images = synth.network_input(3, 224, 11)
+    want = netrun.run(ops, images, 2, 11, 8)
+    net = network.QuantizedNetwork(hq, ops, 11, 8, fuse_depthwise=True)
+    got = net.build(images, 2)
+    torch.cuda.synchronize()
+    blocks = [item for item in net.schedule if item[0] == "dw+pw"]
+    assert len(blocks) >= 5, [item[0] for item in net.schedule]
+    assert all("depthwise-front" in item[1].plan.detail for item in blocks)
+    for key, t in got.items():
+        if t.dtype == torch.uint8 and key != "in":
+            t.zero_()
+    net.forward()
+    torch.cuda.synchronize()
+    assert all(not got[key].any() for key in net.fused_away)          # never written by the timed pass
+    compare(net, got, want, skip=net.fused_away)
+    rc, site = hq.device_status()
+    assert rc == 0, (rc, site)
+
+
 @pytest.mark.parametrize("name,batch", [("mobilenet_v1", 128), ("resnet50", 256), ("mobilenet_v2_14", 256)])
 def test_network_full_batch_sampled_images(hq, name, batch):
     ops = synth.NETWORKS[name]()
