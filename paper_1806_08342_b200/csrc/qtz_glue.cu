@@ -42,6 +42,9 @@ add_u8_kernel(const uint8_t* __restrict__ a, const uint8_t* __restrict__ b, int6
 }
 
 // One thread per (output pixel, 16-channel group).
+// kK > 0: the window size, known at compile time, so that all its loads are in flight together (out-of-image
+// taps read as 0, the neutral element of max over unsigned codes); kK = 0: any window.
+template <int kK>
 __global__ void __launch_bounds__(kThreads)
 maxpool_u8_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ y, int batch, int hh, int ww, int pitch,
                   int k, int stride, int pad, int oh_n, int ow_n)
@@ -56,14 +59,31 @@ maxpool_u8_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ y, int ba
     const int oh = static_cast<int>(p % oh_n);
     const int b = static_cast<int>(p / oh_n);
     uint4 m = make_uint4(0, 0, 0, 0);
-    for (int i = 0; i < k; ++i) {
-        const int ih = oh * stride - pad + i;
-        if (ih < 0 || ih >= hh) continue;
-        for (int j = 0; j < k; ++j) {
-            const int iw = ow * stride - pad + j;
-            if (iw < 0 || iw >= ww) continue;
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + ((static_cast<int64_t>(b) * hh + ih) * ww + iw) * pitch) + g);
-            m.x = __vmaxu4(m.x, v.x); m.y = __vmaxu4(m.y, v.y); m.z = __vmaxu4(m.z, v.z); m.w = __vmaxu4(m.w, v.w);
+    if (kK > 0) {
+        uint4 v[kK > 0 ? kK * kK : 1];
+#pragma unroll
+        for (int i = 0; i < kK; ++i)
+#pragma unroll
+            for (int j = 0; j < kK; ++j) {
+                const int ih = oh * stride - pad + i, iw = ow * stride - pad + j;
+                const bool in = ih >= 0 && ih < hh && iw >= 0 && iw < ww;
+                v[i * kK + j] = in ? __ldg(reinterpret_cast<const uint4*>(x + ((static_cast<int64_t>(b) * hh + ih) * ww + iw) * pitch) + g)
+                                   : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+        for (int q = 0; q < kK * kK; ++q) {
+            m.x = __vmaxu4(m.x, v[q].x); m.y = __vmaxu4(m.y, v[q].y); m.z = __vmaxu4(m.z, v[q].z); m.w = __vmaxu4(m.w, v[q].w);
+        }
+    } else {
+        for (int i = 0; i < k; ++i) {
+            const int ih = oh * stride - pad + i;
+            if (ih < 0 || ih >= hh) continue;
+            for (int j = 0; j < k; ++j) {
+                const int iw = ow * stride - pad + j;
+                if (iw < 0 || iw >= ww) continue;
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + ((static_cast<int64_t>(b) * hh + ih) * ww + iw) * pitch) + g);
+                m.x = __vmaxu4(m.x, v.x); m.y = __vmaxu4(m.y, v.y); m.z = __vmaxu4(m.z, v.z); m.w = __vmaxu4(m.w, v.w);
+            }
         }
     }
     reinterpret_cast<uint4*>(y + ((static_cast<int64_t>(b) * oh_n + oh) * ow_n + ow) * pitch)[g] = m;
@@ -135,8 +155,14 @@ extern "C" qtz_status qtz_maxpool_u8(qtz_handle h, const uint8_t* x_dev, uint8_t
     const int oh_n = (hh + 2 * pad - k) / stride + 1, ow_n = (ww + 2 * pad - k) / stride + 1;
     if (oh_n <= 0 || ow_n <= 0) return QTZ_ERR_INVALID_ARG;
     const int64_t total = static_cast<int64_t>(batch) * oh_n * ow_n * (c_pitch >> 4);
-    maxpool_u8_kernel<<<static_cast<unsigned>(ceil_div(total, kThreads)), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        x_dev, y_dev, batch, hh, ww, c_pitch, k, stride, pad, oh_n, ow_n);
+    const unsigned blocks = static_cast<unsigned>(ceil_div(total, kThreads));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (k == 3)
+        maxpool_u8_kernel<3><<<blocks, kThreads, 0, st>>>(x_dev, y_dev, batch, hh, ww, c_pitch, k, stride, pad, oh_n, ow_n);
+    else if (k == 2)
+        maxpool_u8_kernel<2><<<blocks, kThreads, 0, st>>>(x_dev, y_dev, batch, hh, ww, c_pitch, k, stride, pad, oh_n, ow_n);
+    else
+        maxpool_u8_kernel<0><<<blocks, kThreads, 0, st>>>(x_dev, y_dev, batch, hh, ww, c_pitch, k, stride, pad, oh_n, ow_n);
     QTZ_LAUNCH_CHECK(h, "maxpool_u8_kernel");
     return QTZ_OK;
 }

@@ -174,7 +174,7 @@ def test_maxpool_and_global_avgpool(hq):
     got = host(hq.maxpool_u8(dev(x), 24, 3, 2, 1))
     assert got.shape == want.shape and np.array_equal(got[..., :24], want[..., :24])
     for shape, k, st, pad in [((2, 112, 112, 64), 3, 2, 1), ((1, 9, 12, 16), 3, 2, 0), ((2, 8, 7, 48), 3, 2, 2), ((1, 10, 10, 16), 2, 2, 0),
-                              ((1, 11, 9, 32), 3, 1, 1)]:
+                              ((1, 11, 9, 32), 3, 1, 1), ((2, 12, 13, 16), 5, 2, 2), ((1, 6, 6, 16), 1, 1, 0)]:
         xx = pitched(synth.uniform_u8(shape, 12, shape[1]))
         got = host(hq.maxpool_u8(dev(xx), shape[3], k, st, pad))
         assert np.array_equal(got, oracle.maxpool_u8(xx, k, st, pad, c=shape[3]))
