@@ -546,6 +546,32 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     clocks = sampler.stop()
     ms = t0.elapsed_time(t1)
+    # The same K steps replayed from a CUDA graph of one step (no host launch gaps between the ten kernels).
+    graph_ms = None
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for c in cases:
+                c.run()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for c in cases:
+                    c.run()
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(3):
+            g.replay()
+        barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for step in range(args.steps):
+            g.replay()
+        g1.record()
+        barrier()
+        graph_ms = g0.elapsed_time(g1)
+    except Exception as exc:   # capture is a convenience of the harness, not of the library
+        graph_ms = None
+        sys.stderr.write(f"graph replay skipped: {type(exc).__name__}: {exc}\n")
     # The same K steps once more with the library's profiling hook on: CUDA events on the launch stream around every
     # launch of the dominant kernel (and the activation-sum pre-pass it runs beside).  These per-launch durations
     # feed `roofline` and `sweep`; the events between launches cost a little, so this region is not the one timed above.
@@ -641,7 +667,8 @@ def run_ours(args, rank, world, local_rank):
         "config": {"workload": WORKLOAD if len(SIZES) == 5 else WORKLOAD + f" [subset {list(SIZES)}]", "parallelism": f"replicas x{world}",
                    "l2": "operands larger than L2: 268 MB touched per step, 201 MB by the largest size alone",
                    "kernels_per_step": "5 x (pixel_sum_kernel + conv_tc_kernel)",
-                   "per_launch_events": f"taken in a second pass of the same {args.steps} steps ({ms_profiled / args.steps:.4f} ms per step with the events)"},
+                   "per_launch_events": f"taken in a second pass of the same {args.steps} steps ({ms_profiled / args.steps:.4f} ms per step with the events)",
+                   "graph_replay_ms_per_step": None if graph_ms is None else round(graph_ms / args.steps, 4)},
         "clocks": clocks,
         "e2e": {"value": world * ops * e2e_steps / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                 "h2d_bytes_per_step": int(sum(c.a_host.numel() for c in cases)),
