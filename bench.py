@@ -337,6 +337,53 @@ def time_layer(hq, qtz, torch, spec, reps=20):
             "GB/s": round(nbytes / ms / 1e6, 1), "distinct_outputs": int(torch.unique(y[..., :n]).numel())}
 
 
+def time_block(hq, qtz, torch, spec, reps=20):
+    """One depthwise-separable block: spec = "batch,h,c,n,stride" (3x3 depthwise on h x h x c, then 1x1 to n channels,
+    both between ReLU6 tensors).  Times the depthwise kernel, the pointwise kernel, the two in a row and the fused
+    call qtz_conv2d_dw_pw_u8, each as a CUDA-graph replay of `reps` launches (profiling runs)."""
+    b, hh, c, n, stride = (int(v) for v in spec.split(","))
+    x = torch.randint(0, 256, (b, hh, hh, (c + 15) // 16 * 16), dtype=torch.uint8, device="cuda")
+    wd = torch.randint(-127, 128, (3, 3, c), dtype=torch.int8, device="cuda")
+    m, r = qtz.quantize_multiplier(1.0 / 600.0)
+    dw = hq.conv_create(qtz.conv_desc(b, hh, hh, c, c, 3, 3, stride, 1), wd, None, None, np.full(c, m, np.int32),
+                        np.full(c, r, np.int32), depthwise=True)
+    wp = torch.randint(-127, 128, (n, 1, 1, c), dtype=torch.int8, device="cuda")
+    m2, r2 = qtz.quantize_multiplier(1.0 / (40.0 * c ** 0.5 * 73.0))
+    pw = hq.conv_create(qtz.conv_desc(b, dw.oh, dw.ow, c, n, 1, 1, 1, 0), wp, None, None, np.full(n, m2, np.int32),
+                        np.full(n, r2, np.int32))
+    mid, y, y2 = dw.empty_output("cuda"), pw.empty_output("cuda"), pw.empty_output("cuda")
+
+    def replayed(fn):
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(reps):
+                    fn()
+        torch.cuda.current_stream().wait_stream(side)
+        g.replay(); torch.cuda.synchronize()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        for _ in range(5):
+            g.replay()
+        e.record(); torch.cuda.synchronize()
+        return round(s.elapsed_time(e) / (5 * reps) * 1e3, 1)
+
+    out = {"block": spec,
+           "depthwise_us": replayed(lambda: dw(x, 0, 0, 0, 255, out=mid)),
+           "pointwise_us": replayed(lambda: pw(mid, 0, 0, 0, 255, out=y)),
+           "both_us": replayed(lambda: (dw(x, 0, 0, 0, 255, out=mid), pw(mid, 0, 0, 0, 255, out=y)))}
+    try:
+        out["fused_us"] = replayed(lambda: pw.after_depthwise(dw, x, 0, 0, 0, 255, 0, 0, 255, out=y2))
+        out["fused_equals_both"] = bool(torch.equal(y, y2))
+        out["fused_kernel"] = pw.detail
+    except qtz.QtzError as exc:
+        out["fused_us"], out["fused_kernel"] = None, str(exc)
+    return out
+
+
 NETWORK_CONFIGS = [("mobilenet_v1", 128, 8), ("resnet50", 256, 8), ("mobilenet_v2_14", 256, 4)]
 
 
@@ -517,6 +564,9 @@ def run_ours(args, rank, world, local_rank):
         return
     if args.layer:
         print(json.dumps({"layers": [time_layer(hq, qtz, torch, sp) for sp in args.layer.split(";")]}), flush=True)
+        return
+    if args.block:
+        print(json.dumps({"blocks": [time_block(hq, qtz, torch, sp) for sp in args.block.split(";")]}), flush=True)
         return
     if args.networks_only:
         print(json.dumps({"networks": time_networks(hq, qtz, torch, peaks, detail=True)}), flush=True)
@@ -711,6 +761,7 @@ def main():
     ap.add_argument("--hbm-only", action="store_true",
                     help="run only the element-wise / depthwise kernel table (profiling runs); prints it as JSON")
     ap.add_argument("--layer", default="", help='time single conv layers: "batch,h,w,c,n,k,stride[,dw];..." (profiling runs)')
+    ap.add_argument("--block", default="", help='time depthwise-separable blocks, separate and fused: "batch,h,c,n,stride;..." (profiling runs)')
     ap.add_argument("--networks-only", action="store_true",
                     help="run only the whole-network timings, with per-layer times; prints them as JSON")
     ap.add_argument("--sizes", default="", help="comma-separated subset of the sweep (profiling runs); default: all")

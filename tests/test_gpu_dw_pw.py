@@ -60,6 +60,7 @@ def block_case(hq, b, h, w, c, n, stride, seed, z_x=None, mid=(0, 0, 255), out=(
     (2, 17, 19, 64, 32, 2),        # odd extents, stride 2, narrow output
     (1, 9, 9, 40, 24, 1),          # channels that fill neither a K block nor a 16-byte group
     (4, 7, 7, 256, 256, 1),        # tiles spanning several small images
+    (5, 7, 7, 64, 96, 1),          # ... whose last tile runs past the batch
 ])
 def test_block_shapes(hq, b, h, w, c, n, stride):
     block_case(hq, b, h, w, c, n, stride, seed=100 + c + n)
