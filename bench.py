@@ -333,7 +333,7 @@ def time_layer(hq, qtz, torch, spec, reps=20):
     oh, ow = plan.oh, plan.ow
     macs = b * oh * ow * n * k * k * (1 if dw else c)
     nbytes = b * hh * ww * c + b * oh * ow * n
-    return {"layer": spec, "kernel": plan.kernel, "ms": round(ms, 4), "TOP/s": round(2 * macs / ms / 1e9, 1),
+    return {"layer": spec, "kernel": plan.kernel, "detail": plan.detail, "ms": round(ms, 4), "TOP/s": round(2 * macs / ms / 1e9, 1),
             "GB/s": round(nbytes / ms / 1e6, 1), "distinct_outputs": int(torch.unique(y[..., :n]).numel())}
 
 

@@ -29,6 +29,7 @@
 // Every wait on an mbarrier is bounded; on expiry the kernel records a status word and returns.
 #include <algorithm>
 #include <new>
+#include <string>
 
 #include "qtz_dw_math.cuh"
 #include "qtz_plan.cuh"
@@ -489,6 +490,8 @@ qtz_status qtz_depthwise_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, uin
     const int mode = raw ? kModeRaw : ((p->rshift_max > 53 || p->rshift_min < 32) ? kModeGeneral : kModeFast);
     const bool clamp = !(act_min == 0 && act_max == 255);
     const DwKernel kernel = pick_kernel(d.stride, p->w_zp_signed != 0, mode, clamp);
+    p->detail = std::string("depthwise tile ") + std::to_string(a.tw) + "x" + std::to_string(a.th) + "x" + std::to_string(a.nb) +
+                " stages:" + std::to_string(a.stages);
     if (p->ev_start) QTZ_CUDA(p->h, cudaEventRecord(p->ev_start, st));
     {
         cudaLaunchConfig_t cfg = {};
