@@ -122,6 +122,12 @@ struct TcArgs {
     int64_t frame_row;                       // row-window layers: row pitch of the padded frame, its rows per image,
     int32_t frame_rows, seg_bytes;           // and the bytes of a frame row one tile takes
     int32_t a_blk;                           // bytes of one activation K block in the ring (0: 128 rows of BK bytes)
+    // Row-window layers with few output channels compute rrows consecutive output rows in one tile: the weight matrix
+    // holds rrows copies of the layer side by side (bn_row columns each), copy r shifted down by r * cstride frame rows,
+    // so that every frame row of the tile is multiplied once against all the output rows it feeds.  Column j of the
+    // accumulator is then channel j % bn_row of output row h0 + j / bn_row, and staging box r (bn_row bytes wide) is
+    // output row h0 + r.  (rrows = 1: an ordinary tile.)
+    int32_t rrows, bn_row;
     int32_t kb_per_tap, c_pad;
     int32_t BK, BN, N, out_box, stages, groups;   // groups: epilogue groups in use (1 or 2)
     int32_t obuf;                           // staging boxes per epilogue group (1..4)
@@ -294,7 +300,7 @@ __device__ __forceinline__ void tile_origin(const TcArgs& a, uint32_t m_tile, in
         const uint32_t q1 = fdiv(m_tile, a.dv_tiles_w);              // m_tile / tiles_w
         const uint32_t q2 = fdiv(q1, a.dv_tiles_h);                   // ... / tiles_h
         w0 = static_cast<int>(m_tile - q1 * a.dv_tiles_w.d) * a.tw;
-        h0 = static_cast<int>(q1 - q2 * a.dv_tiles_h.d) * a.th;
+        h0 = static_cast<int>(q1 - q2 * a.dv_tiles_h.d) * a.th * a.rrows;
         b0 = static_cast<int>(q2) * a.tb;
     } else {
         w0 = static_cast<int>(m_tile) * kTileM;
@@ -693,7 +699,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // the boxes of this group's tiles, in the order the epilogue fills them
             struct BoxIter {
                 uint32_t tile;
-                int nn, left, w0, h0, b0;
+                int nn, left, w0, h0, b0, bx;     // bx: index of the box in its tile (several output rows per tile: the row)
             };
             auto enter_tile = [&](BoxIter& it) {
                 // (a column tile that lies wholly beyond the real channels has no box at all: skip it)
@@ -703,6 +709,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     decode_tile(a, it.tile, m_tile, n_tile, prank);
                     it.nn = n_tile * a.BN;
                     it.left = a.BN;
+                    it.bx = 0;
                     if (it.nn >= a.N) continue;
                     tile_origin(a, m_tile, it.w0, it.h0, it.b0);
                     return;
@@ -711,7 +718,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             auto advance = [&](BoxIter& it) {
                 it.nn += a.out_box;
                 it.left -= a.out_box;
-                if (!(it.left > 0 && it.nn < a.N)) {
+                ++it.bx;
+                if (a.rrows > 1 ? it.bx >= a.rrows : !(it.left > 0 && it.nn < a.N)) {
                     it.tile += a.groups * tile_step;
                     enter_tile(it);
                 }
@@ -720,12 +728,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // "empty" barrier of the box carries the bytes of that copy
             auto fetch_shortcut = [&](uint32_t slot_, const BoxIter& it) {
                 mbar_arrive_expect_tx(oempty + 8 * slot_, static_cast<uint32_t>(a.rows * a.out_box));   // a box has a.rows rows
-                if (a.is4d)
+                if (a.rrows > 1)
+                    tma_load_4d(out_addr + slot_ * box_bytes, &map_s, oempty + 8 * slot_, 0, it.w0, it.h0 + it.bx, it.b0);
+                else if (a.is4d)
                     tma_load_4d(out_addr + slot_ * box_bytes, &map_s, oempty + 8 * slot_, it.nn, it.w0, it.h0, it.b0);
                 else
                     tma_load_2d(out_addr + slot_ * box_bytes, &map_s, oempty + 8 * slot_, it.nn, it.w0);
             };
-            BoxIter cur{tile0 + grp * tile_step, 0, 0, 0, 0, 0};
+            BoxIter cur{tile0 + grp * tile_step, 0, 0, 0, 0, 0, 0};
             enter_tile(cur);
             BoxIter ahead = cur;
             if (a.res)
@@ -749,7 +759,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     *abort_flag = 1;
                     break;
                 }
-                if (a.is4d)
+                if (a.rrows > 1)       // (rows past the image's last are clipped by the store)
+                    tma_store_4d(&map_y, out_addr + slot * box_bytes, 0, cur.w0, cur.h0 + cur.bx, cur.b0);
+                else if (a.is4d)
                     tma_store_4d(&map_y, out_addr + slot * box_bytes, cur.nn, cur.w0, cur.h0, cur.b0);
                 else
                     tma_store_2d(&map_y, out_addr + slot * box_bytes, cur.nn, cur.w0);
@@ -977,7 +989,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t ofull = bar_ofull + 8 * kMaxObuf * grp, oempty = bar_oempty + 8 * kMaxObuf * grp;
         uint32_t slot = 0, slot_phase = 0;                                           // box written next
         const int boxes = (a.BN + a.out_box - 1) / a.out_box;
-        const int half_cols = a.out_box / halves;    // 32, 64 or 128 columns per thread and box
+        const int half_cols = max(32, a.out_box / halves);   // 32, 64 or 128 columns per thread and box (a 32-byte box: one of the two warps)
         const int32_t span = a.act_max - a.act_min, off = a.zy - a.act_min;
         const uint32_t lo4 = 0x01010101u * static_cast<uint32_t>(a.act_min);
         const bool fold = a.fold != 0;
@@ -1049,7 +1061,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 // shift, and the rounding constant with the output offset folded in
                 named_barrier(bar_tbl, gthreads);            // everyone is done with the old tables
                 for (int j = gt; j < a.BN; j += gthreads) {
-                    const int n = n0 + j;
+                    const int n = a.rrows > 1 ? j % a.bn_row : n0 + j;      // (several output rows per tile: the layer's channels repeat)
                     const bool live = n < a.N;
                     const int32_t bias = live ? __ldg(a.bias + n) : 0;
                     const int32_t m = (live && !a.raw) ? __ldg(a.mult + n) : 0;
@@ -1137,7 +1149,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
             // uint8 output: one staging box (128 rows x out_box bytes) at a time
             for (int bx = 0; bx < boxes; ++bx) {
-                const int nn = n0 + bx * a.out_box;
+                // (several output rows per tile: box bx holds all channels of output row h0 + bx)
+                const int nn = a.rrows > 1 ? 0 : n0 + bx * a.out_box;
                 if (nn >= a.N) break;                // boxes entirely beyond the real channels
                 uint8_t* const dst = out_s + slot * box_bytes;
                 // the store that last used this box has read it
@@ -1151,7 +1164,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     dead = true;
                     break;
                 }
-                for (int col = half * half_cols; col < (half + 1) * half_cols && nn + col < a.N; col += 32) {
+                for (int col = half * half_cols; col < min((half + 1) * half_cols, a.out_box) && nn + col < a.N; col += 32) {
                     const int j0 = bx * a.out_box + col;
                     uint32_t v[32];
                     tmem_ld_32x32(taddr + j0, v);
@@ -1190,7 +1203,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     *p0 = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     *p1 = make_uint4(packed[4], packed[5], packed[6], packed[7]);
                 }
-                const bool drained = bx == boxes - 1 || nn + a.out_box >= a.N;
+                const bool drained = bx == boxes - 1 || (a.rrows == 1 && nn + a.out_box >= a.N);
                 if (drained) tc_fence_before();
                 fence_proxy_async_smem();            // this thread's box writes, for the TMA store
                 __syncwarp();
@@ -1392,20 +1405,24 @@ pad_copy_kernel(const uint8_t* __restrict__ x, uint8_t* __restrict__ xp, int bat
     reinterpret_cast<uint4*>(xp)[i] = make_uint4(words[0], words[1], words[2], words[3]);
 }
 
-// OHWI codes -> int8 [n_pad][kh][rb / fp pixels][fp bytes]: filter row dy of output channel `row` laid
+// OHWI codes -> int8 [n_pad][taps][rb / fp pixels][fp bytes]: filter row dy of output channel `row` laid
 // over the rb-byte run of frame pixels it meets; positions beyond kw pixels or c channels weigh zero.
+// With several output rows per tile (bn_row < n_pad) matrix row j is channel j % bn_row of output row j / bn_row of
+// the tile, and frame row f of the tile meets it with filter row f - (j / bn_row) * stride (zero outside 0 .. kh-1).
 __global__ void __launch_bounds__(kPrepThreads)
 prepack_rowwin_kernel(const void* __restrict__ w, int wkind, int n, int kh, int kw, int c, int n_pad, int fp, int rb,
-                      int8_t* __restrict__ out)
+                      int taps, int bn_row, int stride, int8_t* __restrict__ out)
 {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * kPrepThreads + threadIdx.x;
-    if (i >= static_cast<int64_t>(n_pad) * kh * rb) return;
+    if (i >= static_cast<int64_t>(n_pad) * taps * rb) return;
     const int byte = static_cast<int>(i % rb);
-    const int dy = static_cast<int>((i / rb) % kh);
-    const int64_t row = (i / rb) / kh;
+    const int f = static_cast<int>((i / rb) % taps);
+    const int64_t j = (i / rb) / taps;
+    const int64_t row = j % bn_row;
+    const int dy = f - static_cast<int>(j / bn_row) * stride;
     const int px = byte / fp, ch = byte % fp;
     int8_t v = 0;
-    if (row < n && px < kw && ch < c)
+    if (row < n && dy >= 0 && dy < kh && px < kw && ch < c)
         v = static_cast<int8_t>(qtz_dev::load_code_s8(w, wkind, row, (static_cast<int64_t>(dy) * kw + px) * c + ch, static_cast<int64_t>(kh) * kw * c));
     out[i] = v;
 }
@@ -1717,6 +1734,29 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     // every accumulator a tile ahead lets the MMA warp start a tile before an epilogue group is back
     a.n_acc = std::min(kMaxAcc, kTmemCols / a.BN);
     a.acc_stride = a.BN;
+    // Row-window layers with few output channels: several output rows per tile (see TcArgs::rrows).  As many rows (4 or
+    // 2) as keep the tile within 256 columns and the widened weights resident in shared memory.
+    a.rrows = 1;
+    a.bn_row = a.BN;
+    if (rw && a.n_tiles == 1 && d.outkind == QTZ_OUT_U8 && (a.BN == 32 || a.BN == 64 || a.BN == 128) && !h->single_row_stems) {
+        for (int r = 4; r >= 2; r >>= 1) {
+            const int taps_r = (r - 1) * d.stride + d.kh;
+            if (r * a.BN <= 256 && r <= p->oh && static_cast<int64_t>(taps_r) * r * a.BN * t->rb <= kResidentBMax) {
+                a.rrows = r;
+                break;
+            }
+        }
+        if (a.rrows > 1) {
+            a.out_box = a.BN;                                 // one staging box per output row
+            a.BN *= a.rrows;
+            a.taps = (a.rrows - 1) * d.stride + d.kh;          // frame rows a tile reads
+            a.n_acc = std::min(kMaxAcc, kTmemCols / a.BN);
+            a.acc_stride = a.BN;
+            // the frame reaches down to the last frame row of the last tile
+            const int tiles_h = (p->oh + a.rrows - 1) / a.rrows;
+            t->hp = std::max(t->hp, ((tiles_h * a.rrows - 1) * d.stride + d.kh + d.stride - 1) / d.stride * d.stride);
+        }
+    }
     t->n_pad = a.n_tiles * a.BN;
     a.ncls = (pw || rw) ? 1 : kMaxCls;
 
@@ -1740,7 +1780,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
             // a tile is a run of 128 output columns of one output row (columns beyond the image are
             // computed from whatever follows in the frame and clipped by the store)
             a.tw = kRunCols; a.th = 1; a.tb = 1;
-            best_tiles = static_cast<int64_t>((a.W + kRunCols - 1) / kRunCols) * a.H * a.B;
+            best_tiles = static_cast<int64_t>((a.W + kRunCols - 1) / kRunCols) * ((a.H + a.rrows - 1) / a.rrows) * a.B;
         } else {
             for (int tw = 1; tw <= std::min(a.W, kTileM); ++tw)
                 for (int th = 1; th <= std::min(a.H, kTileM / tw); ++th) {
@@ -1754,7 +1794,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
         }
         a.rows = a.tw * a.th * a.tb;
         a.tiles_w = (a.W + a.tw - 1) / a.tw;
-        a.tiles_h = (a.H + a.th - 1) / a.th;
+        a.tiles_h = (a.H + a.th * a.rrows - 1) / (a.th * a.rrows);
         if (best_tiles * a.n_tiles > 0x7fffffff) return QTZ_ERR_UNSUPPORTED;
         a.num_tiles = static_cast<uint32_t>(best_tiles * a.n_tiles);
     }
@@ -1817,7 +1857,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->w_packed), static_cast<size_t>(wbytes)));
     if (rw)
         prepack_rowwin_kernel<<<static_cast<unsigned>((wbytes + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
-            w_q_dev, d.wkind, d.n, d.kh, d.kw, d.c, t->n_pad, t->fp, t->rb, t->w_packed);
+            w_q_dev, d.wkind, d.n, d.kh, d.kw, d.c, t->n_pad, t->fp, t->rb, a.taps, a.rrows > 1 ? a.bn_row : t->n_pad, d.stride, t->w_packed);
     else
         prepack_tc_kernel<<<static_cast<unsigned>((wbytes + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
             w_q_dev, d.wkind, d.n, a.taps, d.c, t->n_pad, a.c_pad, t->w_packed, t->im2col ? t->cs : d.c, t->im2col ? p->d.c : d.c);
@@ -2080,7 +2120,8 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.w4_row = (a.taps * a.c_pad) >> 1;
     p->detail = std::string("tcgen05") + (t->rowwin ? " row-window" : (t->im2col ? " im2col" : (pw ? " pointwise" : " 3x3"))) +
                 (a.bres > 0 ? (a.w4 ? " weights:int4-expanded-in-smem" : " weights:resident") : " weights:streamed") +
-                (a.pair ? " cta-pairs" : "") + (a.res ? " +residual-add" : "");
+                (a.pair ? " cta-pairs" : "") + (a.rrows > 1 ? " rows-per-tile:" + std::to_string(a.rrows) : std::string()) +
+                (a.res ? " +residual-add" : "");
     if (p->ev_start && a.zw == 0) QTZ_CUDA(h, cudaEventRecord(p->ev_start, st));
     {
         // cluster of two for the pair form; early start beside pixel_sum_kernel when that kernel was just launched

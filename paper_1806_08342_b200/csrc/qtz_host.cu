@@ -37,6 +37,7 @@ extern "C" qtz_status qtz_create(qtz_handle* out, int device)
     if (!h) return QTZ_ERR_INVALID_ARG;
     h->device = device;
     if (const char* v = std::getenv("QTZ_NO_PAIRS")) h->no_pairs = v[0] == '1';
+    if (const char* v = std::getenv("QTZ_SINGLE_ROW_STEMS")) h->single_row_stems = v[0] == '1';
     cudaError_t e = cudaSetDevice(device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) e = cudaMalloc(&h->status_dev, 2 * sizeof(int32_t));

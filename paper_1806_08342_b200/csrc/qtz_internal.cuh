@@ -25,6 +25,7 @@ struct qtz_ctx {
     float* reduce_host = nullptr;  // pinned
     size_t reduce_host_bytes = 0;
     bool no_pairs = false;                  // never run layers on CTA pairs (A/B comparisons; set by QTZ_NO_PAIRS=1)
+    bool single_row_stems = false;          // row-window layers: one output row per tile (A/B comparisons; QTZ_SINGLE_ROW_STEMS=1)
     long long wait_budget = 2000000000LL;   // cycle budget of every bounded device-side wait (about one second)
     std::string last_error;
 };

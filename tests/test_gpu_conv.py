@@ -104,6 +104,8 @@ STEM_SHAPES = [
     (1, 23, 21, 3, 64, 7, 2, 3),      # ResNet stem shape
     (1, 20, 250, 3, 256, 7, 2, 3),    # stems whose weights do not stay resident (they share ring stages with the frame
     (1, 12, 14, 4, 272, 5, 2, 2),     # runs), several tiles per output row (125 columns), two column tiles
+    (2, 11, 260, 3, 32, 3, 2, 1),     # several output rows per tile, two tiles per output row, a ragged last row group
+    (1, 10, 12, 5, 32, 5, 1, 2),      # a stride-1 stem (16-byte frame pixels), four output rows per tile
     (1, 9, 9, 5, 7, 3, 1, 1),         # odd channel counts, n not a multiple of 4
     (3, 6, 7, 20, 70, 1, 1, 0),       # pointwise, ragged n tile
     (1, 8, 8, 16, 16, 3, 1, 0),       # no padding
