@@ -90,8 +90,41 @@ class ClockSampler:
 
     def __init__(self, index: int):
         self.index, self.lines, self.proc = index, [], None
+        self.nvml, self.samples, self.stop_flag, self.thread = None, [], False, None
+
+    def _poll(self):
+        """NVML polled from a thread: (SM MHz, max SM MHz, clock-event reason bits) per sample."""
+        nv, dev = self.nvml
+        try:
+            top = nv.nvmlDeviceGetMaxClockInfo(dev, nv.NVML_CLOCK_SM)
+        except Exception:
+            top = 0
+        while not self.stop_flag:
+            try:
+                self.samples.append((nv.nvmlDeviceGetClockInfo(dev, nv.NVML_CLOCK_SM), top,
+                                     nv.nvmlDeviceGetCurrentClocksEventReasons(dev)))
+            except Exception:
+                break
+            time.sleep(0.001)
 
     def start(self):
+        # the timed region of the default run lasts a few milliseconds: poll NVML directly where it is available
+        # (same counters as nvidia-smi's clocks.sm / clocks_event_reasons), else fall back to nvidia-smi at 100 ms
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            idx = self.index
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            if vis and all(v.strip().isdigit() for v in vis.split(",")) and idx < len(vis.split(",")):
+                idx = int(vis.split(",")[idx])
+            dev = nv.nvmlDeviceGetHandleByIndex(idx)
+            nv.nvmlDeviceGetCurrentClocksEventReasons(dev)
+            self.nvml = (nv, dev)
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
                                           "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
@@ -104,6 +137,19 @@ class ClockSampler:
             self.lines.append(line.strip())
 
     def stop(self):
+        if self.nvml is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=1.0)
+            nv = self.nvml[0]
+            names = (("hw_slowdown", getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8)),
+                     ("hw_thermal_slowdown", getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40)),
+                     ("sw_thermal_slowdown", getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20)),
+                     ("sw_power_cap", getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)))
+            reasons = sorted({n for _, _, bits in self.samples for n, mask in names if bits & mask})
+            busy = [c for c, _, _ in self.samples if c > 0]
+            return {"sm_mhz": float(np.median(busy)) if busy else None,
+                    "sm_max_mhz": float(max(m for _, m, _ in self.samples)) if self.samples else None,
+                    "reasons": reasons, "samples": len(self.samples), "source": "nvml polled back to back"}
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.15)
