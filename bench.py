@@ -472,12 +472,14 @@ def roofline_sum_ms(ops, batch, wbits, peaks, resolution=224):
     return total * 1e3
 
 
-def time_networks(hq, qtz, torch, peaks, reps=10, detail=False):
+def time_networks(hq, qtz, torch, peaks, reps=10, detail=False, only=""):
     """Images/s of whole-network integer inference at the batch sizes of the network workloads
     (calibration and plan creation outside the timed region; activations stay in HBM)."""
     from paper_1806_08342_b200 import network
     res = {}
     for name, batch, wbits in NETWORK_CONFIGS:
+        if only and name not in only.split(","):
+            continue
         ops = synth.NETWORKS[name]()
         images = synth.network_input(batch, 224, 12)
         net = network.QuantizedNetwork(hq, ops, 12, wbits)
@@ -618,7 +620,8 @@ def run_ours(args, rank, world, local_rank):
         print(json.dumps({"blocks": [time_block(hq, qtz, torch, sp) for sp in args.block.split(";")]}), flush=True)
         return
     if args.networks_only:
-        print(json.dumps({"networks": time_networks(hq, qtz, torch, peaks, detail=True)}), flush=True)
+        print(json.dumps({"networks": time_networks(hq, qtz, torch, peaks, reps=args.network_reps, detail=True,
+                                                    only=args.networks)}), flush=True)
         return
     cases = [GemmCase(hq, qtz, torch, s) for s in SIZES]
     torch.cuda.synchronize()
@@ -816,6 +819,8 @@ def main():
     ap.add_argument("--block", default="", help='time depthwise-separable blocks, separate and fused: "batch,h,c,n,stride;..." (profiling runs)')
     ap.add_argument("--networks-only", action="store_true",
                     help="run only the whole-network timings, with per-layer times; prints them as JSON")
+    ap.add_argument("--networks", default="", help="with --networks-only: comma-separated subset of the networks (profiling runs)")
+    ap.add_argument("--network-reps", type=int, default=10, help="with --networks-only: timed passes per network")
     ap.add_argument("--sizes", default="", help="comma-separated subset of the sweep (profiling runs); default: all")
     args = ap.parse_args()
     if args.sizes:
