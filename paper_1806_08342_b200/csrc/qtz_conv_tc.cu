@@ -1522,6 +1522,7 @@ struct qtz_tc_state {
     TcArgs args{};
     qtz_conv_desc eff{};       // the layer as the kernel sees it (im2col layers become pointwise over the window matrix)
     bool im2col = false;
+    bool strided_view = false; // strided 1x1 layer read through a strided tensor map (no gather pre-pass)
     bool rowwin = false;       // row-window layer: padded frame read through a sliding operand descriptor (see pad_copy_kernel)
     int hp = 0, wp = 0;        // its frame extent
     int fp = 16, rb = 128;     // bytes per frame pixel, bytes of one filter-row run
@@ -1761,7 +1762,12 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.ncls = (pw || rw) ? 1 : kMaxCls;
 
     // pixel tiling
-    if (pw) {
+    // (a strided 1x1 layer with symmetric weights reads its input through a strided view of the tensor -- every
+    //  stride-th pixel of every stride-th row -- and is tiled as boxes of that view; with a weight zero point the
+    //  activation sums need the compacted copy, so those layers gather first)
+    const bool strided_view = pw && d.stride > 1 && p->w_zp_signed == 0;
+    t->strided_view = strided_view;
+    if (pw && !strided_view) {
         a.is4d = 0;
         a.tw = kTileM; a.th = 1; a.tb = 1; a.rows = kTileM;
         a.tiles_w = static_cast<int32_t>((t->in_pixels + kTileM - 1) / kTileM);
@@ -1811,7 +1817,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
     a.pair = 0;
     // (measured: layers of the networks with K = 1024..2048 and a few hundred tiles, which are bound by HBM and by
     //  latency rather than by the tensor cores, run about 10 % slower on pairs, so the bar is set above them)
-    if (pw && a.BN == 256 && d.c >= 2048 && d.n >= 2048 && a.num_tiles >= 2 * static_cast<uint32_t>(h->num_sms) && !h->no_pairs) {
+    if (pw && !strided_view && a.BN == 256 && d.c >= 2048 && d.n >= 2048 && a.num_tiles >= 2 * static_cast<uint32_t>(h->num_sms) && !h->no_pairs) {
         int clusters = 0;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(static_cast<unsigned>(h->num_sms / 2 * 2));
@@ -1877,7 +1883,7 @@ qtz_status qtz_tc_prepare(qtz_plan* p, const void* w_q_dev, cudaStream_t st)
 
     if (p->w_zp_signed != 0)
         QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&t->xsum), sizeof(int32_t) * static_cast<size_t>(t->in_pixels)));
-    if ((pw && d.stride > 1) || t->im2col)
+    if ((pw && d.stride > 1 && !strided_view) || t->im2col)
         QTZ_CUDA(h, cudaMalloc(reinterpret_cast<void**>(&p->x_gather), static_cast<size_t>(t->in_pixels) * d.c_pitch_in));
     if (rw) {
         // the last tiles of a row read past its end (into the next row, or into this slack after the last one)
@@ -1961,7 +1967,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
             x, p->x_gather, o.h, o.w, o.c, t->cs, o.c_pitch_in, o.kh, o.kw, o.stride, o.pad, p->oh, p->ow, tp, d.c, d.c_pitch_in, x_zp);
         QTZ_LAUNCH_CHECK(h, "im2col_kernel");
         xin = p->x_gather;
-    } else if (pw && d.stride > 1) {
+    } else if (pw && d.stride > 1 && !t->strided_view) {
         const int64_t work = t->in_pixels * (d.c_pitch_in >> 4);
         stride_gather_kernel<<<static_cast<unsigned>((work + kPrepThreads - 1) / kPrepThreads), kPrepThreads, 0, st>>>(
             x, p->x_gather, d.batch, d.h, d.w, d.c_pitch_in, d.stride, p->oh, p->ow);
@@ -1991,6 +1997,15 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     const uint64_t pitch = static_cast<uint64_t>(d.c_pitch_in);
     if (t->rowwin) {
         map_a = t->map_b;   // encoded below, once the number of filter rows per ring stage is known
+    } else if (t->strided_view) {
+        // every stride-th pixel of every stride-th row, as a tensor of the output's extent
+        const uint64_t sv = static_cast<uint64_t>(p->d.stride);
+        const uint64_t dims[4] = {static_cast<uint64_t>(d.c), static_cast<uint64_t>(p->ow), static_cast<uint64_t>(p->oh),
+                                  static_cast<uint64_t>(d.batch)};
+        const uint64_t strides[3] = {pitch * sv, pitch * p->d.w * sv, pitch * p->d.w * p->d.h};
+        const uint32_t box[4] = {static_cast<uint32_t>(a.BK), static_cast<uint32_t>(a.tw), static_cast<uint32_t>(a.th),
+                                 static_cast<uint32_t>(a.tb)};
+        if (!encode_map(&map_a, xin, 4, dims, strides, box, a.BK)) return QTZ_ERR_CUDA;
     } else if (pw) {
         const uint64_t dims[2] = {static_cast<uint64_t>(d.c), static_cast<uint64_t>(t->in_pixels)};
         const uint64_t strides[1] = {pitch};
@@ -2010,7 +2025,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
         a.y_raw = static_cast<int32_t*>(y);
     } else {
         const uint64_t opitch = static_cast<uint64_t>(d.c_pitch_out);
-        if (pw) {
+        if (pw && !t->strided_view) {
             const uint64_t dims[2] = {static_cast<uint64_t>(d.n), static_cast<uint64_t>(t->in_pixels)};
             const uint64_t strides[1] = {opitch};
             const uint32_t box[2] = {static_cast<uint32_t>(a.out_box), static_cast<uint32_t>(kTileM)};
@@ -2118,7 +2133,7 @@ qtz_status qtz_tc_launch(qtz_plan* p, const uint8_t* x, int32_t x_zp, void* y, i
     a.full_count = a.lsu ? (a.bres > 0 ? 1 : 2) : 1;
     a.w4 = (t->w_packed4 && a.bres > 0) ? t->w_packed4 : nullptr;
     a.w4_row = (a.taps * a.c_pad) >> 1;
-    p->detail = std::string("tcgen05") + (t->rowwin ? " row-window" : (t->im2col ? " im2col" : (pw ? " pointwise" : " 3x3"))) +
+    p->detail = std::string("tcgen05") + (t->rowwin ? " row-window" : (t->im2col ? " im2col" : (pw ? (t->strided_view ? " pointwise strided-view" : " pointwise") : " 3x3"))) +
                 (a.bres > 0 ? (a.w4 ? " weights:int4-expanded-in-smem" : " weights:resident") : " weights:streamed") +
                 (a.pair ? " cta-pairs" : "") + (a.rrows > 1 ? " rows-per-tile:" + std::to_string(a.rrows) : std::string()) +
                 (a.res ? " +residual-add" : "");

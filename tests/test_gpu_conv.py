@@ -146,6 +146,8 @@ TC_SHAPES = [
     (1, 16, 16, 256, 272, 1, 1, 0),   # two K blocks, N beyond one 256 tile
     (2, 9, 9, 512, 24, 1, 1, 0),      # long K, narrow N
     (1, 12, 12, 64, 32, 1, 2, 0),     # strided pointwise (ResNet down-sampling shortcut)
+    (3, 15, 13, 256, 512, 1, 2, 0),   # ... odd extents, several images, two K blocks, two column tiles
+    (2, 56, 56, 40, 72, 1, 3, 0),     # ... stride 3, many pixel tiles
     (2, 24, 24, 32, 128, 1, 1, 0),    # pointwise outputs of 128, 192, 256 and 8 channels: whole tiles leave as one
     (1, 40, 40, 48, 192, 1, 1, 0),    # contiguous run (rows of 8, 12, 16 and 1 sixteen-byte pieces, staged in
     (1, 30, 30, 64, 256, 1, 1, 0),    # rotated order), several tiles and a short last one
