@@ -93,7 +93,10 @@ typedef struct {
 /* ---- library ------------------------------------------------------------------------- */
 
 /* Creates a handle bound to CUDA device `device` (allocates a few MB of device scratch).
- * Blocking.  QTZ_ERR_NO_DEVICE when the device cannot be used.                            */
+ * Blocking.  QTZ_ERR_NO_DEVICE when the device cannot be used.
+ * Two environment variables, read here, switch scheduling choices off for A/B timing (results are the
+ * same either way): QTZ_NO_PAIRS=1 keeps large GEMM-like layers on single CTAs instead of CTA pairs;
+ * QTZ_SINGLE_ROW_STEMS=1 keeps image stems at one output row per tile.                      */
 QTZ_API qtz_status qtz_create(qtz_handle* out, int device);
 QTZ_API qtz_status qtz_destroy(qtz_handle h);
 QTZ_API const char* qtz_status_string(qtz_status s);
